@@ -1,0 +1,180 @@
+/*
+ * sj.h -- C ABI of the B200 (sm_100a) verification step for judge speculative decoding.
+ *
+ * One call, sj_verify(), runs the target decoder over the block [x_t, d_1 .. d_gamma] of each
+ * sequence against a paged KV cache (Eq. 2), forms the target probabilities p and the final
+ * hidden states h (Eq. 4), applies the probability-ratio acceptance test (Eq. 3; at
+ * temperature 0 the strict "draft == target greedy token" test of Sec. 3.1), the judge
+ * verifier  Verifier(h) = sigmoid(w.h + b) > theta  (Eq. 5), accepts a token if EITHER test
+ * passes (Sec. 3.2, App. D.2), stops at the first rejection (Sec. 3.1), emits the next token
+ * and sets the cache length.  Every step runs in hand-written CUDA kernels; there is no CPU
+ * fallback: without a CUDA device every compute call returns SJ_ERR_CUDA.
+ *
+ * Conventions
+ *   - All matrices are row-major [out_features, in_features] (y = W x), dtype = config.dtype.
+ *   - "device" pointers are CUDA device pointers on the device current at sj_create_target();
+ *     "host" pointers are ordinary host memory.  The caller owns every buffer it passes in.
+ *     Weights are BORROWED: they must stay valid and unchanged for the life of the handle.
+ *   - The library owns its handles, the KV page pool and its workspace (cudaMalloc'ed at
+ *     creation / first use, freed by the destroy calls).
+ *   - Every call returns an sj_status; sj_last_error() gives a message for the calling thread.
+ *     Argument errors are detected on the host before any launch.  sj_verify() and
+ *     sj_rollback_kv() are asynchronous on the target's stream; errors only the device can see
+ *     (a bounded wait that ran out, a rollback beyond the true length) are recorded in a device
+ *     status word and returned by the next sj_sync().
+ *   - One stream per target; calls on one handle are not re-entrant.
+ *   - Row j (0..gamma) of a sequence's block: row 0's input is the pending token x_t (set by
+ *     sj_kv_set_pending() or by the previous committed sj_verify()), row j>=1's input is d_j.
+ *     Row j sits at absolute position kv_len + j.  Row j's logits are the target distribution for
+ *     drafted position j+1 (row gamma: the bonus token); row j's final hidden state is the judge
+ *     input for d_j.
+ */
+#ifndef SJ_H_
+#define SJ_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SJ_OK = 0,
+  SJ_ERR_INVALID_ARG = 1, /* null pointer, value out of range */
+  SJ_ERR_SHAPE = 2,       /* dimensions the kernels do not support */
+  SJ_ERR_STATE = 3,       /* call not valid in the handle's current state */
+  SJ_ERR_OOM = 4,         /* page pool or device memory exhausted (nothing was launched) */
+  SJ_ERR_UNSUPPORTED = 5,
+  SJ_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed (includes "no device") */
+  SJ_ERR_TIMEOUT = 7      /* a bounded device-side wait ran out */
+} sj_status;
+
+typedef struct sj_target sj_target; /* config + borrowed weights + judge head + workspace */
+typedef struct sj_kv sj_kv;         /* page pool, block tables, kv_len[], pending[] */
+
+enum { SJ_DTYPE_F32 = 0, SJ_DTYPE_BF16 = 1 };
+enum { SJ_MODE_GREEDY = 0, SJ_MODE_SAMPLING = 1 };
+
+enum {
+  SJ_MAX_BATCH = 256,  /* sequences per sj_verify() call */
+  SJ_MAX_GAMMA = 31,   /* drafted tokens per sequence */
+  SJ_MAX_ROWS = 512    /* B * (gamma + 1) */
+};
+
+/* Decoder shape.  Pre-norm decoder: RMSNorm, rotary embedding (rotate-half pairing, angle
+ * pos * rope_theta^(-2i/head_dim)), grouped-query attention, SwiGLU FFN -- the Llama-3 /
+ * Qwen-2.5 family the paper evaluates (Sec. 4).  max_rows sizes the workspace: the largest
+ * B*(gamma+1) any sj_verify() call will use (0 -> 64). */
+typedef struct {
+  int n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+  float rope_theta, rms_eps;
+  int dtype;            /* SJ_DTYPE_*: storage type of weights, activations and the KV cache */
+  int tied_embeddings;  /* informational; pass the same pointer for embed and lm_head */
+  int qkv_bias;         /* 1: bq/bk/bv are read */
+  int max_rows;
+} sj_model_config;
+
+/* Device pointers to the weights; the per-layer members are HOST arrays of n_layers device
+ * pointers (the arrays themselves are copied, the tensors are borrowed).
+ *   embed, lm_head [vocab, d_model]; final_norm, norm_attn[l], norm_ffn[l] [d_model];
+ *   wq [Hq*hd, d]; wk, wv [Hkv*hd, d]; wo [d, Hq*hd]; w_gate, w_up [d_ffn, d]; w_down [d, d_ffn];
+ *   bq [Hq*hd]; bk, bv [Hkv*hd] (may be NULL when qkv_bias == 0).
+ * bf16 matrices must be 16-byte aligned. */
+typedef struct {
+  const void *embed, *lm_head, *final_norm;
+  const void *const *wq, *const *wk, *const *wv, *const *wo, *const *w_gate, *const *w_up, *const *w_down;
+  const void *const *norm_attn, *const *norm_ffn;
+  const void *const *bq, *const *bk, *const *bv;
+} sj_weights;
+
+/* Create a target on the current CUDA device.  cuda_stream is a cudaStream_t (NULL: the legacy
+ * default stream) on which all work of this handle and of its KV objects is issued.
+ * Errors: INVALID_ARG (null / non-positive dims), SHAPE (head_dim not in {64,128}, odd group,
+ * dims not multiples of 8 ...), CUDA, OOM. */
+sj_status sj_create_target(const sj_model_config *cfg, const sj_weights *w, void *cuda_stream, sj_target **out);
+sj_status sj_destroy_target(sj_target *t);
+
+/* Judge verifier head of Eq. 5: score = sigmoid(w . h + bias), accept when score > theta
+ * (strict).  w: [d_model] fp32, host memory (copied).  The hidden state h is the last layer's
+ * output after the final RMSNorm.  Until this is called the judge test never fires. */
+sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, float theta);
+
+/* Runtime switches (for tests and measurements).  Names:
+ *   "gemm_impl"  0 = CUDA-core kernels, 1 = tcgen05/TMA kernels (bf16 only; default for bf16)
+ *   "attn_impl"  0 = CUDA-core kernel,  1 = tensor-core kernel  (bf16 only; default for bf16)
+ *   "graph"      1 = replay the step as a CUDA graph (default), 0 = plain launches
+ *   "pdl"        1 = programmatic dependent launch between the step's kernels (default)
+ * Errors: INVALID_ARG for an unknown name, UNSUPPORTED for a value the dtype cannot honour. */
+sj_status sj_set_option(sj_target *t, const char *name, int value);
+
+/* Wait for the target's stream and return the device status word (SJ_OK, SJ_ERR_TIMEOUT,
+ * SJ_ERR_STATE ...), clearing it. */
+sj_status sj_sync(sj_target *t);
+
+/* Paged KV cache for up to max_seqs sequences sharing max_pages pages of page_size (16) tokens.
+ * A page holds, per layer, K and V rows [Hkv, page_size, head_dim] in the model dtype; keys are
+ * stored AFTER the rotary embedding. */
+sj_status sj_kv_create(sj_target *t, int max_seqs, long max_pages, int page_size, sj_kv **out);
+sj_status sj_kv_destroy(sj_kv *kv);
+
+/* Write n_tokens cache rows of one layer of one sequence starting at token index `start`,
+ * reserving pages as needed.  k, v: device, [n_tokens, Hkv, head_dim], model dtype, K already
+ * rotated.  Does not change the sequence length.  Errors: OOM (pool exhausted), INVALID_ARG. */
+sj_status sj_kv_fill(sj_kv *kv, int seq, int layer, int start, int n_tokens, const void *k, const void *v);
+/* Read rows back (same layout); synchronises the stream.  For tests. */
+sj_status sj_kv_read(sj_kv *kv, int seq, int layer, int start, int n_tokens, void *k_out, void *v_out);
+/* Set the length of sequences (tokens [0,len) are live).  len must not exceed the rows reserved
+ * by fills/verifies.  seq_ids, lens: host [B]. */
+sj_status sj_kv_set_len(sj_kv *kv, const int *seq_ids, const int *lens, int B);
+/* Set the pending token x_t of sequences (fed at row 0 of the next block).  host [B]. */
+sj_status sj_kv_set_pending(sj_kv *kv, const int *seq_ids, const int *tokens, int B);
+/* Current lengths (host out[B]); synchronises the stream and returns unused pages to the pool. */
+sj_status sj_kv_len(sj_kv *kv, const int *seq_ids, int *out_len, int B);
+
+typedef struct {
+  int B, gamma;
+  const int *seq_ids;        /* host   [B] distinct sequence slots of the sj_kv */
+  const int *draft_ids;      /* device [B, gamma]      d_1..d_gamma */
+  const float *draft_q_tok;  /* device [B, gamma]      q_j(d_j); required iff mode == SAMPLING */
+  const float *draft_q_full; /* device [B, gamma, V]   full draft distributions; required iff SAMPLING */
+  const float *uniforms;     /* device [B, gamma+1]    [:, :gamma] = u_1..u_gamma of Eq. 3,
+                                                       [:, gamma] drives the emitted token; iff SAMPLING */
+  int mode;                  /* SJ_MODE_GREEDY (temperature 0, the paper's setting) or SJ_MODE_SAMPLING */
+  float temperature;         /* SAMPLING: p = softmax(logits / temperature), > 0 */
+  int use_align, use_judge;  /* which of the two tests may accept (App. D.2 ablation) */
+  float theta_override;      /* >= 0: use instead of the loaded theta */
+  int commit;                /* 1: kv_len <- kv_len + 1 + accepted_len, pending <- next_token */
+} sj_verify_args;
+
+typedef struct {
+  int *accepted_len;    /* device [B]         n = number of drafts accepted before the first rejection */
+  int *next_token;      /* device [B]         greedy: argmax of row n (lowest id on ties); sampling: inverse
+                                              CDF (vocab order, uniforms[:,gamma]) of norm(max(0, p_n - q_{n+1}))
+                                              when n < gamma, of p_gamma otherwise */
+  float *judge_scores;  /* device [B, gamma]  sigmoid scores of d_1..d_gamma (all positions) */
+  float *p_draft;       /* device [B, gamma]  p_j(d_j) (at temperature 1 in greedy mode) */
+  int *new_kv_len;      /* device [B]         kv_len + 1 + n */
+  float *dbg_hidden;    /* device [B, gamma+1, d_model] or NULL: hidden states after the final norm */
+  float *dbg_logits;    /* device [B, gamma+1, vocab]   or NULL: raw logits (tests only) */
+} sj_verify_out;
+
+/* One verification step (see the file comment).  Appends gamma+1 K/V rows per sequence at
+ * [kv_len, kv_len+gamma]; with commit the sequence keeps the first 1+n of them.
+ * Errors before launch: INVALID_ARG, SHAPE (B*(gamma+1) > max_rows), OOM (page pool), STATE. */
+sj_status sj_verify(sj_target *t, sj_kv *kv, const sj_verify_args *args, const sj_verify_out *out);
+
+/* Truncate sequences to new_len <= current length (host arrays [B]).  Asynchronous; if new_len
+ * exceeds the true length the device leaves the sequence unchanged and sj_sync() returns
+ * SJ_ERR_STATE.  new_len above what the host knows could be live fails at once with STATE. */
+sj_status sj_rollback_kv(sj_kv *kv, const int *seq_ids, const int *new_len, int B);
+
+/* Skinny GEMM used by every projection of the step, exposed for kernel-level tests and
+ * measurement:  y[R, N] (fp32) = a[R, K] . w[N, K]^T,  a and w in `dtype`, device pointers.
+ * impl as in "gemm_impl".  Synchronous with respect to `cuda_stream` ordering only. */
+sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, const void *a, const void *w, float *y,
+                         void *cuda_stream);
+
+const char *sj_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SJ_H_ */

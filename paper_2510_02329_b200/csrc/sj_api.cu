@@ -1,0 +1,981 @@
+// Host runtime and C ABI of the verification step: handles, paged-KV bookkeeping, argument checks,
+// launch sequence (optionally replayed as a CUDA graph with programmatic dependent launches).
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/sj.h"
+#include "sj_gemm_tc.cuh"
+
+using namespace sj;
+
+// ---------------------------------------------------------------------------------------------
+// errors
+// ---------------------------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+static sj_status fail(sj_status st, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return st;
+}
+
+#define CU_TRY(expr)                                                                              \
+  do {                                                                                            \
+    cudaError_t e_ = (expr);                                                                      \
+    if (e_ != cudaSuccess) {                                                                      \
+      cudaGetLastError();                                                                         \
+      return fail(e_ == cudaErrorMemoryAllocation ? SJ_ERR_OOM : SJ_ERR_CUDA, "%s: %s", #expr,    \
+                  cudaGetErrorString(e_));                                                        \
+    }                                                                                             \
+  } while (0)
+
+extern "C" const char* sj_last_error(void) { return g_err; }
+
+// ---------------------------------------------------------------------------------------------
+// launch helper (programmatic dependent launch attribute on request)
+// ---------------------------------------------------------------------------------------------
+template <typename... KArgs, typename... Args>
+static cudaError_t launch(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                          Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(std::forward<Args>(args))...);
+}
+
+// ---------------------------------------------------------------------------------------------
+// TMA descriptors (driver entry point fetched at run time: no link-time dependency on libcuda)
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+static sj_status get_encode() {
+  if (g_encode) return SJ_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  CU_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+  if (!fn || qres != cudaDriverEntryPointSuccess) return fail(SJ_ERR_CUDA, "cuTensorMapEncodeTiled not available");
+  g_encode = (EncodeTiledFn)fn;
+  return SJ_OK;
+}
+
+// bf16 row-major [rows, K] matrix, box = [box_rows, 64] with 128-byte swizzle, zero fill out of bounds
+static sj_status make_map(CUtensorMap* tm, const void* base, long rows, long K, int box_rows) {
+  sj_status st = get_encode();
+  if (st != SJ_OK) return st;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) != 0 || (K * 2) % 16 != 0)
+    return fail(SJ_ERR_INVALID_ARG, "bf16 matrix must be 16-byte aligned with K a multiple of 8");
+  cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t gstr[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(SJ_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", (int)r);
+  return SJ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// tensor-core GEMM sites
+// ---------------------------------------------------------------------------------------------
+struct TcSite {
+  // static per site
+  int N = 0, K = 0, n_tiles = 0, KB = 0, G = 0, nseg = 0;
+  int seg_tile_end[3] = {0, 0, 0};
+  int max_slots = 1;
+  int2* d_tile_slots = nullptr;
+  bool lm = false;
+};
+
+static int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// Which blocks contribute to which tile (must mirror the kernel's u_lo/u_hi arithmetic).
+static void build_tile_slots(int n_tiles, int KB, int G, std::vector<int2>& out, int& max_slots) {
+  long long U = (long long)n_tiles * KB;
+  out.assign(n_tiles, make_int2(0, 0));
+  std::vector<int> first(n_tiles, -1), cnt(n_tiles, 0);
+  for (int c = 0; c < G; ++c) {
+    long long lo = (long long)c * U / G, hi = (long long)(c + 1) * U / G;
+    if (hi <= lo) continue;
+    int t0 = (int)(lo / KB), t1 = (int)((hi - 1) / KB);
+    for (int t = t0; t <= t1; ++t) {
+      if (first[t] < 0) first[t] = c;
+      cnt[t] = c - first[t] + 1;
+    }
+  }
+  max_slots = 1;
+  for (int t = 0; t < n_tiles; ++t) {
+    out[t] = make_int2(first[t], cnt[t]);
+    max_slots = std::max(max_slots, cnt[t]);
+  }
+}
+
+struct RowGeom {  // how R activation rows are fed to the MMA
+  int NB, nblk, acc_stride, acc_bufs, stages, a_stage_bytes;
+  uint32_t tmem_cols;
+  size_t smem_bytes;
+};
+
+static RowGeom row_geom(int R) {
+  RowGeom g;
+  int rp = round_up(std::max(R, 1), 16);
+  g.NB = rp > 256 ? 2 : 1;
+  g.nblk = round_up((rp + g.NB - 1) / g.NB, 16);
+  int cols = g.NB * g.nblk;
+  g.acc_bufs = (2 * cols <= 512) ? 2 : 1;
+  g.acc_stride = cols;
+  uint32_t need = (uint32_t)(cols * g.acc_bufs), tc = 32;
+  while (tc < need) tc <<= 1;
+  g.tmem_cols = tc;
+  g.a_stage_bytes = round_up(cols * 128, 1024);
+  int stage = kWTileBytes + g.a_stage_bytes;
+  const int budget = 200 * 1024;
+  g.stages = std::max(2, std::min(12, budget / stage));
+  g.smem_bytes = (size_t)g.stages * stage + sizeof(TcSmemCtl) + 1024;
+  return g;
+}
+
+// ---------------------------------------------------------------------------------------------
+// handles
+// ---------------------------------------------------------------------------------------------
+struct LayerW {
+  const void *wq, *wk, *wv, *wo, *wg, *wu, *wd, *na, *nf, *bq, *bk, *bv;
+  CUtensorMap m_q, m_k, m_v, m_o, m_g, m_u, m_d;
+};
+
+struct StepKey {
+  int B, gamma, mode, chunk_len, gemm_impl, attn_impl, pdl, scratch;
+  bool operator<(const StepKey& o) const {
+    return std::tie(B, gamma, mode, chunk_len, gemm_impl, attn_impl, pdl, scratch) <
+           std::tie(o.B, o.gamma, o.mode, o.chunk_len, o.gemm_impl, o.attn_impl, o.pdl, o.scratch);
+  }
+};
+
+struct sj_target {
+  sj_model_config cfg;
+  Dims dm;
+  cudaStream_t stream = nullptr;
+  int device = 0, sm_count = 0, max_rows = 64;
+  bool bf = false;
+  const void *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  CUtensorMap m_lm;
+  std::vector<LayerW> layers;
+  Work work;
+  StepArgs* d_args = nullptr;
+  float* d_judge_w = nullptr;
+  double* d_inv_freq = nullptr;
+  float theta = 0.5f, judge_bias = 0.f;
+  bool has_judge = false;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1;
+  TcSite s_qkv, s_o, s_gu, s_down, s_lm;
+  size_t p_elems = 0;
+  size_t att_chunks_cap = 0;
+  int att_rows_cap = 0;
+  size_t logits_rows = 0;
+  std::map<StepKey, cudaGraphExec_t> graphs;
+  std::map<int, CUtensorMap> mapA_d, mapA_q, mapA_f;  // activation maps per R
+  std::vector<void*> owned;
+};
+
+struct sj_kv {
+  sj_target* t = nullptr;
+  KvView view;
+  int max_seqs = 0;
+  long max_pages = 0;
+  std::vector<std::vector<int>> pages;  // per sequence
+  std::vector<int> free_pages;
+  std::vector<int> len_hi;              // upper bound of the live length known to the host
+  std::vector<char> exact;              // len_hi is the exact length
+  int* d_block_table = nullptr;
+  int* d_tmp = nullptr;                 // [2 * SJ_MAX_BATCH] staging for rollback / set_len
+};
+
+static void clear_graphs(sj_target* t) {
+  for (auto& kvp : t->graphs) cudaGraphExecDestroy(kvp.second);
+  t->graphs.clear();
+}
+
+template <typename T>
+static sj_status dev_alloc(sj_target* t, T** p, size_t n) {
+  void* q = nullptr;
+  cudaError_t e = cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(e == cudaErrorMemoryAllocation ? SJ_ERR_OOM : SJ_ERR_CUDA, "cudaMalloc(%zu bytes): %s", n * sizeof(T),
+                cudaGetErrorString(e));
+  }
+  *p = reinterpret_cast<T*>(q);
+  if (t) t->owned.push_back(q);
+  return SJ_OK;
+}
+
+static sj_status setup_site(sj_target* t, TcSite& s, int nseg, const int* seg_rows, int K, bool lm) {
+  s.nseg = nseg;
+  s.K = K;
+  s.KB = K / kBK;
+  s.lm = lm;
+  int tiles = 0;
+  s.N = 0;
+  for (int i = 0; i < 3; ++i) {
+    if (i < nseg) {
+      tiles += (seg_rows[i] + kTileN - 1) / kTileN;
+      s.N += seg_rows[i];
+    }
+    s.seg_tile_end[i] = tiles;
+  }
+  s.n_tiles = tiles;
+  s.G = std::min(t->sm_count, lm ? tiles : (int)std::min<long long>((long long)tiles * s.KB, t->sm_count));
+  if (!lm) {
+    std::vector<int2> slots;
+    build_tile_slots(tiles, s.KB, s.G, slots, s.max_slots);
+    sj_status st = dev_alloc(t, &s.d_tile_slots, slots.size());
+    if (st != SJ_OK) return st;
+    CU_TRY(cudaMemcpy(s.d_tile_slots, slots.data(), slots.size() * sizeof(int2), cudaMemcpyHostToDevice));
+  }
+  return SJ_OK;
+}
+
+static bool tc_shapes_ok(const sj_model_config& c) {
+  auto m128 = [](int x) { return x % 128 == 0; };
+  return c.dtype == SJ_DTYPE_BF16 && m128(c.n_q_heads * c.head_dim) && m128(c.n_kv_heads * c.head_dim) &&
+         m128(c.d_ffn) && m128(c.d_model) && c.d_model % kBK == 0 && c.d_ffn % kBK == 0 &&
+         (c.n_q_heads * c.head_dim) % kBK == 0;
+}
+
+extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weights* w, void* cuda_stream,
+                                      sj_target** out) {
+  if (!cfg || !w || !out) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  *out = nullptr;
+  const sj_model_config& c = *cfg;
+  if (c.n_layers <= 0 || c.d_model <= 0 || c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 ||
+      c.d_ffn <= 0 || c.vocab <= 0)
+    return fail(SJ_ERR_INVALID_ARG, "non-positive dimension");
+  if (c.dtype != SJ_DTYPE_F32 && c.dtype != SJ_DTYPE_BF16) return fail(SJ_ERR_INVALID_ARG, "unknown dtype %d", c.dtype);
+  if (c.head_dim != 64 && c.head_dim != 128) return fail(SJ_ERR_SHAPE, "head_dim must be 64 or 128");
+  if (c.n_q_heads % c.n_kv_heads != 0) return fail(SJ_ERR_SHAPE, "n_q_heads must be a multiple of n_kv_heads");
+  if (c.d_model % 8 || c.d_ffn % 8) return fail(SJ_ERR_SHAPE, "d_model and d_ffn must be multiples of 8");
+  if (c.d_model > 12288) return fail(SJ_ERR_SHAPE, "d_model above 12288 is not supported");
+  if (!(c.rms_eps >= 0.f) || !(c.rope_theta > 0.f)) return fail(SJ_ERR_INVALID_ARG, "bad rms_eps / rope_theta");
+  int max_rows = c.max_rows > 0 ? c.max_rows : 64;
+  if (max_rows > SJ_MAX_ROWS) return fail(SJ_ERR_SHAPE, "max_rows above %d", SJ_MAX_ROWS);
+  if (!w->embed || !w->lm_head || !w->final_norm || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up ||
+      !w->w_down || !w->norm_attn || !w->norm_ffn)
+    return fail(SJ_ERR_INVALID_ARG, "null weight pointer");
+  if (c.qkv_bias && (!w->bq || !w->bk || !w->bv)) return fail(SJ_ERR_INVALID_ARG, "qkv_bias set but biases missing");
+  for (int l = 0; l < c.n_layers; ++l) {
+    if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l] ||
+        !w->norm_attn[l] || !w->norm_ffn[l])
+      return fail(SJ_ERR_INVALID_ARG, "null weight pointer in layer %d", l);
+    if (c.qkv_bias && (!w->bq[l] || !w->bk[l] || !w->bv[l])) return fail(SJ_ERR_INVALID_ARG, "null bias in layer %d", l);
+  }
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  CU_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(SJ_ERR_UNSUPPORTED, "built for sm_100a; device is sm_%d%d", prop.major, prop.minor);
+
+  sj_target* t = new sj_target();
+  t->cfg = c;
+  t->dm = Dims{c.n_layers, c.d_model, c.n_q_heads, c.n_kv_heads, c.head_dim, c.d_ffn, c.vocab, c.rms_eps};
+  t->stream = (cudaStream_t)cuda_stream;
+  t->device = dev;
+  t->sm_count = prop.multiProcessorCount;
+  t->max_rows = max_rows;
+  t->bf = c.dtype == SJ_DTYPE_BF16;
+  t->embed = w->embed;
+  t->lm_head = w->lm_head;
+  t->final_norm = w->final_norm;
+  t->layers.resize(c.n_layers);
+  for (int l = 0; l < c.n_layers; ++l) {
+    LayerW& L = t->layers[l];
+    L.wq = w->wq[l]; L.wk = w->wk[l]; L.wv = w->wv[l]; L.wo = w->wo[l];
+    L.wg = w->w_gate[l]; L.wu = w->w_up[l]; L.wd = w->w_down[l];
+    L.na = w->norm_attn[l]; L.nf = w->norm_ffn[l];
+    L.bq = c.qkv_bias ? w->bq[l] : nullptr; L.bk = c.qkv_bias ? w->bk[l] : nullptr; L.bv = c.qkv_bias ? w->bv[l] : nullptr;
+  }
+  const bool tc = tc_shapes_ok(c);
+  t->opt_gemm = tc ? 1 : 0;
+  t->opt_attn = 0;
+
+  sj_status st = SJ_OK;
+  auto bail = [&](sj_status s) { sj_destroy_target(t); return s; };
+  const size_t esz = t->bf ? 2 : 4;
+  const int qd = c.n_q_heads * c.head_dim, kd = c.n_kv_heads * c.head_dim, R = max_rows;
+  Work& W = t->work;
+  memset(&W, 0, sizeof(W));
+  uint8_t* tmp = nullptr;
+#define ALLOC(field, type, count)                                                     \
+  do {                                                                                \
+    type* p_ = nullptr;                                                               \
+    if ((st = dev_alloc(t, &p_, (count))) != SJ_OK) return bail(st);                  \
+    field = p_;                                                                       \
+  } while (0)
+  ALLOC(W.X, float, (size_t)R * c.d_model);
+  ALLOC(tmp, uint8_t, (size_t)R * c.d_model * esz); W.A = tmp;
+  ALLOC(tmp, uint8_t, (size_t)R * qd * esz); W.Q = tmp;
+  ALLOC(tmp, uint8_t, (size_t)R * qd * esz); W.ATT = tmp;
+  ALLOC(tmp, uint8_t, (size_t)R * c.d_ffn * esz); W.H = tmp;
+  ALLOC(W.Hf, float, (size_t)R * c.d_model);
+  ALLOC(W.rope, float2, (size_t)R * (c.head_dim / 2));
+  ALLOC(W.row_pos, int, R);
+  ALLOC(W.chunk_start, int, SJ_MAX_BATCH + 1);
+  const int n_vtiles = (c.vocab + kTileN - 1) / kTileN;
+  ALLOC(W.stats, RowStat, (size_t)n_vtiles * R);
+  ALLOC(W.tgt_logit, float, R);
+  ALLOC(W.rowstat, RowStat, R);
+  ALLOC(W.status, int, 1);
+  ALLOC(t->d_args, StepArgs, 1);
+  ALLOC(t->d_judge_w, float, c.d_model);
+  ALLOC(t->d_inv_freq, double, c.head_dim / 2);
+  W.judge_w = t->d_judge_w;
+  W.inv_freq = t->d_inv_freq;
+  {
+    cudaError_t e = cudaMemset(W.status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(t->d_judge_w, 0, sizeof(float) * c.d_model);
+    if (e == cudaSuccess) e = cudaMemset(W.tgt_logit, 0, sizeof(float) * R);
+    std::vector<double> inv(c.head_dim / 2);
+    for (int i = 0; i < c.head_dim / 2; ++i) inv[i] = std::pow((double)c.rope_theta, -2.0 * i / c.head_dim);
+    if (e == cudaSuccess) e = cudaMemcpy(t->d_inv_freq, inv.data(), inv.size() * sizeof(double), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "workspace init: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
+  }
+  // GEMM sites and the partial buffer
+  size_t p_elems = (size_t)R * std::max({qd + 2 * kd, c.d_model, 2 * c.d_ffn});
+  if (tc) {
+    int seg_qkv[3] = {qd, kd, kd}, seg_o[1] = {c.d_model}, seg_gu[2] = {c.d_ffn, c.d_ffn}, seg_d[1] = {c.d_model},
+        seg_lm[1] = {c.vocab};
+    if ((st = setup_site(t, t->s_qkv, 3, seg_qkv, c.d_model, false)) != SJ_OK) return bail(st);
+    if ((st = setup_site(t, t->s_o, 1, seg_o, qd, false)) != SJ_OK) return bail(st);
+    if ((st = setup_site(t, t->s_gu, 2, seg_gu, c.d_model, false)) != SJ_OK) return bail(st);
+    if ((st = setup_site(t, t->s_down, 1, seg_d, c.d_ffn, false)) != SJ_OK) return bail(st);
+    if ((st = setup_site(t, t->s_lm, 1, seg_lm, c.d_model, true)) != SJ_OK) return bail(st);
+    p_elems = 0;
+    for (TcSite* s : {&t->s_qkv, &t->s_o, &t->s_gu, &t->s_down})
+      p_elems = std::max(p_elems, (size_t)s->max_slots * R * s->N);
+    for (int l = 0; l < c.n_layers; ++l) {
+      LayerW& L = t->layers[l];
+      if ((st = make_map(&L.m_q, L.wq, qd, c.d_model, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_k, L.wk, kd, c.d_model, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_v, L.wv, kd, c.d_model, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_o, L.wo, c.d_model, qd, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_g, L.wg, c.d_ffn, c.d_model, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_u, L.wu, c.d_ffn, c.d_model, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_d, L.wd, c.d_model, c.d_ffn, kTileN)) != SJ_OK) return bail(st);
+    }
+    if ((st = make_map(&t->m_lm, t->lm_head, c.vocab, c.d_model, kTileN)) != SJ_OK) return bail(st);
+    cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "smem opt-in: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
+  }
+  t->p_elems = p_elems;
+  ALLOC(W.P, float, p_elems);
+#undef ALLOC
+  {
+    cudaError_t e;
+    if (t->bf) e = cudaFuncSetAttribute(k_attn_simt<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    else e = cudaFuncSetAttribute(k_attn_simt<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
+    if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "smem opt-in: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
+  }
+  *out = t;
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_destroy_target(sj_target* t) {
+  if (!t) return SJ_OK;
+  cudaStreamSynchronize(t->stream);
+  clear_graphs(t);
+  for (void* p : t->owned) cudaFree(p);
+  delete t;
+  cudaGetLastError();
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_load_judge_head(sj_target* t, const float* w_host, float bias, float theta) {
+  if (!t || !w_host) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (!(theta == theta) || !(bias == bias)) return fail(SJ_ERR_INVALID_ARG, "NaN judge parameter");
+  CU_TRY(cudaMemcpyAsync(t->d_judge_w, w_host, sizeof(float) * t->dm.d, cudaMemcpyHostToDevice, t->stream));
+  CU_TRY(cudaStreamSynchronize(t->stream));
+  t->judge_bias = bias;
+  t->theta = theta;
+  t->has_judge = true;
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
+  if (!t || !name) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  std::string n(name);
+  if (n == "gemm_impl") {
+    if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "gemm_impl must be 0 or 1");
+    if (value == 1 && !tc_shapes_ok(t->cfg)) return fail(SJ_ERR_UNSUPPORTED, "tensor-core GEMM needs bf16 and 128-multiples");
+    t->opt_gemm = value;
+  } else if (n == "attn_impl") {
+    if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "attn_impl must be 0 or 1");
+    if (value == 1) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention is not available in this build");
+    t->opt_attn = value;
+  } else if (n == "graph") {
+    t->opt_graph = value ? 1 : 0;
+  } else if (n == "pdl") {
+    t->opt_pdl = value ? 1 : 0;
+  } else {
+    return fail(SJ_ERR_INVALID_ARG, "unknown option '%s'", name);
+  }
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_sync(sj_target* t) {
+  if (!t) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  int st = 0;
+  CU_TRY(cudaMemcpyAsync(&st, t->work.status, sizeof(int), cudaMemcpyDeviceToHost, t->stream));
+  CU_TRY(cudaStreamSynchronize(t->stream));
+  if (st != 0) {
+    CU_TRY(cudaMemsetAsync(t->work.status, 0, sizeof(int), t->stream));
+    return fail((sj_status)st, st == DEV_TIMEOUT ? "a bounded device-side wait ran out"
+                                                 : "device rejected a state change (rollback beyond the live length)");
+  }
+  return SJ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV cache
+// ---------------------------------------------------------------------------------------------
+extern "C" sj_status sj_kv_create(sj_target* t, int max_seqs, long max_pages, int page_size, sj_kv** out) {
+  if (!t || !out) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  *out = nullptr;
+  if (page_size != 16) return fail(SJ_ERR_UNSUPPORTED, "page_size must be 16");
+  if (max_seqs <= 0 || max_pages <= 0 || max_pages > 0x7fffffffL) return fail(SJ_ERR_INVALID_ARG, "bad max_seqs/max_pages");
+  sj_kv* kv = new sj_kv();
+  kv->t = t;
+  kv->max_seqs = max_seqs;
+  kv->max_pages = max_pages;
+  const size_t esz = t->bf ? 2 : 4;
+  const size_t page_elems = (size_t)2 * t->dm.Hkv * page_size * t->dm.hd;
+  const size_t bytes = (size_t)t->dm.n_layers * max_pages * page_elems * esz;
+  void* pool = nullptr;
+  cudaError_t e = cudaMalloc(&pool, bytes);
+  int* meta = nullptr;
+  const int mpps = (int)std::min<long>(max_pages, 1 << 20);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&meta, sizeof(int) * ((size_t)max_seqs * (mpps + 2) + 2 * SJ_MAX_BATCH));
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    if (pool) cudaFree(pool);
+    delete kv;
+    return fail(e == cudaErrorMemoryAllocation ? SJ_ERR_OOM : SJ_ERR_CUDA, "KV pool of %zu bytes: %s", bytes,
+                cudaGetErrorString(e));
+  }
+  cudaMemset(meta, 0, sizeof(int) * ((size_t)max_seqs * (mpps + 2) + 2 * SJ_MAX_BATCH));
+  kv->d_block_table = meta;
+  kv->view.pool = pool;
+  kv->view.block_table = meta;
+  kv->view.kv_len = meta + (size_t)max_seqs * mpps;
+  kv->view.pending = kv->view.kv_len + max_seqs;
+  kv->d_tmp = kv->view.pending + max_seqs;
+  kv->view.n_pages = max_pages;
+  kv->view.max_pages_per_seq = mpps;
+  kv->view.page_size = page_size;
+  kv->view.n_kv_heads = t->dm.Hkv;
+  kv->view.head_dim = t->dm.hd;
+  kv->pages.resize(max_seqs);
+  kv->len_hi.assign(max_seqs, 0);
+  kv->exact.assign(max_seqs, 1);
+  kv->free_pages.resize(max_pages);
+  for (long i = 0; i < max_pages; ++i) kv->free_pages[i] = (int)(max_pages - 1 - i);  // pop_back yields 0,1,2..
+  *out = kv;
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_kv_destroy(sj_kv* kv) {
+  if (!kv) return SJ_OK;
+  cudaStreamSynchronize(kv->t->stream);
+  clear_graphs(kv->t);  // captured steps hold this cache's pointers
+  cudaFree(kv->view.pool);
+  cudaFree(kv->d_block_table);
+  delete kv;
+  cudaGetLastError();
+  return SJ_OK;
+}
+
+// Make sure `seq` owns pages for `tokens` tokens; uploads the new block-table entries.
+static sj_status reserve(sj_kv* kv, int seq, long tokens, std::vector<std::pair<int, int>>* undo) {
+  const int ps = kv->view.page_size;
+  const long need = (tokens + ps - 1) / ps;
+  std::vector<int>& pg = kv->pages[seq];
+  if (need > kv->view.max_pages_per_seq) return fail(SJ_ERR_OOM, "sequence %d would exceed the block table", seq);
+  const size_t had = pg.size();
+  if ((long)had >= need) return SJ_OK;
+  if ((long)kv->free_pages.size() < need - (long)had)
+    return fail(SJ_ERR_OOM, "KV page pool exhausted (%zu free, %ld needed)", kv->free_pages.size(), need - (long)had);
+  while ((long)pg.size() < need) {
+    pg.push_back(kv->free_pages.back());
+    kv->free_pages.pop_back();
+  }
+  if (undo) undo->push_back({seq, (int)had});
+  CU_TRY(cudaMemcpyAsync(kv->d_block_table + (size_t)seq * kv->view.max_pages_per_seq + had, pg.data() + had,
+                         sizeof(int) * (pg.size() - had), cudaMemcpyHostToDevice, kv->t->stream));
+  return SJ_OK;
+}
+
+static void release_beyond(sj_kv* kv, int seq, long tokens) {
+  const int ps = kv->view.page_size;
+  const size_t keep = (size_t)((tokens + ps - 1) / ps);
+  std::vector<int>& pg = kv->pages[seq];
+  while (pg.size() > keep) {
+    kv->free_pages.push_back(pg.back());
+    pg.pop_back();
+  }
+}
+
+static sj_status check_seqs(sj_kv* kv, const int* seq_ids, int B) {
+  if (!kv || !seq_ids) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (B <= 0 || B > SJ_MAX_BATCH) return fail(SJ_ERR_INVALID_ARG, "B out of range");
+  for (int i = 0; i < B; ++i)
+    if (seq_ids[i] < 0 || seq_ids[i] >= kv->max_seqs) return fail(SJ_ERR_INVALID_ARG, "sequence id %d out of range", seq_ids[i]);
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_kv_fill(sj_kv* kv, int seq, int layer, int start, int n_tokens, const void* k, const void* v) {
+  if (!kv || !k || !v) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (seq < 0 || seq >= kv->max_seqs || layer < 0 || layer >= kv->t->dm.n_layers || start < 0 || n_tokens <= 0)
+    return fail(SJ_ERR_INVALID_ARG, "sj_kv_fill: index out of range");
+  sj_status st = reserve(kv, seq, (long)start + n_tokens, nullptr);
+  if (st != SJ_OK) return st;
+  cudaError_t e;
+  if (kv->t->bf)
+    e = launch(k_kv_copy<bf16>, dim3(n_tokens), dim3(256), 0, kv->t->stream, false, kv->view, seq, layer, start, n_tokens,
+               (bf16*)k, (bf16*)v, 1);
+  else
+    e = launch(k_kv_copy<float>, dim3(n_tokens), dim3(256), 0, kv->t->stream, false, kv->view, seq, layer, start, n_tokens,
+               (float*)k, (float*)v, 1);
+  CU_TRY(e);
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_kv_read(sj_kv* kv, int seq, int layer, int start, int n_tokens, void* k_out, void* v_out) {
+  if (!kv || !k_out || !v_out) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (seq < 0 || seq >= kv->max_seqs || layer < 0 || layer >= kv->t->dm.n_layers || start < 0 || n_tokens <= 0)
+    return fail(SJ_ERR_INVALID_ARG, "sj_kv_read: index out of range");
+  if ((size_t)(start + n_tokens) > kv->pages[seq].size() * kv->view.page_size)
+    return fail(SJ_ERR_INVALID_ARG, "sj_kv_read: rows beyond the reserved pages");
+  cudaError_t e;
+  if (kv->t->bf)
+    e = launch(k_kv_copy<bf16>, dim3(n_tokens), dim3(256), 0, kv->t->stream, false, kv->view, seq, layer, start, n_tokens,
+               (bf16*)k_out, (bf16*)v_out, 0);
+  else
+    e = launch(k_kv_copy<float>, dim3(n_tokens), dim3(256), 0, kv->t->stream, false, kv->view, seq, layer, start, n_tokens,
+               (float*)k_out, (float*)v_out, 0);
+  CU_TRY(e);
+  CU_TRY(cudaStreamSynchronize(kv->t->stream));
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_kv_set_len(sj_kv* kv, const int* seq_ids, const int* lens, int B) {
+  sj_status st = check_seqs(kv, seq_ids, B);
+  if (st != SJ_OK) return st;
+  if (!lens) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  for (int i = 0; i < B; ++i)
+    if (lens[i] < 0 || (size_t)lens[i] > kv->pages[seq_ids[i]].size() * kv->view.page_size)
+      return fail(SJ_ERR_STATE, "length %d of sequence %d exceeds its reserved rows", lens[i], seq_ids[i]);
+  for (int i = 0; i < B; ++i) {
+    CU_TRY(cudaMemcpyAsync(kv->view.kv_len + seq_ids[i], lens + i, sizeof(int), cudaMemcpyHostToDevice, kv->t->stream));
+    kv->len_hi[seq_ids[i]] = lens[i];
+    kv->exact[seq_ids[i]] = 1;
+  }
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_kv_set_pending(sj_kv* kv, const int* seq_ids, const int* tokens, int B) {
+  sj_status st = check_seqs(kv, seq_ids, B);
+  if (st != SJ_OK) return st;
+  if (!tokens) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  for (int i = 0; i < B; ++i) {
+    if (tokens[i] < 0 || tokens[i] >= kv->t->dm.V) return fail(SJ_ERR_INVALID_ARG, "token id out of range");
+  }
+  for (int i = 0; i < B; ++i)
+    CU_TRY(cudaMemcpyAsync(kv->view.pending + seq_ids[i], tokens + i, sizeof(int), cudaMemcpyHostToDevice, kv->t->stream));
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_kv_len(sj_kv* kv, const int* seq_ids, int* out_len, int B) {
+  sj_status st = check_seqs(kv, seq_ids, B);
+  if (st != SJ_OK) return st;
+  if (!out_len) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  for (int i = 0; i < B; ++i)
+    CU_TRY(cudaMemcpyAsync(out_len + i, kv->view.kv_len + seq_ids[i], sizeof(int), cudaMemcpyDeviceToHost, kv->t->stream));
+  CU_TRY(cudaStreamSynchronize(kv->t->stream));
+  for (int i = 0; i < B; ++i) {
+    kv->len_hi[seq_ids[i]] = out_len[i];
+    kv->exact[seq_ids[i]] = 1;
+    release_beyond(kv, seq_ids[i], out_len[i]);
+  }
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_rollback_kv(sj_kv* kv, const int* seq_ids, const int* new_len, int B) {
+  sj_status st = check_seqs(kv, seq_ids, B);
+  if (st != SJ_OK) return st;
+  if (!new_len) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  for (int i = 0; i < B; ++i) {
+    if (new_len[i] < 0) return fail(SJ_ERR_INVALID_ARG, "negative length");
+    if (new_len[i] > kv->len_hi[seq_ids[i]])
+      return fail(SJ_ERR_STATE, "rollback of sequence %d to %d beyond its length (at most %d)", seq_ids[i], new_len[i],
+                  kv->len_hi[seq_ids[i]]);
+  }
+  int stage[2 * SJ_MAX_BATCH];
+  memcpy(stage, seq_ids, sizeof(int) * B);
+  memcpy(stage + B, new_len, sizeof(int) * B);
+  CU_TRY(cudaMemcpyAsync(kv->d_tmp, stage, sizeof(int) * 2 * B, cudaMemcpyHostToDevice, kv->t->stream));
+  CU_TRY(launch(k_rollback, dim3((B + 127) / 128), dim3(128), 0, kv->t->stream, false, kv->view, (const int*)kv->d_tmp,
+                (const int*)(kv->d_tmp + B), B, kv->t->work.status));
+  for (int i = 0; i < B; ++i) kv->len_hi[seq_ids[i]] = new_len[i];  // still an upper bound if the device refuses
+  return SJ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// the step
+// ---------------------------------------------------------------------------------------------
+static sj_status activation_map(sj_target* t, std::map<int, CUtensorMap>& cache, const void* base, int R, int K,
+                                const CUtensorMap** out) {
+  auto it = cache.find(R);
+  if (it == cache.end()) {
+    CUtensorMap m;
+    RowGeom g = row_geom(R);
+    sj_status st = make_map(&m, base, R, K, g.nblk);
+    if (st != SJ_OK) return st;
+    it = cache.emplace(R, m).first;
+  }
+  *out = &it->second;
+  return SJ_OK;
+}
+
+static cudaError_t launch_tc(sj_target* t, const TcSite& s, const CUtensorMap* mA, const CUtensorMap* w0,
+                             const CUtensorMap* w1, const CUtensorMap* w2, int R, bool pdl) {
+  RowGeom g = row_geom(R);
+  TcGemmParams p;
+  memset(&p, 0, sizeof(p));
+  p.n_tiles = s.n_tiles; p.KB = s.KB; p.G = s.G; p.U = (long long)s.n_tiles * s.KB; p.R = R;
+  p.NB = g.NB; p.nblk = g.nblk; p.N_total = s.N;
+  for (int i = 0; i < 3; ++i) p.seg_tile_end[i] = s.seg_tile_end[i];
+  p.stages = g.stages; p.a_stage_bytes = g.a_stage_bytes; p.tmem_cols = g.tmem_cols;
+  p.acc_bufs = g.acc_bufs; p.acc_stride = g.acc_stride;
+  p.P = t->work.P; p.slot_stride = (size_t)R * s.N; p.tile_slots = s.d_tile_slots;
+  p.lm_mode = s.lm ? 1 : 0; p.status = t->work.status;
+  return launch(k_gemm_tc, dim3(s.G), dim3(kTcThreads), g.smem_bytes, t->stream, pdl, *mA, *w0, *(w1 ? w1 : w0),
+                *(w2 ? w2 : w0), p, (const StepArgs*)t->d_args, t->work, t->dm.V);
+}
+
+template <typename T>
+static cudaError_t launch_simt(sj_target* t, const void* A, const GemmSegs& segs, float* Y, int R, int N, int K, bool pdl) {
+  return launch(k_gemm_simt<T, 8>, dim3((N + 7) / 8), dim3(256), 0, t->stream, pdl, (const T*)A, segs, Y, R, N, K);
+}
+
+template <typename T>
+static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mode, int chunk_len, bool use_scratch,
+                               size_t n_chunks_hi) {
+  const Dims& dm = t->dm;
+  const int R = B * (gamma + 1), qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd;
+  const bool pdl = t->opt_pdl != 0, tc = t->opt_gemm == 1;
+  const StepArgs* args = t->d_args;
+  Work W = t->work;
+  if (!use_scratch) W.logits = nullptr;
+  cudaStream_t s = t->stream;
+  const size_t row_smem = sizeof(float) * dm.d;
+  SplitPlan one{nullptr, 0};
+  const CUtensorMap *mA_d = nullptr, *mA_q = nullptr, *mA_f = nullptr;
+  if (tc) {
+    sj_status st;
+    if ((st = activation_map(t, t->mapA_d, W.A, R, dm.d, &mA_d)) != SJ_OK) return st;
+    if ((st = activation_map(t, t->mapA_q, W.ATT, R, qd, &mA_q)) != SJ_OK) return st;
+    if ((st = activation_map(t, t->mapA_f, W.H, R, dm.F, &mA_f)) != SJ_OK) return st;
+  }
+  auto plan_of = [&](const TcSite& site) { return tc ? SplitPlan{site.d_tile_slots, site.n_tiles} : one; };
+
+  CU_TRY(launch(k_plan, dim3(1), dim3(256), 0, s, false, args, kv->view, W, chunk_len));
+  CU_TRY(launch(k_embed_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, kv->view, W, dm, (const T*)t->embed,
+                (const T*)t->layers[0].na));
+  const int nq = (dm.Hq / dm.Hkv) * (gamma + 1);
+  const size_t att_smem = sizeof(float) * ((size_t)nq * dm.hd + kAttKT * (dm.hd + 1) + kAttKT * dm.hd + (size_t)nq * kAttKT + 3 * nq);
+  const int att_grid = std::max(1, std::min<int>(t->sm_count * 2, (int)n_chunks_hi * dm.Hkv));
+  for (int l = 0; l < dm.n_layers; ++l) {
+    const LayerW& L = t->layers[l];
+    // QKV projection
+    if (tc) {
+      CU_TRY(launch_tc(t, t->s_qkv, mA_d, &L.m_q, &L.m_k, &L.m_v, R, pdl));
+    } else {
+      GemmSegs g{{L.wq, L.wk, L.wv}, {qd, kd, kd}, 3};
+      CU_TRY(launch_simt<T>(t, W.A, g, W.P, R, qd + 2 * kd, dm.d, pdl));
+    }
+    CU_TRY(launch(k_qkv_rope<T>, dim3(R), dim3(256), 0, s, pdl, args, kv->view, W, dm, plan_of(t->s_qkv),
+                  (size_t)R * (qd + 2 * kd), l, (const T*)L.bq, (const T*)L.bk, (const T*)L.bv));
+    // attention
+    CU_TRY(launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
+    CU_TRY(launch(k_attn_combine<T>, dim3(R * dm.Hq), dim3(std::min(dm.hd, 128)), 0, s, pdl, args, W, dm));
+    // O projection + residual + FFN norm
+    if (tc) {
+      CU_TRY(launch_tc(t, t->s_o, mA_q, &L.m_o, nullptr, nullptr, R, pdl));
+    } else {
+      GemmSegs g{{L.wo, nullptr, nullptr}, {dm.d, 0, 0}, 1};
+      CU_TRY(launch_simt<T>(t, W.ATT, g, W.P, R, dm.d, qd, pdl));
+    }
+    CU_TRY(launch(k_reduce_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, W, dm, plan_of(t->s_o), (size_t)R * dm.d,
+                  (const T*)L.nf, 0));
+    // gate/up + SwiGLU
+    if (tc) {
+      CU_TRY(launch_tc(t, t->s_gu, mA_d, &L.m_g, &L.m_u, nullptr, R, pdl));
+    } else {
+      GemmSegs g{{L.wg, L.wu, nullptr}, {dm.F, dm.F, 0}, 2};
+      CU_TRY(launch_simt<T>(t, W.A, g, W.P, R, 2 * dm.F, dm.d, pdl));
+    }
+    CU_TRY(launch(k_swiglu<T>, dim3((dm.F + 255) / 256, R), dim3(256), 0, s, pdl, W, dm, plan_of(t->s_gu),
+                  (size_t)R * 2 * dm.F));
+    // down projection + residual + next norm
+    if (tc) {
+      CU_TRY(launch_tc(t, t->s_down, mA_f, &L.m_d, nullptr, nullptr, R, pdl));
+    } else {
+      GemmSegs g{{L.wd, nullptr, nullptr}, {dm.d, 0, 0}, 1};
+      CU_TRY(launch_simt<T>(t, W.H, g, W.P, R, dm.d, dm.F, pdl));
+    }
+    const bool last = (l == dm.n_layers - 1);
+    const void* gain = last ? t->final_norm : t->layers[l + 1].na;
+    CU_TRY(launch(k_reduce_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, W, dm, plan_of(t->s_down),
+                  (size_t)R * dm.d, (const T*)gain, last ? 1 : 0));
+  }
+  // LM head + statistics
+  const int n_vtiles = (dm.V + kTileN - 1) / kTileN;
+  if (tc) {
+    CU_TRY(launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl));
+  } else {
+    GemmSegs g{{t->lm_head, nullptr, nullptr}, {dm.V, 0, 0}, 1};
+    CU_TRY(launch_simt<T>(t, W.A, g, W.logits, R, dm.V, dm.d, pdl));
+    CU_TRY(launch(k_lm_stats_from_logits, dim3(n_vtiles, (R + 7) / 8), dim3(256), 0, s, pdl, args, W, dm, R));
+  }
+  CU_TRY(launch(k_finalize, dim3(B), dim3(256), 0, s, pdl, args, kv->view, W, dm, n_vtiles, R));
+  if (mode == SJ_MODE_SAMPLING) CU_TRY(launch(k_resample, dim3(B), dim3(1024), 0, s, pdl, args, kv->view, W, dm));
+  return SJ_OK;
+}
+
+static int pick_chunk_len(const sj_target* t, long total_keys) {
+  long want = total_keys * t->dm.Hkv / (2L * t->sm_count);
+  int ch = 64;
+  while (ch < want && ch < 4096) ch <<= 1;
+  return ch;
+}
+
+extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a, const sj_verify_out* o) {
+  if (!t || !kv || !a || !o) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (kv->t != t) return fail(SJ_ERR_INVALID_ARG, "KV cache belongs to another target");
+  if (a->B <= 0 || a->B > SJ_MAX_BATCH) return fail(SJ_ERR_INVALID_ARG, "B out of range");
+  if (a->gamma < 1 || a->gamma > SJ_MAX_GAMMA) return fail(SJ_ERR_INVALID_ARG, "gamma out of range [1,%d]", SJ_MAX_GAMMA);
+  const int B = a->B, gamma = a->gamma, rows = gamma + 1, R = B * rows;
+  if (R > t->max_rows) return fail(SJ_ERR_SHAPE, "B*(gamma+1) = %d exceeds max_rows = %d", R, t->max_rows);
+  sj_status st = check_seqs(kv, a->seq_ids, B);
+  if (st != SJ_OK) return st;
+  {
+    std::vector<char> seen(kv->max_seqs, 0);
+    for (int i = 0; i < B; ++i) {
+      if (seen[a->seq_ids[i]]) return fail(SJ_ERR_INVALID_ARG, "duplicate sequence id %d", a->seq_ids[i]);
+      seen[a->seq_ids[i]] = 1;
+    }
+  }
+  if (a->mode != SJ_MODE_GREEDY && a->mode != SJ_MODE_SAMPLING) return fail(SJ_ERR_INVALID_ARG, "unknown mode");
+  if (!a->draft_ids) return fail(SJ_ERR_INVALID_ARG, "draft_ids is null");
+  if (a->mode == SJ_MODE_SAMPLING) {
+    if (!a->draft_q_tok || !a->draft_q_full || !a->uniforms) return fail(SJ_ERR_INVALID_ARG, "sampling mode needs q and uniforms");
+    if (!(a->temperature > 0.f)) return fail(SJ_ERR_INVALID_ARG, "temperature must be > 0");
+  }
+  if (!o->accepted_len || !o->next_token || !o->judge_scores || !o->p_draft || !o->new_kv_len)
+    return fail(SJ_ERR_INVALID_ARG, "null output pointer");
+  if (a->theta_override == a->theta_override && a->theta_override > 1e30f) return fail(SJ_ERR_INVALID_ARG, "bad theta");
+  if (a->theta_override != a->theta_override) return fail(SJ_ERR_INVALID_ARG, "theta is NaN");
+  const int group = t->dm.Hq / t->dm.Hkv;
+  if (group * rows > kAttMaxQ) return fail(SJ_ERR_SHAPE, "(Hq/Hkv)*(gamma+1) = %d exceeds %d", group * rows, kAttMaxQ);
+
+  // a0: reserve pages for gamma+1 more rows per sequence; nothing is launched if the pool runs out
+  std::vector<std::pair<int, int>> undo;
+  long total_keys = 0;
+  size_t chunk_need_base = 0;
+  for (int i = 0; i < B; ++i) {
+    int s = a->seq_ids[i];
+    st = reserve(kv, s, (long)kv->len_hi[s] + rows, &undo);
+    if (st != SJ_OK) {
+      for (auto& u : undo) {
+        std::vector<int>& pg = kv->pages[u.first];
+        while ((int)pg.size() > u.second) { kv->free_pages.push_back(pg.back()); pg.pop_back(); }
+      }
+      return st;
+    }
+    total_keys += kv->len_hi[s] + rows;
+  }
+  const int chunk_len = pick_chunk_len(t, total_keys);
+  for (int i = 0; i < B; ++i) chunk_need_base += (size_t)(kv->len_hi[a->seq_ids[i]] + rows + chunk_len - 1) / chunk_len;
+
+  const bool use_scratch = a->mode == SJ_MODE_SAMPLING || t->opt_gemm == 0;
+  // grow lazily-sized buffers (outside any capture)
+  if (chunk_need_base > t->att_chunks_cap || rows > t->att_rows_cap) {
+    CU_TRY(cudaStreamSynchronize(t->stream));
+    clear_graphs(t);
+    size_t cap = std::max(chunk_need_base * 2, (size_t)64);
+    int rcap = std::max(rows, t->att_rows_cap);
+    for (float** p : {&t->work.att_m, &t->work.att_l, &t->work.att_o}) {
+      if (*p) {
+        cudaFree(*p);
+        t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)*p), t->owned.end());
+        *p = nullptr;
+      }
+    }
+    size_t n_ml = cap * t->dm.Hq * rcap;
+    if ((st = dev_alloc(t, &t->work.att_m, n_ml)) != SJ_OK) return st;
+    if ((st = dev_alloc(t, &t->work.att_l, n_ml)) != SJ_OK) return st;
+    if ((st = dev_alloc(t, &t->work.att_o, n_ml * t->dm.hd)) != SJ_OK) return st;
+    t->att_chunks_cap = cap;
+    t->att_rows_cap = rcap;
+  }
+  if (use_scratch && (size_t)R > t->logits_rows) {
+    CU_TRY(cudaStreamSynchronize(t->stream));
+    clear_graphs(t);
+    if (t->work.logits) {
+      cudaFree(t->work.logits);
+      t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)t->work.logits), t->owned.end());
+      t->work.logits = nullptr;
+    }
+    if ((st = dev_alloc(t, &t->work.logits, (size_t)R * t->dm.V)) != SJ_OK) return st;
+    t->logits_rows = R;
+  }
+
+  // per-call arguments: one small copy (the driver stages pageable memory before returning)
+  StepArgs h;
+  memset(&h, 0, sizeof(h));
+  h.draft_ids = a->draft_ids; h.q_tok = a->draft_q_tok; h.q_full = a->draft_q_full; h.uniforms = a->uniforms;
+  h.accepted_len = o->accepted_len; h.next_token = o->next_token; h.judge_scores = o->judge_scores;
+  h.p_draft = o->p_draft; h.new_kv_len = o->new_kv_len; h.dbg_hidden = o->dbg_hidden; h.dbg_logits = o->dbg_logits;
+  h.B = B; h.gamma = gamma; h.mode = a->mode; h.use_align = a->use_align ? 1 : 0; h.use_judge = a->use_judge ? 1 : 0;
+  h.commit = a->commit ? 1 : 0;
+  h.inv_temperature = a->mode == SJ_MODE_SAMPLING ? 1.0f / a->temperature : 1.0f;
+  h.theta = a->theta_override >= 0.f ? a->theta_override : t->theta;
+  h.judge_bias = t->judge_bias;
+  h.has_judge = t->has_judge ? 1 : 0;
+  memcpy(h.seq_ids, a->seq_ids, sizeof(int) * B);
+  CU_TRY(cudaMemcpyAsync(t->d_args, &h, sizeof(h), cudaMemcpyHostToDevice, t->stream));
+
+  StepKey key{B, gamma, a->mode, chunk_len, t->opt_gemm, t->opt_attn, t->opt_pdl, use_scratch ? 1 : 0};
+  if (t->opt_graph) {
+    auto it = t->graphs.find(key);
+    if (it == t->graphs.end()) {
+      if (t->opt_gemm == 1) {  // encode activation maps before capturing
+        const CUtensorMap* dummy;
+        if ((st = activation_map(t, t->mapA_d, t->work.A, R, t->dm.d, &dummy)) != SJ_OK) return st;
+      }
+      cudaGraph_t graph = nullptr;
+      CU_TRY(cudaStreamBeginCapture(t->stream, cudaStreamCaptureModeThreadLocal));
+      st = t->bf ? enqueue_step<bf16>(t, kv, B, gamma, a->mode, chunk_len, use_scratch, chunk_need_base)
+                 : enqueue_step<float>(t, kv, B, gamma, a->mode, chunk_len, use_scratch, chunk_need_base);
+      cudaError_t e = cudaStreamEndCapture(t->stream, &graph);
+      if (st != SJ_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        return st;
+      }
+      CU_TRY(e);
+      cudaGraphExec_t exec = nullptr;
+      e = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      CU_TRY(e);
+      it = t->graphs.emplace(key, exec).first;
+    }
+    CU_TRY(cudaGraphLaunch(it->second, t->stream));
+  } else {
+    st = t->bf ? enqueue_step<bf16>(t, kv, B, gamma, a->mode, chunk_len, use_scratch, chunk_need_base)
+               : enqueue_step<float>(t, kv, B, gamma, a->mode, chunk_len, use_scratch, chunk_need_base);
+    if (st != SJ_OK) return st;
+  }
+  if (a->commit) {
+    for (int i = 0; i < B; ++i) {
+      int s = a->seq_ids[i];
+      kv->len_hi[s] += rows;
+      kv->exact[s] = 0;
+    }
+  }
+  return SJ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// standalone skinny GEMM
+// ---------------------------------------------------------------------------------------------
+__global__ void k_sum_slots(const float* __restrict__ P, SplitPlan sp, size_t slot_stride, int R, int N, float* __restrict__ Y) {
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (size_t)R * N) return;
+  Y[i] = reduce_partials(P, sp, slot_stride, N, (int)(i / N), (int)(i % N));
+}
+
+extern "C" sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, const void* a, const void* w, float* y,
+                                    void* cuda_stream) {
+  if (!a || !w || !y) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (R <= 0 || R > SJ_MAX_ROWS || N <= 0 || K <= 0 || K % 8) return fail(SJ_ERR_SHAPE, "bad GEMM shape");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (impl == 0) {
+    GemmSegs g{{w, nullptr, nullptr}, {N, 0, 0}, 1};
+    if (dtype == SJ_DTYPE_BF16)
+      CU_TRY(launch(k_gemm_simt<bf16, 8>, dim3((N + 7) / 8), dim3(256), 0, s, false, (const bf16*)a, g, y, R, N, K));
+    else if (dtype == SJ_DTYPE_F32)
+      CU_TRY(launch(k_gemm_simt<float, 8>, dim3((N + 7) / 8), dim3(256), 0, s, false, (const float*)a, g, y, R, N, K));
+    else
+      return fail(SJ_ERR_INVALID_ARG, "unknown dtype");
+    return SJ_OK;
+  }
+  if (impl != 1) return fail(SJ_ERR_INVALID_ARG, "unknown impl");
+  if (dtype != SJ_DTYPE_BF16 || K % kBK) return fail(SJ_ERR_UNSUPPORTED, "tensor-core GEMM needs bf16 and K %% 64 == 0");
+  cudaDeviceProp prop;
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  CU_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(SJ_ERR_UNSUPPORTED, "built for sm_100a");
+  sj_target tmp;  // borrowed only for its plumbing fields
+  tmp.stream = s;
+  tmp.sm_count = prop.multiProcessorCount;
+  tmp.dm.V = N;
+  memset(&tmp.work, 0, sizeof(tmp.work));
+  TcSite site;
+  int seg[1] = {N};
+  sj_status st = setup_site(&tmp, site, 1, seg, K, false);
+  auto cleanup = [&]() { for (void* p : tmp.owned) cudaFree(p); };
+  if (st != SJ_OK) { cleanup(); return st; }
+  float* P = nullptr;
+  int* status = nullptr;
+  if ((st = dev_alloc(&tmp, &P, (size_t)site.max_slots * R * N)) != SJ_OK) { cleanup(); return st; }
+  if ((st = dev_alloc(&tmp, &status, 1)) != SJ_OK) { cleanup(); return st; }
+  cudaMemsetAsync(status, 0, sizeof(int), s);
+  tmp.work.P = P;
+  tmp.work.status = status;
+  CUtensorMap mA, mW;
+  RowGeom g = row_geom(R);
+  if ((st = make_map(&mA, a, R, K, g.nblk)) != SJ_OK) { cleanup(); return st; }
+  if ((st = make_map(&mW, w, N, K, kTileN)) != SJ_OK) { cleanup(); return st; }
+  cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess) e = launch_tc(&tmp, site, &mA, &mW, nullptr, nullptr, R, false);
+  if (e == cudaSuccess)
+    e = launch(k_sum_slots, dim3((unsigned)(((size_t)R * N + 255) / 256)), dim3(256), 0, s, false, (const float*)P,
+               SplitPlan{site.d_tile_slots, site.n_tiles}, (size_t)R * N, R, N, y);
+  int hstatus = 0;
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&hstatus, status, sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  cleanup();
+  if (e != cudaSuccess) { cudaGetLastError(); return fail(SJ_ERR_CUDA, "sj_gemm_skinny: %s", cudaGetErrorString(e)); }
+  if (hstatus != 0) return fail(SJ_ERR_TIMEOUT, "a bounded device-side wait ran out");
+  return SJ_OK;
+}

@@ -1,0 +1,211 @@
+"""GPU parity: the CUDA library through its C ABI against the CPU oracle on the same seeded bytes."""
+import numpy as np
+import pytest
+import torch
+
+import harness
+import helpers
+from oracle import sj_oracle as orc
+from paper_2510_02329_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GQA = synth.ModelShape("gqa-small", 3, 256, 4, 2, 64, 512, 1024, rope_theta=5e5)
+GQA128 = synth.ModelShape("gqa-hd128", 2, 512, 8, 2, 128, 1024, 2048, rope_theta=5e5, qkv_bias=True)
+
+
+def _binding():
+    from paper_2510_02329_b200 import binding
+    return binding
+
+
+# ------------------------------------------------------------------------------------------------
+# kernel level: the skinny GEMM
+# ------------------------------------------------------------------------------------------------
+GEMM_SHAPES = [(5, 384, 256), (9, 1000, 512), (17, 4096, 4096), (72, 2048, 1024), (1, 128, 64), (16, 256, 8192)]
+
+
+@pytest.mark.parametrize("R,N,K", GEMM_SHAPES)
+@pytest.mark.parametrize("dtype,impl", [(torch.float32, 0), (torch.bfloat16, 0), (torch.bfloat16, 1)],
+                         ids=["f32-cudacore", "bf16-cudacore", "bf16-tcgen05"])
+def test_gemm_skinny_matches_fp64_matmul(R, N, K, dtype, impl):
+    b = _binding()
+    a = synth.normal(synth.tensor_key(1, 50, R), (R, K), 1.0, dtype)
+    w = synth.normal(synth.tensor_key(1, 51, N), (N, K), 0.02, dtype)
+    y = b.gemm_skinny(a.cuda(), w.cuda(), impl).cpu().numpy()
+    a64, w64 = helpers.np64(a), helpers.np64(w)
+    ref = a64 @ w64.T
+    bound = 1e-5 * (np.abs(a64) @ np.abs(w64).T) + 1e-7
+    err = np.abs(y - ref)
+    assert (err <= bound).all(), f"max err {err.max():.3e} at {np.unravel_index(err.argmax(), err.shape)}"
+
+
+@pytest.mark.parametrize("R", [288, 512])
+def test_gemm_skinny_tcgen05_many_rows(R):
+    b = _binding()
+    N, K = 640, 1024
+    a = synth.normal(synth.tensor_key(2, 50, R), (R, K), 1.0, torch.bfloat16)
+    w = synth.normal(synth.tensor_key(2, 51, N), (N, K), 0.02, torch.bfloat16)
+    y = b.gemm_skinny(a.cuda(), w.cuda(), 1).cpu().numpy()
+    a64, w64 = helpers.np64(a), helpers.np64(w)
+    assert (np.abs(y - a64 @ w64.T) <= 1e-5 * (np.abs(a64) @ np.abs(w64).T) + 1e-7).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# whole step
+# ------------------------------------------------------------------------------------------------
+def _run(case, mode, temperature=1.0, theta=0.5, use_align=True, use_judge=True, options=None):
+    for k, v in (options or {}).items():
+        case.target.set_option(k, v)
+    v, f = case.run_oracle(mode, temperature, theta, use_align, use_judge)
+    g = case.run_gpu(mode, temperature, theta, use_align, use_judge)
+    return harness.compare(case, v, f, g, mode, temperature, theta), g
+
+
+CFG1_VARIANTS = [
+    ("f32", torch.float32, {}),
+    ("f32-nograph-nopdl", torch.float32, {"graph": 0, "pdl": 0}),
+    ("bf16-cudacore", torch.bfloat16, {"gemm_impl": 0}),
+    ("bf16-tcgen05", torch.bfloat16, {"gemm_impl": 1}),
+    ("bf16-tcgen05-nograph", torch.bfloat16, {"gemm_impl": 1, "graph": 0, "pdl": 0}),
+]
+
+
+@pytest.mark.parametrize("name,dtype,options", CFG1_VARIANTS, ids=[v[0] for v in CFG1_VARIANTS])
+def test_config1_tiny_target(name, dtype, options):
+    """2 layers, d 256, 4 MHA heads of 64, FFN 1024, vocab 4096; batch 1, 128 cached tokens, gamma 4."""
+    case = harness.Case(synth.TINY, dtype, [128], 4, seed=0).gpu_setup()
+    try:
+        exact = 0
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 1.0), (orc.SAMPLING, 0.1)]:
+            rep, _ = _run(case, mode, T, options=options)
+            exact += rep.exact
+            print(name, "mode", mode, "T", T, rep)
+        if dtype == torch.float32:
+            assert exact >= 2  # fp32 decisions are crisp except true near-ties
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("dtype,options", [(torch.float32, {}), (torch.bfloat16, {"gemm_impl": 0}),
+                                            (torch.bfloat16, {"gemm_impl": 1})], ids=["f32", "bf16-cudacore", "bf16-tcgen05"])
+@pytest.mark.parametrize("kv_lens,gamma", [([5, 37, 130], 3), ([15, 16, 17, 0], 5), ([200], 1), ([63, 64], 16)])
+def test_ragged_batches_and_page_edges(dtype, options, kv_lens, gamma):
+    case = harness.Case(GQA, dtype, kv_lens, gamma, seed=3).gpu_setup()
+    try:
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 0.2)]:
+            rep, _ = _run(case, mode, T, options=options)
+            assert rep.exact + rep.margin == len(kv_lens)
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("options", [{"gemm_impl": 0}, {"gemm_impl": 1}], ids=["cudacore", "tcgen05"])
+def test_head_dim_128_with_qkv_bias(options):
+    case = harness.Case(GQA128, torch.bfloat16, [70, 300], 8, seed=4).gpu_setup()
+    try:
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 0.2)]:
+            _run(case, mode, T, options=options)
+    finally:
+        case.close()
+
+
+def test_drafts_following_the_target_are_accepted_and_judge_flags():
+    """Drafts that equal the oracle's greedy chain are accepted; ablation flags and theta limits."""
+    shape, L, gamma = GQA, 40, 6
+    probe = harness.Case(shape, torch.float32, [L], gamma, seed=7)
+    # greedy chain from the oracle: feed pending, take argmax, append, repeat
+    osh, top = probe.osh, probe.top64
+    caches = [[(helpers.np64(k), helpers.np64(v)) for k, v in probe.cache_t[0]]]
+    chain, toks = [], [int(probe.inputs.pending[0])]
+    for _ in range(gamma - 2):
+        fwd = orc.forward_blocks(osh, top, probe.model.layer64, [np.array(toks)], caches)[0]
+        chain.append(int(np.argmax(fwd.logits[-1])))
+        toks.append(chain[-1])
+    drafts = probe.inputs.draft_ids.copy()
+    drafts[0, :gamma - 2] = chain
+    case = harness.Case(shape, torch.float32, [L], gamma, seed=7, draft_ids=drafts).gpu_setup()
+    try:
+        rep, g = _run(case, orc.GREEDY, use_judge=False)
+        assert rep.exact == 1 and g["accepted_len"][0] >= gamma - 2
+        n_off = int(g["accepted_len"][0])
+        rep, g = _run(case, orc.GREEDY, theta=0.0)
+        assert g["accepted_len"][0] == gamma                         # sigmoid > 0 always
+        rep, g = _run(case, orc.GREEDY, theta=1.0)
+        assert g["accepted_len"][0] == n_off                         # judge can never fire
+        prev = gamma
+        for th in (0.3, 0.5, 0.7):
+            rep, g = _run(case, orc.GREEDY, theta=th)
+            assert rep.exact == 1 and g["accepted_len"][0] <= prev
+            prev = int(g["accepted_len"][0])
+        rep, g = _run(case, orc.GREEDY, use_align=False)              # judge only
+        assert rep.exact == 1
+    finally:
+        case.close()
+
+
+def test_commit_second_step_and_rollback():
+    b = _binding()
+    shape, L, gamma = GQA, 21, 4
+    case = harness.Case(shape, torch.float32, [L], gamma, seed=11).gpu_setup()
+    try:
+        v1, f1 = case.run_oracle(orc.GREEDY, use_judge=True, theta=0.5)
+        g1 = case.run_gpu(orc.GREEDY, theta=0.5, commit=True)
+        rep = harness.compare(case, v1, f1, g1, orc.GREEDY)
+        assert rep.exact == 1
+        n = v1[0].accepted_len
+        assert case.kv.lengths([0]) == [L + 1 + n]
+        # committed cache rows equal the oracle's new rows (first 1+n)
+        for l in range(shape.n_layers):
+            k, v = case.kv.read(0, l, L, 1 + n)
+            assert np.abs(k.cpu().double().numpy() - f1[0].k_new[l][:1 + n]).max() < 1e-4
+            assert np.abs(v.cpu().double().numpy() - f1[0].v_new[l][:1 + n]).max() < 1e-4
+        # second step: pending is the first step's next token (set on the device by the commit)
+        si2 = synth.step_inputs(shape.vocab, 1, gamma, seed=12)
+        caches2 = [[(np.concatenate([helpers.np64(case.cache_t[0][l][0]), f1[0].k_new[l][:1 + n]]),
+                     np.concatenate([helpers.np64(case.cache_t[0][l][1]), f1[0].v_new[l][:1 + n]]))
+                    for l in range(shape.n_layers)]]
+        v2, f2 = orc.verify(case.osh, case.top64, case.model.layer64, [v1[0].next_token], si2.draft_ids, caches2,
+                            mode=orc.GREEDY, judge_w=case.judge_w64, theta=0.5)
+        out = b.VerifyBuffers(1, gamma, shape.d_model, shape.vocab, debug=True)
+        b.verify(case.target, case.kv, [0], torch.from_numpy(si2.draft_ids).cuda(), out, commit=False)
+        case.target.sync()
+        assert np.abs(out.dbg_logits.cpu().numpy()[0] - f2[0].logits).max() < 1e-3
+        assert int(out.accepted_len[0]) == v2[0].accepted_len and int(out.next_token[0]) == v2[0].next_token
+        # rollback to L and run the first step again: identical outputs
+        case.kv.rollback([0], [L])
+        g3 = case.run_gpu(orc.GREEDY, theta=0.5, commit=False)
+        for key in ("accepted_len", "next_token", "new_kv_len"):
+            assert np.array_equal(g1[key], g3[key])
+        assert np.array_equal(g1["logits"], g3["logits"])            # bit-reproducible
+        # rollback beyond the live length: refused by the host, or flagged by the device
+        with pytest.raises(b.SjError) as ei:
+            case.kv.rollback([0], [L + 100])
+        assert ei.value.status == 3
+    finally:
+        case.close()
+
+
+def test_page_pool_exhaustion_is_reported_before_any_launch():
+    b = _binding()
+    case = harness.Case(GQA, torch.float32, [30], 4, seed=2).gpu_setup(page_slack=0)
+    try:
+        # the pool holds pages for 30 + 5 tokens (+1); a long block needs more
+        with pytest.raises(b.SjError) as ei:
+            for _ in range(40):
+                case.run_gpu(orc.GREEDY, commit=True, debug=False)
+        assert ei.value.status == 4
+        case.target.sync()
+    finally:
+        case.close()
+
+
+def test_bit_reproducible_across_runs():
+    case = harness.Case(synth.TINY, torch.bfloat16, [128], 4, seed=0).gpu_setup()
+    try:
+        a = case.run_gpu(orc.SAMPLING, 1.0)
+        c = case.run_gpu(orc.SAMPLING, 1.0)
+        for k in a:
+            assert np.array_equal(a[k], c[k]), k
+    finally:
+        case.close()
