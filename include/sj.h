@@ -100,7 +100,8 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
 /* Runtime switches (for tests and measurements).  Names:
  *   "gemm_impl"  0 = CUDA-core kernels, 1 = tcgen05/TMA kernels (bf16 only; default for bf16)
  *   "attn_impl"  0 = CUDA-core kernel,  1 = tensor-core kernel  (bf16 only; default for bf16)
- *   "graph"      1 = replay the step as a CUDA graph (default), 0 = plain launches
+ *   "graph"      1 = replay the step as a CUDA graph (default unless the stream is NULL, which
+ *                cannot be captured), 0 = plain launches
  *   "pdl"        1 = programmatic dependent launch between the step's kernels (default)
  * Errors: INVALID_ARG for an unknown name, UNSUPPORTED for a value the dtype cannot honour. */
 sj_status sj_set_option(sj_target *t, const char *name, int value);

@@ -130,7 +130,7 @@ class Target:
         dt = top["embed"].dtype
         self.dtype = dt
         self.shape = shape
-        self.stream = stream if stream is not None else torch.cuda.current_stream()
+        self.stream = stream if stream is not None else torch.cuda.Stream()
         cfg = ModelConfig(shape.n_layers, shape.d_model, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                           shape.d_ffn, shape.vocab, shape.rope_theta, shape.rms_eps, _dtype_code(dt),
                           int(shape.tied_embeddings), int(shape.qkv_bias), max_rows)
@@ -176,12 +176,16 @@ class KVCache:
 
     def fill(self, seq: int, layer: int, start: int, k: torch.Tensor, v: torch.Tensor) -> None:
         assert k.dtype == self.target.dtype and v.dtype == self.target.dtype and k.shape == v.shape
+        self.target.stream.wait_stream(torch.cuda.current_stream())
+        k.record_stream(self.target.stream)
+        v.record_stream(self.target.stream)
         check(self._lib.sj_kv_fill(self.handle, seq, layer, start, k.shape[0], _ptr(k), _ptr(v)))
 
     def read(self, seq: int, layer: int, start: int, n: int):
         s = self.target.shape
         k = torch.empty((n, s.n_kv_heads, s.head_dim), dtype=self.target.dtype, device="cuda")
         v = torch.empty_like(k)
+        self.target.stream.wait_stream(torch.cuda.current_stream())
         check(self._lib.sj_kv_read(self.handle, seq, layer, start, n, _ptr(k), _ptr(v)))
         return k, v
 
@@ -240,6 +244,7 @@ def verify(target: Target, kv: KVCache, seq_ids: Sequence[int], draft_ids: torch
     args = VerifyArgs(B, gamma, ids, _ptr(draft_ids), _ptr(draft_q_tok), _ptr(draft_q_full), _ptr(uniforms), mode,
                       temperature, int(use_align), int(use_judge), theta, int(commit))
     o = out.struct()
+    target.stream.wait_stream(torch.cuda.current_stream())   # inputs were produced on the caller's stream
     check(target._lib.sj_verify(target.handle, kv.handle, C.byref(args), C.byref(o)))
 
 

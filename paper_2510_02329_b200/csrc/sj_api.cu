@@ -316,6 +316,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   const bool tc = tc_shapes_ok(c);
   t->opt_gemm = tc ? 1 : 0;
   t->opt_attn = 0;
+  t->opt_graph = t->stream ? 1 : 0;  // the legacy default stream cannot be captured
 
   sj_status st = SJ_OK;
   auto bail = [&](sj_status s) { sj_destroy_target(t); return s; };
@@ -331,10 +332,11 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     field = p_;                                                                       \
   } while (0)
   ALLOC(W.X, float, (size_t)R * c.d_model);
-  ALLOC(tmp, uint8_t, (size_t)R * c.d_model * esz); W.A = tmp;
-  ALLOC(tmp, uint8_t, (size_t)R * qd * esz); W.Q = tmp;
-  ALLOC(tmp, uint8_t, (size_t)R * qd * esz); W.ATT = tmp;
-  ALLOC(tmp, uint8_t, (size_t)R * c.d_ffn * esz); W.H = tmp;
+  const size_t act_rows = t->bf ? (size_t)2 * pad16(R) : (size_t)R;  // bf16: hi and lo planes
+  ALLOC(tmp, uint8_t, act_rows * c.d_model * esz); W.A = tmp;
+  ALLOC(W.Q, float, (size_t)R * qd);
+  ALLOC(tmp, uint8_t, act_rows * qd * esz); W.ATT = tmp;
+  ALLOC(tmp, uint8_t, act_rows * c.d_ffn * esz); W.H = tmp;
   ALLOC(W.Hf, float, (size_t)R * c.d_model);
   ALLOC(W.rope, float2, (size_t)R * (c.head_dim / 2));
   ALLOC(W.row_pos, int, R);
@@ -431,6 +433,7 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     if (value == 1) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention is not available in this build");
     t->opt_attn = value;
   } else if (n == "graph") {
+    if (value && !t->stream) return fail(SJ_ERR_UNSUPPORTED, "the legacy default stream cannot be captured into a graph");
     t->opt_graph = value ? 1 : 0;
   } else if (n == "pdl") {
     t->opt_pdl = value ? 1 : 0;
@@ -650,13 +653,19 @@ extern "C" sj_status sj_rollback_kv(sj_kv* kv, const int* seq_ids, const int* ne
 // ---------------------------------------------------------------------------------------------
 // the step
 // ---------------------------------------------------------------------------------------------
+// Rows handed to the MMA for R activation rows: both bf16 planes (hi at row 0, lo at row pad16(R)) while
+// they fit the 512 TMEM columns, else the hi plane alone.
+static bool planes_fit(int R) { return 2 * pad16(R) <= 512; }
+static int fed_rows(int R, bool planes) { return planes && planes_fit(R) ? 2 * pad16(R) : R; }
+
 static sj_status activation_map(sj_target* t, std::map<int, CUtensorMap>& cache, const void* base, int R, int K,
                                 const CUtensorMap** out) {
   auto it = cache.find(R);
   if (it == cache.end()) {
     CUtensorMap m;
-    RowGeom g = row_geom(R);
-    sj_status st = make_map(&m, base, R, K, g.nblk);
+    const int fed = fed_rows(R, true);
+    RowGeom g = row_geom(fed);
+    sj_status st = make_map(&m, base, fed, K, g.nblk);
     if (st != SJ_OK) return st;
     it = cache.emplace(R, m).first;
   }
@@ -665,10 +674,11 @@ static sj_status activation_map(sj_target* t, std::map<int, CUtensorMap>& cache,
 }
 
 static cudaError_t launch_tc(sj_target* t, const TcSite& s, const CUtensorMap* mA, const CUtensorMap* w0,
-                             const CUtensorMap* w1, const CUtensorMap* w2, int R, bool pdl) {
-  RowGeom g = row_geom(R);
+                             const CUtensorMap* w1, const CUtensorMap* w2, int R, bool pdl, bool planes) {
+  RowGeom g = row_geom(fed_rows(R, planes));
   TcGemmParams p;
   memset(&p, 0, sizeof(p));
+  p.lo_off = (planes && planes_fit(R)) ? pad16(R) : 0;
   p.n_tiles = s.n_tiles; p.KB = s.KB; p.G = s.G; p.U = (long long)s.n_tiles * s.KB; p.R = R;
   p.NB = g.NB; p.nblk = g.nblk; p.N_total = s.N;
   for (int i = 0; i < 3; ++i) p.seg_tile_end[i] = s.seg_tile_end[i];
@@ -682,7 +692,8 @@ static cudaError_t launch_tc(sj_target* t, const TcSite& s, const CUtensorMap* m
 
 template <typename T>
 static cudaError_t launch_simt(sj_target* t, const void* A, const GemmSegs& segs, float* Y, int R, int N, int K, bool pdl) {
-  return launch(k_gemm_simt<T, 8>, dim3((N + 7) / 8), dim3(256), 0, t->stream, pdl, (const T*)A, segs, Y, R, N, K);
+  return launch(k_gemm_simt<T, 8>, dim3((N + 7) / 8), dim3(256), 0, t->stream, pdl, (const T*)A, segs, Y, R, N, K,
+                t->bf ? 2 : 1);
 }
 
 template <typename T>
@@ -716,7 +727,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
     const LayerW& L = t->layers[l];
     // QKV projection
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_qkv, mA_d, &L.m_q, &L.m_k, &L.m_v, R, pdl));
+      CU_TRY(launch_tc(t, t->s_qkv, mA_d, &L.m_q, &L.m_k, &L.m_v, R, pdl, true));
     } else {
       GemmSegs g{{L.wq, L.wk, L.wv}, {qd, kd, kd}, 3};
       CU_TRY(launch_simt<T>(t, W.A, g, W.P, R, qd + 2 * kd, dm.d, pdl));
@@ -728,7 +739,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
     CU_TRY(launch(k_attn_combine<T>, dim3(R * dm.Hq), dim3(std::min(dm.hd, 128)), 0, s, pdl, args, W, dm));
     // O projection + residual + FFN norm
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_o, mA_q, &L.m_o, nullptr, nullptr, R, pdl));
+      CU_TRY(launch_tc(t, t->s_o, mA_q, &L.m_o, nullptr, nullptr, R, pdl, true));
     } else {
       GemmSegs g{{L.wo, nullptr, nullptr}, {dm.d, 0, 0}, 1};
       CU_TRY(launch_simt<T>(t, W.ATT, g, W.P, R, dm.d, qd, pdl));
@@ -737,7 +748,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
                   (const T*)L.nf, 0));
     // gate/up + SwiGLU
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_gu, mA_d, &L.m_g, &L.m_u, nullptr, R, pdl));
+      CU_TRY(launch_tc(t, t->s_gu, mA_d, &L.m_g, &L.m_u, nullptr, R, pdl, true));
     } else {
       GemmSegs g{{L.wg, L.wu, nullptr}, {dm.F, dm.F, 0}, 2};
       CU_TRY(launch_simt<T>(t, W.A, g, W.P, R, 2 * dm.F, dm.d, pdl));
@@ -746,7 +757,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
                   (size_t)R * 2 * dm.F));
     // down projection + residual + next norm
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_down, mA_f, &L.m_d, nullptr, nullptr, R, pdl));
+      CU_TRY(launch_tc(t, t->s_down, mA_f, &L.m_d, nullptr, nullptr, R, pdl, true));
     } else {
       GemmSegs g{{L.wd, nullptr, nullptr}, {dm.d, 0, 0}, 1};
       CU_TRY(launch_simt<T>(t, W.H, g, W.P, R, dm.d, dm.F, pdl));
@@ -759,7 +770,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   // LM head + statistics
   const int n_vtiles = (dm.V + kTileN - 1) / kTileN;
   if (tc) {
-    CU_TRY(launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl));
+    CU_TRY(launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl, true));
   } else {
     GemmSegs g{{t->lm_head, nullptr, nullptr}, {dm.V, 0, 0}, 1};
     CU_TRY(launch_simt<T>(t, W.A, g, W.logits, R, dm.V, dm.d, pdl));
@@ -931,9 +942,9 @@ extern "C" sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, co
   if (impl == 0) {
     GemmSegs g{{w, nullptr, nullptr}, {N, 0, 0}, 1};
     if (dtype == SJ_DTYPE_BF16)
-      CU_TRY(launch(k_gemm_simt<bf16, 8>, dim3((N + 7) / 8), dim3(256), 0, s, false, (const bf16*)a, g, y, R, N, K));
+      CU_TRY(launch(k_gemm_simt<bf16, 8>, dim3((N + 7) / 8), dim3(256), 0, s, false, (const bf16*)a, g, y, R, N, K, 1));
     else if (dtype == SJ_DTYPE_F32)
-      CU_TRY(launch(k_gemm_simt<float, 8>, dim3((N + 7) / 8), dim3(256), 0, s, false, (const float*)a, g, y, R, N, K));
+      CU_TRY(launch(k_gemm_simt<float, 8>, dim3((N + 7) / 8), dim3(256), 0, s, false, (const float*)a, g, y, R, N, K, 1));
     else
       return fail(SJ_ERR_INVALID_ARG, "unknown dtype");
     return SJ_OK;
@@ -967,7 +978,7 @@ extern "C" sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, co
   if ((st = make_map(&mA, a, R, K, g.nblk)) != SJ_OK) { cleanup(); return st; }
   if ((st = make_map(&mW, w, N, K, kTileN)) != SJ_OK) { cleanup(); return st; }
   cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess) e = launch_tc(&tmp, site, &mA, &mW, nullptr, nullptr, R, false);
+  if (e == cudaSuccess) e = launch_tc(&tmp, site, &mA, &mW, nullptr, nullptr, R, false, false);
   if (e == cudaSuccess)
     e = launch(k_sum_slots, dim3((unsigned)(((size_t)R * N + 255) / 256)), dim3(256), 0, s, false, (const float*)P,
                SplitPlan{site.d_tile_slots, site.n_tiles}, (size_t)R * N, R, N, y);

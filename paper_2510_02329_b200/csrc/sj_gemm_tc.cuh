@@ -33,6 +33,8 @@ struct TcGemmParams {
   int n_tiles, KB, G;
   long long U;          // n_tiles * KB
   int R;                // valid rows
+  int lo_off;           // > 0: activations come as hi/lo bf16 planes; the lo plane's accumulator
+                        // columns start at lo_off and are added to the hi columns in the epilogue
   int NB, nblk;         // activation rows are fed as NB blocks of nblk rows (nblk % 16 == 0, <= 256)
   int N_total;          // output features (all segments)
   int seg_tile_end[3];  // exclusive prefix of tiles per weight segment
@@ -305,6 +307,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         for (int c0 = 0; c0 < p.R; c0 += 16) {
           float v[16];
           tc_ld16(taddr + c0, v);
+          if (p.lo_off) {
+            float lo[16];
+            tc_ld16(taddr + p.lo_off + c0, lo);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += lo[i];
+          }
           if (n < p.N_total) {
 #pragma unroll
             for (int i = 0; i < 16; ++i)
@@ -315,6 +323,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         for (int c0 = 0; c0 < p.R; c0 += 16) {
           float v[16];
           tc_ld16(taddr + c0, v);
+          if (p.lo_off) {
+            float lo[16];
+            tc_ld16(taddr + p.lo_off + c0, lo);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += lo[i];
+          }
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const int r = c0 + i;

@@ -9,10 +9,14 @@ namespace sj {
 // Device workspace of one target (all sized for max_rows).
 struct Work {
   float* X;          // [R, d]        fp32 residual stream
-  void* A;           // [R, d]        T  normalised activations (input of QKV / gate-up / LM head)
-  void* Q;           // [R, Hq*hd]    T  rotated queries
-  void* ATT;         // [R, Hq*hd]    T  attention output (input of the O projection)
-  void* H;           // [R, F]        T  silu(gate)*up (input of the down projection)
+  // GEMM inputs.  fp32 models: one plane [R, K] of floats.  bf16 models: TWO bf16 planes
+  // [2][Rp][K] (Rp = R rounded up to 16): plane 0 holds bf16(x), plane 1 holds bf16(x - plane 0), so
+  // that the tensor cores see x to ~2^-17 instead of 2^-9; the product with both planes is summed
+  // in the fp32 accumulator's epilogue.
+  void* A;           // normalised activations (input of QKV / gate-up / LM head), K = d
+  float* Q;          // [R, Hq*hd]    fp32 rotated queries
+  void* ATT;         // attention output (input of the O projection), K = Hq*hd
+  void* H;           // silu(gate)*up (input of the down projection), K = F
   float* P;          // partial sums of the current GEMM: [slot][R][N]
   float* Hf;         // [R, d]        fp32 hidden state after the final norm
   float2* rope;      // [R, hd/2]     (cos, sin) of this step's positions
@@ -34,6 +38,21 @@ struct Dims {
   int n_layers, d, Hq, Hkv, hd, F, V;
   float eps;
 };
+
+__host__ __device__ __forceinline__ int pad16(int r) { return (r + 15) & ~15; }
+
+// Store one GEMM-input element (row r of R, column i of K).
+template <typename T> __device__ __forceinline__ void store_act(void* base, int R, int K, int r, int i, float y);
+template <> __device__ __forceinline__ void store_act<float>(void* base, int R, int K, int r, int i, float y) {
+  reinterpret_cast<float*>(base)[(size_t)r * K + i] = y;
+}
+template <> __device__ __forceinline__ void store_act<bf16>(void* base, int R, int K, int r, int i, float y) {
+  bf16 hi = __float2bfloat16_rn(y);
+  bf16 lo = __float2bfloat16_rn(y - __bfloat162float(hi));
+  bf16* b = reinterpret_cast<bf16*>(base);
+  b[(size_t)r * K + i] = hi;
+  b[((size_t)pad16(R) + r) * K + i] = lo;
+}
 
 // ---------------------------------------------------------------------------------------------
 // step set-up: row positions and the attention chunk list (needs the true cache lengths)
@@ -62,14 +81,14 @@ __global__ void k_plan(const StepArgs* __restrict__ args, KvView kv, Work w, int
 // RMSNorm of a row held in shared memory; writes T activations and optional fp32 copies.
 template <typename T>
 __device__ __forceinline__ void norm_row_from_smem(const float* xs, int d, const T* __restrict__ gain, float eps,
-                                                   T* a_row, float* hf_row, float* dbg_row, float* red) {
+                                                   void* act, int R, int r, float* hf_row, float* dbg_row, float* red) {
   float ss = 0.f;
   for (int i = threadIdx.x; i < d; i += blockDim.x) ss += xs[i] * xs[i];
   ss = block_sum(ss, red);
   float inv = 1.0f / sqrtf(ss / (float)d + eps);
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float y = xs[i] * inv * to_f(gain[i]);
-    a_row[i] = from_f<T>(y);
+    store_act<T>(act, R, d, r, i, y);
     if (hf_row) hf_row[i] = y;
     if (dbg_row) dbg_row[i] = y;
   }
@@ -101,7 +120,7 @@ __global__ void k_embed_norm(const StepArgs* __restrict__ args, KvView kv, Work 
     w.rope[(size_t)r * (dm.hd / 2) + i] = make_float2((float)c, (float)s);
   }
   __syncthreads();
-  norm_row_from_smem<T>(xs, dm.d, gain, dm.eps, reinterpret_cast<T*>(w.A) + (size_t)r * dm.d, nullptr, nullptr, red);
+  norm_row_from_smem<T>(xs, dm.d, gain, dm.eps, w.A, gridDim.x, r, nullptr, nullptr, red);
 }
 
 // a6/a8 tail + a2/a9: X += sum of partials; A = RMSNorm(X) * gain.  final: also fp32 hidden.
@@ -121,7 +140,7 @@ __global__ void k_reduce_norm(const StepArgs* __restrict__ args, Work w, Dims dm
   __syncthreads();
   float* hf = final_norm ? w.Hf + (size_t)r * dm.d : nullptr;
   float* dbg = (final_norm && args->dbg_hidden) ? args->dbg_hidden + (size_t)r * dm.d : nullptr;
-  norm_row_from_smem<T>(xs, dm.d, gain, dm.eps, reinterpret_cast<T*>(w.A) + (size_t)r * dm.d, hf, dbg, red);
+  norm_row_from_smem<T>(xs, dm.d, gain, dm.eps, w.A, gridDim.x, r, hf, dbg, red);
 }
 
 // a3 tail + a4: reduce QKV partials, add bias, rotate q and k, store q, append k and v rows.
@@ -155,9 +174,9 @@ __global__ void k_qkv_rope(const StepArgs* __restrict__ args, KvView kv, Work w,
     float y1 = x1 * cs.x - x2 * cs.y;
     float y2 = x2 * cs.x + x1 * cs.y;
     if (head < dm.Hq) {
-      T* q = reinterpret_cast<T*>(w.Q) + (size_t)r * qd;
-      q[n1] = from_f<T>(y1);
-      q[n2] = from_f<T>(y2);
+      float* q = w.Q + (size_t)r * qd;
+      q[n1] = y1;
+      q[n2] = y2;
     } else {
       T* krow = kv_row<T>(kv, layer, page, 0, head - dm.Hq, slot);
       krow[i] = from_f<T>(y1);
@@ -183,7 +202,7 @@ __global__ void k_swiglu(Work w, Dims dm, SplitPlan sp, size_t slot_stride) {
   float g = reduce_partials(w.P, sp, slot_stride, 2 * dm.F, r, f);
   float u = reduce_partials(w.P, sp, slot_stride, 2 * dm.F, r, dm.F + f);
   float y = g / (1.0f + expf(-g)) * u;
-  reinterpret_cast<T*>(w.H)[(size_t)r * dm.F + f] = from_f<T>(y);
+  store_act<T>(w.H, gridDim.y, dm.F, r, f, y);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -211,8 +230,10 @@ __device__ __forceinline__ void unpack(const uint4& v, float* f) {
   }
 }
 
+// `planes` = 2: the input is a hi/lo pair of bf16 planes (see Work); the two are added before use.
 template <typename T, int RT>
-__global__ void k_gemm_simt(const T* __restrict__ A, GemmSegs segs, float* __restrict__ Y, int R, int N, int K) {
+__global__ void k_gemm_simt(const T* __restrict__ A, GemmSegs segs, float* __restrict__ Y, int R, int N, int K,
+                            int planes) {
   pdl_wait();
   pdl_launch();
   constexpr int VN = Vec<T>::n;
@@ -235,6 +256,12 @@ __global__ void k_gemm_simt(const T* __restrict__ A, GemmSegs segs, float* __res
         if (r0 + i < R) {
           float af[VN];
           unpack(*reinterpret_cast<const V*>(A + (size_t)(r0 + i) * K + k), af);
+          if (planes == 2) {
+            float lo[VN];
+            unpack(*reinterpret_cast<const V*>(A + ((size_t)pad16(R) + r0 + i) * K + k), lo);
+#pragma unroll
+            for (int e = 0; e < VN; ++e) af[e] += lo[e];
+          }
 #pragma unroll
           for (int e = 0; e < VN; ++e) acc[i] = fmaf(af[e], wf[e], acc[i]);
         }
@@ -295,8 +322,8 @@ __global__ void k_attn_simt(const StepArgs* __restrict__ args, KvView kv, Work w
     // queries of this KV head's group: q index = g * rows + j
     for (int i = tid; i < nq * hd; i += kAttThreads) {
       int q = i / hd, dd = i % hd, g = q / rows, j = q % rows;
-      const T* qrow = reinterpret_cast<const T*>(w.Q) + (size_t)(b * rows + j) * (dm.Hq * hd) + (kvh * group + g) * hd;
-      qs[i] = to_f(qrow[dd]);
+      const float* qrow = w.Q + (size_t)(b * rows + j) * (dm.Hq * hd) + (kvh * group + g) * hd;
+      qs[i] = qrow[dd];
     }
     for (int q = tid; q < nq; q += kAttThreads) { m_run[q] = -INFINITY; l_run[q] = 0.f; }
     float acc[48];
@@ -406,7 +433,7 @@ __global__ void k_attn_combine(const StepArgs* __restrict__ args, Work w, Dims d
       float m = w.att_m[pi];
       if (m != -INFINITY) o += w.att_o[pi * dm.hd + dd] * expf(m - M);
     }
-    reinterpret_cast<T*>(w.ATT)[(size_t)r * (dm.Hq * dm.hd) + h * dm.hd + dd] = from_f<T>(o / Lsum);
+    store_act<T>(w.ATT, gridDim.x / dm.Hq, dm.Hq * dm.hd, r, h * dm.hd + dd, o / Lsum);
   }
 }
 
