@@ -1,0 +1,398 @@
+#!/usr/bin/env python
+"""Benchmark of the verification step (one step = the whole hot path over one batch of drafts).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.  ``value`` is positions verified per second over all GPUs (each
+sequence's step verifies gamma drafted positions plus the bonus position), with weights, cache and
+inputs resident in HBM; ``e2e`` is the same metric with the step's inputs copied from pinned host
+memory and its results copied back inside the timed region.  With N > 1 every rank runs an
+independent replica on its own sequences (the path has no exchange step): weak scaling.
+``--impl reference`` times the CPU oracle on the host cores on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+import numpy as np
+import torch
+
+from paper_2510_02329_b200 import synth
+
+METRIC = "verified_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ----------------------------------------------------------------------------------------------
+# helpers
+# ----------------------------------------------------------------------------------------------
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        busy = [x for x in sm if x >= 0.5 * max(sm)]
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def reduce_max_and_sum(ms_local: float, units_local: float, world: int, device=None):
+    """max over ranks of the elapsed time, sum over ranks of the units processed."""
+    if world == 1:
+        return ms_local, units_local
+    import torch.distributed as dist
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and the reference arm)
+# ----------------------------------------------------------------------------------------------
+class OracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of a workload.
+
+    The sample is `n_layers` decoder layers, the LM head over the first vocab/`vocab_div` tokens, and
+    (once, in `acceptance_seconds`) the acceptance rule on full-vocabulary logits, for at most two
+    sequences with the cache capped at 2048 tokens.  `time_step()` runs the sample once and returns
+    the seconds scaled to the whole step (layers by count, head by vocabulary share, total by
+    sequence count).  Weight conversion to fp64 is done at set-up, outside the timing.
+    """
+
+    def __init__(self, wl: synth.Workload, n_layers: int, vocab_div: int = 1, seed: int = 0):
+        import helpers
+        from oracle import sj_oracle as orc
+        self.orc, self.wl = orc, wl
+        shape = wl.shape
+        self.n_layers = n_layers
+        cut = shape.cut(n_layers)
+        gen = "cuda" if torch.cuda.is_available() else "cpu"
+        dtype = torch.bfloat16
+        self.lens = [int(min(x, 2048)) for x in synth.kv_lengths(wl, seed)[:2]]
+        self.nseq = len(self.lens)
+        self.osh = helpers.oracle_shape(cut)
+        self.vs = shape.vocab // vocab_div
+        self.vocab_div = vocab_div
+        layers = [synth.layer_weights(cut, l, dtype, gen, seed) for l in range(n_layers)]
+        self.layers64 = [{k: helpers.np64(v) for k, v in lw.items()} for lw in layers]
+        del layers
+        top = synth.top_weights(cut, dtype, gen, seed)
+        self.si = synth.step_inputs(shape.vocab, self.nseq, wl.gamma, seed)
+        self.tokens = [np.concatenate([[int(self.si.pending[b])], self.si.draft_ids[b].astype(np.int64)])
+                       for b in range(self.nseq)]
+        need = np.unique(np.concatenate(self.tokens))
+        # the oracle indexes the embedding by token id: keep only the rows the sample touches
+        rows = helpers.np64(top["embed"][torch.from_numpy(need).to(top["embed"].device)])
+        self.tok_local = [np.searchsorted(need, t) for t in self.tokens]
+        self.top64 = {"embed": rows, "final_norm": helpers.np64(top["final_norm"]),
+                      "lm_head": helpers.np64(top["lm_head"][: self.vs])}
+        self.caches = [[tuple(helpers.np64(t) for t in synth.cache_fill(cut, l, b, self.lens[b], dtype, gen, seed))
+                        for l in range(n_layers)] for b in range(self.nseq)]
+        self.judge_w = helpers.np64(synth.judge_head(cut, gen, seed))
+        del top
+        try:
+            import threadpoolctl
+            self.threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
+        except Exception:
+            self.threads = os.cpu_count() or 1
+        # acceptance rule on full-vocabulary logits, timed once
+        rng = np.random.default_rng(0)
+        logits = rng.standard_normal((wl.gamma + 1, shape.vocab)) * 1.28
+        hidden = rng.standard_normal((wl.gamma + 1, shape.d_model))
+        t0 = time.perf_counter()
+        orc.verdict(logits, hidden, self.si.draft_ids[0], self.lens[0], mode=orc.GREEDY, judge_w=self.judge_w, theta=0.5)
+        self.acceptance_seconds = time.perf_counter() - t0
+
+    def describe(self) -> str:
+        return (f"{self.n_layers} of {self.wl.shape.n_layers} layers + LM head over 1/{self.vocab_div} of the vocabulary "
+                f"+ acceptance rule, {self.nseq} of {self.wl.batch} sequence(s), cache capped at 2048 tokens; scaled by "
+                f"layer count, vocabulary share and sequence count")
+
+    def time_step(self) -> float:
+        orc, osh = self.orc, self.osh
+        t0 = time.perf_counter()
+        orc.forward_blocks(osh, self.top64, lambda l: self.layers64[l], self.tok_local, self.caches)
+        t1 = time.perf_counter()
+        head_only = orc.Shape(0, osh.d_model, osh.n_q_heads, osh.n_kv_heads, osh.head_dim, osh.d_ffn, self.vs,
+                              osh.rope_theta, osh.rms_eps)
+        orc.forward_blocks(head_only, self.top64, None, self.tok_local, [[] for _ in range(self.nseq)])
+        t2 = time.perf_counter()
+        t_head = t2 - t1
+        t_layers = max((t1 - t0) - t_head, 1e-9)
+        per_seq = (t_layers * self.wl.shape.n_layers / self.n_layers + t_head * self.vocab_div) / self.nseq \
+            + self.acceptance_seconds
+        return per_seq * self.wl.batch
+
+
+def run_reference(args, wl, rank, world):
+    if rank != 0:
+        return
+    R = wl.batch * (wl.gamma + 1)
+    sample = OracleSample(wl, max(1, args.ref_layers), vocab_div=8)
+    times = []
+    for i in range(args.warmup + args.steps):
+        full = sample.time_step()
+        if i >= args.warmup:
+            times.append(full)
+    ms = 1e3 * sum(times) / len(times)
+    value = R / (ms / 1e3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "batch": wl.batch, "gamma": wl.gamma, "kv_len": wl.kv_len,
+                       "positions_per_step": R},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": sample.threads, "kind": "oracle",
+                             "sample": sample.describe()},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# main arm
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg3", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--mode", default="greedy", choices=["greedy", "sampling"])
+    ap.add_argument("--layers", type=int, default=0, help="cut the model to this many layers (profiling only)")
+    ap.add_argument("--ref-layers", type=int, default=1, help="layers in the reference arm's per-step sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-breakdown", action="store_true")
+    ap.add_argument("--set", action="append", default=[], help="library option name=value")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank, local_rank, world = dist_env()
+    wl = synth.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank, world)
+        return
+
+    from paper_2510_02329_b200 import binding
+    from paper_2510_02329_b200.workload import DeviceWorkload
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    mode = binding.MODE_SAMPLING if args.mode == "sampling" else binding.MODE_GREEDY
+
+    dw = DeviceWorkload(wl, torch.bfloat16, seed=rank, n_layers=args.layers or None)
+    for kvs in args.set:
+        k, v = kvs.split("=")
+        dw.target.set_option(k, int(v))
+    stream = dw.target.stream
+    R = dw.R
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- device-resident timing ----------------
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            dw.step(mode)
+        dw.target.sync()
+        with ClockSampler(local_rank) as clk:
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                dw.step(mode)
+            e1.record(stream)
+            barrier()
+            ms_total = e0.elapsed_time(e1)
+            dw.target.sync()
+
+            # ---------------- end to end: host buffers in, results out, every step ----------------
+            si = dw.inputs
+            h_in = {"draft": torch.from_numpy(si.draft_ids).pin_memory(), "unif": torch.from_numpy(si.uniforms).pin_memory(),
+                    "qtok": torch.from_numpy(si.draft_q_tok).pin_memory()}
+            if mode == binding.MODE_SAMPLING:
+                h_in["qfull"] = torch.from_numpy(si.draft_q_full).pin_memory()
+            out = dw.out
+            h_out = {k: torch.empty_like(getattr(out, k), device="cpu").pin_memory()
+                     for k in ("accepted_len", "next_token", "judge_scores", "new_kv_len")}
+            h2d = sum(t.numel() * t.element_size() for t in h_in.values()) + 4 * dw.B
+            d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+
+            def e2e_step():
+                dw.d_draft.copy_(h_in["draft"], non_blocking=True)
+                dw.d_unif.copy_(h_in["unif"], non_blocking=True)
+                dw.d_qtok.copy_(h_in["qtok"], non_blocking=True)
+                if "qfull" in h_in:
+                    dw.d_qfull.copy_(h_in["qfull"], non_blocking=True)
+                dw.step(mode)
+                for k, t in h_out.items():
+                    t.copy_(getattr(out, k), non_blocking=True)
+                stream.synchronize()
+
+            for _ in range(3):
+                e2e_step()
+            barrier()
+            n_e2e = max(10, args.steps // 2)
+            e0.record(stream)
+            for _ in range(n_e2e):
+                e2e_step()
+            e1.record(stream)
+            barrier()
+            ms_e2e_total = e0.elapsed_time(e1)
+        clocks = clk.summary()
+        accepted = out.accepted_len.cpu().numpy()
+
+    ms_step_local = ms_total / args.steps
+    ms_step, units = reduce_max_and_sum(ms_step_local, float(R), world, device="cuda")
+    ms_e2e, _ = reduce_max_and_sum(ms_e2e_total / n_e2e, float(R), world, device="cuda")
+    value = units / (ms_step / 1e3)
+    e2e_value = units / (ms_e2e / 1e3)
+
+    if rank != 0:
+        dw.close()
+        return
+
+    peak, peak_kind = measured_peaks()
+    w_bytes, kv_bytes = dw.weight_bytes(), dw.kv_bytes()
+    step_gbs = (w_bytes + kv_bytes) / (ms_step_local / 1e3) / 1e9
+
+    # ---------------- dominant kernel: event-bracketed launches (instrumented pass) ----------------
+    roofline = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": None,
+                "peak_kind": peak_kind}
+    breakdown = {}
+    if not args.no_breakdown:
+        with torch.cuda.stream(stream):
+            dw.target.set_option("graph", 0)
+            dw.target.set_option("timing", 1)
+            n_inst = 3
+            dw.step(mode)                      # untimed: settles allocations
+            dw.target.set_option("timing", 1)  # clears the records
+            for _ in range(n_inst):
+                dw.step(mode)
+            dw.target.sync()
+            tot = 0.0
+            for name in ("plan", "embed_norm", "gemm_qkv", "gemm_o", "gemm_gateup", "gemm_down", "gemm_lm_head",
+                         "qkv_rope", "attn_combine", "reduce_norm", "swiglu", "finalize", "resample"):
+                ms, n = dw.target.kernel_time(name)
+                if n:
+                    breakdown[name] = {"launches_per_step": n // n_inst, "ms_per_step": ms / n_inst}
+                    tot += ms / n_inst
+            ms_a, n_a = dw.target.kernel_time("attn")
+            ms_c, n_c = dw.target.kernel_time("attn_combine")
+            breakdown["attn"] = {"launches_per_step": (n_a - n_c) // n_inst, "ms_per_step": (ms_a - ms_c) / n_inst}
+            tot += (ms_a - ms_c) / n_inst
+            for v in breakdown.values():
+                v["share"] = v["ms_per_step"] / tot
+            g_ms, g_n = dw.target.kernel_time("gemm")
+            dw.target.set_option("timing", 0)
+            dw.target.set_option("graph", 1)
+        # k_gemm_tc: all projections + LM head; algorithmic bytes = every streamed weight byte once
+        per_launch_bytes = w_bytes / (g_n / n_inst)
+        per_launch_s = (g_ms / g_n) / 1e3
+        roofline.update({"kernel": "k_gemm_tc", "launches_per_step": g_n // n_inst,
+                         "achieved": per_launch_bytes / per_launch_s / 1e9,
+                         "avg_launch_us": per_launch_s * 1e6, "algorithmic_bytes_per_launch": per_launch_bytes})
+        roofline["frac"] = roofline["achieved"] / peak
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline and world == 1:
+        t0 = time.perf_counter()
+        sample = OracleSample(wl, min(4, wl.shape.n_layers), vocab_div=1)
+        full = min(sample.time_step() for _ in range(2))
+        cpu_baseline = {"value": R / full, "unit": UNIT, "cores": sample.threads, "kind": "oracle",
+                        "sample": sample.describe(), "seconds_spent": time.perf_counter() - t0}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "shape": dw.shape.name, "layers": dw.shape.n_layers, "batch": wl.batch,
+                   "gamma": wl.gamma, "kv_len_total": int(sum(dw.kv_lens)), "mode": args.mode, "replicas": world,
+                   "positions_per_step": R, "l2": "inputs larger than L2 (weights stream from HBM every step)"},
+        "verify_steps_per_s": world * 1e3 / ms_step,
+        "committed_tokens_per_s": float((accepted + 1).sum()) * world * 1e3 / ms_step,
+        "step_hbm_gbs": step_gbs, "step_hbm_frac_of_measured_copy": step_gbs / peak, "step_hbm_frac_of_8tbs": step_gbs / 8000.0,
+        "algorithmic_bytes_per_step": w_bytes + kv_bytes,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e},
+        "gpu_launches": dw.launches_per_step(mode) * args.steps,
+        "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline, "kernel_breakdown": breakdown,
+    }
+    print(json.dumps(line))
+    dw.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -103,8 +103,15 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *   "graph"      1 = replay the step as a CUDA graph (default unless the stream is NULL, which
  *                cannot be captured), 0 = plain launches
  *   "pdl"        1 = programmatic dependent launch between the step's kernels (default)
+ *   "timing"     1 = bracket every kernel launch of a step with CUDA events (needs "graph" 0; turns
+ *                programmatic launches off for those steps); setting it (0 or 1) clears old records
  * Errors: INVALID_ARG for an unknown name, UNSUPPORTED for a value the dtype cannot honour. */
 sj_status sj_set_option(sj_target *t, const char *name, int value);
+
+/* Device time of the launches recorded under "timing" whose kernel name starts with `name`
+ * ("gemm", "gemm_gateup", "attn", "reduce_norm", ...): sum of event-bracketed durations and their
+ * count.  Synchronises the stream. */
+sj_status sj_kernel_time(sj_target *t, const char *name, double *total_ms, long *launches);
 
 /* Wait for the target's stream and return the device status word (SJ_OK, SJ_ERR_TIMEOUT,
  * SJ_ERR_STATE ...), clearing it. */

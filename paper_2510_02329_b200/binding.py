@@ -23,7 +23,7 @@ MODE_GREEDY, MODE_SAMPLING = 0, 1
 
 EXPORTS = ["sj_create_target", "sj_destroy_target", "sj_load_judge_head", "sj_set_option", "sj_sync",
            "sj_kv_create", "sj_kv_destroy", "sj_kv_fill", "sj_kv_read", "sj_kv_set_len", "sj_kv_set_pending",
-           "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_last_error"]
+           "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_last_error", "sj_kernel_time"]
 
 
 class SjError(RuntimeError):
@@ -84,6 +84,7 @@ def load(build_if_needed: bool = True) -> C.CDLL:
     lib.sj_load_judge_head.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_float, C.c_float]
     lib.sj_set_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int]
     lib.sj_sync.argtypes = [C.c_void_p]
+    lib.sj_kernel_time.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_double), C.POINTER(C.c_long)]
     lib.sj_kv_create.argtypes = [C.c_void_p, C.c_int, C.c_long, C.c_int, C.POINTER(C.c_void_p)]
     lib.sj_kv_destroy.argtypes = [C.c_void_p]
     lib.sj_kv_fill.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
@@ -154,6 +155,12 @@ class Target:
 
     def sync(self) -> None:
         check(self._lib.sj_sync(self.handle))
+
+    def kernel_time(self, name: str):
+        """(total ms, launches) of the event-bracketed launches whose name starts with ``name``."""
+        ms, n = C.c_double(), C.c_long()
+        check(self._lib.sj_kernel_time(self.handle, name.encode(), C.byref(ms), C.byref(n)))
+        return ms.value, n.value
 
     def close(self) -> None:
         if self.handle:

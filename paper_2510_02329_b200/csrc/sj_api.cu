@@ -186,7 +186,9 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0;
+  struct Timed { const char* name; cudaEvent_t a, b; };
+  std::vector<Timed> timed;
   TcSite s_qkv, s_o, s_gu, s_down, s_lm;
   size_t p_elems = 0;
   size_t att_chunks_cap = 0;
@@ -404,6 +406,7 @@ extern "C" sj_status sj_destroy_target(sj_target* t) {
   if (!t) return SJ_OK;
   cudaStreamSynchronize(t->stream);
   clear_graphs(t);
+  for (auto& e : t->timed) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
   for (void* p : t->owned) cudaFree(p);
   delete t;
   cudaGetLastError();
@@ -437,6 +440,11 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     t->opt_graph = value ? 1 : 0;
   } else if (n == "pdl") {
     t->opt_pdl = value ? 1 : 0;
+  } else if (n == "timing") {
+    cudaStreamSynchronize(t->stream);
+    for (auto& e : t->timed) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+    t->timed.clear();
+    t->opt_timing = value ? 1 : 0;
   } else {
     return fail(SJ_ERR_INVALID_ARG, "unknown option '%s'", name);
   }
@@ -696,12 +704,29 @@ static cudaError_t launch_simt(sj_target* t, const void* A, const GemmSegs& segs
                 t->bf ? 2 : 1);
 }
 
+// Launch `expr`; in timing mode bracket it with events filed under `name`.
+#define TIMED(name, expr)                                                        \
+  do {                                                                           \
+    cudaEvent_t ea_ = nullptr, eb_ = nullptr;                                    \
+    if (timing) {                                                                \
+      CU_TRY(cudaEventCreate(&ea_));                                             \
+      CU_TRY(cudaEventCreate(&eb_));                                             \
+      CU_TRY(cudaEventRecord(ea_, s));                                           \
+    }                                                                            \
+    CU_TRY(expr);                                                                \
+    if (timing) {                                                                \
+      CU_TRY(cudaEventRecord(eb_, s));                                           \
+      t->timed.push_back({name, ea_, eb_});                                      \
+    }                                                                            \
+  } while (0)
+
 template <typename T>
 static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mode, int chunk_len, bool use_scratch,
                                size_t n_chunks_hi) {
   const Dims& dm = t->dm;
   const int R = B * (gamma + 1), qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd;
-  const bool pdl = t->opt_pdl != 0, tc = t->opt_gemm == 1;
+  const bool timing = t->opt_timing != 0 && !t->opt_graph;
+  const bool pdl = t->opt_pdl != 0 && !timing, tc = t->opt_gemm == 1;
   const StepArgs* args = t->d_args;
   Work W = t->work;
   if (!use_scratch) W.logits = nullptr;
@@ -717,8 +742,8 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   }
   auto plan_of = [&](const TcSite& site) { return tc ? SplitPlan{site.d_tile_slots, site.n_tiles} : one; };
 
-  CU_TRY(launch(k_plan, dim3(1), dim3(256), 0, s, false, args, kv->view, W, chunk_len));
-  CU_TRY(launch(k_embed_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, kv->view, W, dm, (const T*)t->embed,
+  TIMED("plan", launch(k_plan, dim3(1), dim3(256), 0, s, false, args, kv->view, W, chunk_len));
+  TIMED("embed_norm", launch(k_embed_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, kv->view, W, dm, (const T*)t->embed,
                 (const T*)t->layers[0].na));
   const int nq = (dm.Hq / dm.Hkv) * (gamma + 1);
   const size_t att_smem = sizeof(float) * ((size_t)nq * dm.hd + kAttKT * (dm.hd + 1) + kAttKT * dm.hd + (size_t)nq * kAttKT + 3 * nq);
@@ -727,57 +752,77 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
     const LayerW& L = t->layers[l];
     // QKV projection
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_qkv, mA_d, &L.m_q, &L.m_k, &L.m_v, R, pdl, true));
+      TIMED("gemm_qkv", launch_tc(t, t->s_qkv, mA_d, &L.m_q, &L.m_k, &L.m_v, R, pdl, true));
     } else {
       GemmSegs g{{L.wq, L.wk, L.wv}, {qd, kd, kd}, 3};
-      CU_TRY(launch_simt<T>(t, W.A, g, W.P, R, qd + 2 * kd, dm.d, pdl));
+      TIMED("gemm_cudacore", launch_simt<T>(t, W.A, g, W.P, R, qd + 2 * kd, dm.d, pdl));
     }
-    CU_TRY(launch(k_qkv_rope<T>, dim3(R), dim3(256), 0, s, pdl, args, kv->view, W, dm, plan_of(t->s_qkv),
+    TIMED("qkv_rope", launch(k_qkv_rope<T>, dim3(R), dim3(256), 0, s, pdl, args, kv->view, W, dm, plan_of(t->s_qkv),
                   (size_t)R * (qd + 2 * kd), l, (const T*)L.bq, (const T*)L.bk, (const T*)L.bv));
     // attention
-    CU_TRY(launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
-    CU_TRY(launch(k_attn_combine<T>, dim3(R * dm.Hq), dim3(std::min(dm.hd, 128)), 0, s, pdl, args, W, dm));
+    TIMED("attn", launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
+    TIMED("attn_combine", launch(k_attn_combine<T>, dim3(R * dm.Hq), dim3(std::min(dm.hd, 128)), 0, s, pdl, args, W, dm));
     // O projection + residual + FFN norm
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_o, mA_q, &L.m_o, nullptr, nullptr, R, pdl, true));
+      TIMED("gemm_o", launch_tc(t, t->s_o, mA_q, &L.m_o, nullptr, nullptr, R, pdl, true));
     } else {
       GemmSegs g{{L.wo, nullptr, nullptr}, {dm.d, 0, 0}, 1};
-      CU_TRY(launch_simt<T>(t, W.ATT, g, W.P, R, dm.d, qd, pdl));
+      TIMED("gemm_cudacore", launch_simt<T>(t, W.ATT, g, W.P, R, dm.d, qd, pdl));
     }
-    CU_TRY(launch(k_reduce_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, W, dm, plan_of(t->s_o), (size_t)R * dm.d,
+    TIMED("reduce_norm", launch(k_reduce_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, W, dm, plan_of(t->s_o), (size_t)R * dm.d,
                   (const T*)L.nf, 0));
     // gate/up + SwiGLU
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_gu, mA_d, &L.m_g, &L.m_u, nullptr, R, pdl, true));
+      TIMED("gemm_gateup", launch_tc(t, t->s_gu, mA_d, &L.m_g, &L.m_u, nullptr, R, pdl, true));
     } else {
       GemmSegs g{{L.wg, L.wu, nullptr}, {dm.F, dm.F, 0}, 2};
-      CU_TRY(launch_simt<T>(t, W.A, g, W.P, R, 2 * dm.F, dm.d, pdl));
+      TIMED("gemm_cudacore", launch_simt<T>(t, W.A, g, W.P, R, 2 * dm.F, dm.d, pdl));
     }
-    CU_TRY(launch(k_swiglu<T>, dim3((dm.F + 255) / 256, R), dim3(256), 0, s, pdl, W, dm, plan_of(t->s_gu),
+    TIMED("swiglu", launch(k_swiglu<T>, dim3((dm.F + 255) / 256, R), dim3(256), 0, s, pdl, W, dm, plan_of(t->s_gu),
                   (size_t)R * 2 * dm.F));
     // down projection + residual + next norm
     if (tc) {
-      CU_TRY(launch_tc(t, t->s_down, mA_f, &L.m_d, nullptr, nullptr, R, pdl, true));
+      TIMED("gemm_down", launch_tc(t, t->s_down, mA_f, &L.m_d, nullptr, nullptr, R, pdl, true));
     } else {
       GemmSegs g{{L.wd, nullptr, nullptr}, {dm.d, 0, 0}, 1};
-      CU_TRY(launch_simt<T>(t, W.H, g, W.P, R, dm.d, dm.F, pdl));
+      TIMED("gemm_cudacore", launch_simt<T>(t, W.H, g, W.P, R, dm.d, dm.F, pdl));
     }
     const bool last = (l == dm.n_layers - 1);
     const void* gain = last ? t->final_norm : t->layers[l + 1].na;
-    CU_TRY(launch(k_reduce_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, W, dm, plan_of(t->s_down),
+    TIMED("reduce_norm", launch(k_reduce_norm<T>, dim3(R), dim3(256), row_smem, s, pdl, args, W, dm, plan_of(t->s_down),
                   (size_t)R * dm.d, (const T*)gain, last ? 1 : 0));
   }
   // LM head + statistics
   const int n_vtiles = (dm.V + kTileN - 1) / kTileN;
   if (tc) {
-    CU_TRY(launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl, true));
+    TIMED("gemm_lm_head", launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl, true));
   } else {
     GemmSegs g{{t->lm_head, nullptr, nullptr}, {dm.V, 0, 0}, 1};
-    CU_TRY(launch_simt<T>(t, W.A, g, W.logits, R, dm.V, dm.d, pdl));
-    CU_TRY(launch(k_lm_stats_from_logits, dim3(n_vtiles, (R + 7) / 8), dim3(256), 0, s, pdl, args, W, dm, R));
+    TIMED("gemm_cudacore", launch_simt<T>(t, W.A, g, W.logits, R, dm.V, dm.d, pdl));
+    TIMED("lm_stats", launch(k_lm_stats_from_logits, dim3(n_vtiles, (R + 7) / 8), dim3(256), 0, s, pdl, args, W, dm, R));
   }
-  CU_TRY(launch(k_finalize, dim3(B), dim3(256), 0, s, pdl, args, kv->view, W, dm, n_vtiles, R));
-  if (mode == SJ_MODE_SAMPLING) CU_TRY(launch(k_resample, dim3(B), dim3(1024), 0, s, pdl, args, kv->view, W, dm));
+  TIMED("finalize", launch(k_finalize, dim3(B), dim3(256), 0, s, pdl, args, kv->view, W, dm, n_vtiles, R));
+  if (mode == SJ_MODE_SAMPLING) TIMED("resample", launch(k_resample, dim3(B), dim3(1024), 0, s, pdl, args, kv->view, W, dm));
+  return SJ_OK;
+}
+
+#undef TIMED
+
+extern "C" sj_status sj_kernel_time(sj_target* t, const char* name, double* total_ms, long* launches) {
+  if (!t || !name || !total_ms || !launches) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  CU_TRY(cudaStreamSynchronize(t->stream));
+  double tot = 0.0;
+  long n = 0;
+  const size_t len = strlen(name);
+  for (auto& e : t->timed) {
+    if (strncmp(e.name, name, len) != 0) continue;  // prefix match: "gemm" covers every projection
+    float ms = 0.f;
+    CU_TRY(cudaEventElapsedTime(&ms, e.a, e.b));
+    tot += ms;
+    ++n;
+  }
+  *total_ms = tot;
+  *launches = n;
   return SJ_OK;
 }
 
