@@ -180,6 +180,39 @@ sj_status sj_rollback_kv(sj_kv *kv, const int *seq_ids, const int *new_len, int 
 sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, const void *a, const void *w, float *y,
                          void *cuda_stream);
 
+/* The same product as sj_gemm_skinny(SJ_DTYPE_BF16, impl 1, ...), for callers that must not allocate.
+ * (The paper has no counterpart to this call; it exists for the library's users.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unsafe -- inside a serving
+ * engine that has handed all of the GPU's memory to its own pool, while another thread is capturing a
+ * stream (cudaMalloc and cudaFree are illegal during a capture and break it), or on a latency path
+ * where the implicit device synchronisation of cudaFree cannot be afforded.  sj_gemm_skinny() takes
+ * its split-K partial-sum buffer from cudaMalloc on every call; this variant keeps that buffer in a
+ * fixed array of SJ_NOALLOC_SCRATCH_BYTES that is part of the library image.  Every GPU on which the
+ * library's kernels are loaded holds those bytes until the process exits, used or not.
+ *
+ *   y[R, N] (fp32) = a[R, K] . w[N, K]^T,  a and w bf16, row-major, 16-byte aligned device pointers,
+ *   K a multiple of 64.  The caller owns a, w and y.  Work is queued on `cuda_stream` and the call
+ *   returns after that stream has drained (it reads back the device status word).
+ *
+ * Size limit: 256 + round_up(8 * T, 256) + 4 * slots * R * N bytes must fit in the array, with
+ * T = ceil(N/128) tiles and slots = the largest number of thread blocks that share one tile's K range:
+ * the T * (K/64) work units are dealt evenly to G = min(#SMs, T * K/64) blocks, so
+ * slots <= ceil((K/64) / floor(T * (K/64) / G)) + 1.  Larger problems are refused with SJ_ERR_SHAPE and
+ * a message naming the bytes needed; nothing is launched.
+ *
+ * The first call on each device resolves the array's device address (cudaGetSymbolAddress, with that
+ * device current) and opts the kernel into its shared-memory size; make that first call outside any
+ * stream capture.  No call allocates or frees device memory or calls a routine that does.
+ *
+ * All calls on one device share the array, and it keeps whatever the previous call left: each call
+ * zeroes the status word and rewrites the slot table and every partial sum before reading them.
+ * Two calls whose kernels overlap on the GPU (different streams, or different host threads) race on
+ * that memory and give wrong results: serialise them.
+ * Errors: INVALID_ARG (null), SHAPE (sizes, scratch limit), UNSUPPORTED (not sm_100), CUDA, TIMEOUT. */
+enum { SJ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024 };
+sj_status sj_gemm_skinny_noalloc(int R, int N, int K, const void *a, const void *w, float *y, void *cuda_stream);
+
 const char *sj_last_error(void);
 
 #ifdef __cplusplus

@@ -23,7 +23,8 @@ MODE_GREEDY, MODE_SAMPLING = 0, 1
 
 EXPORTS = ["sj_create_target", "sj_destroy_target", "sj_load_judge_head", "sj_set_option", "sj_sync",
            "sj_kv_create", "sj_kv_destroy", "sj_kv_fill", "sj_kv_read", "sj_kv_set_len", "sj_kv_set_pending",
-           "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_last_error", "sj_kernel_time"]
+           "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_gemm_skinny_noalloc", "sj_last_error",
+           "sj_kernel_time"]
 
 
 class SjError(RuntimeError):
@@ -96,6 +97,7 @@ def load(build_if_needed: bool = True) -> C.CDLL:
     lib.sj_rollback_kv.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int]
     lib.sj_gemm_skinny.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p]
+    lib.sj_gemm_skinny_noalloc.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     _lib = lib
     return lib
 
@@ -263,3 +265,17 @@ def gemm_skinny(a: torch.Tensor, w: torch.Tensor, impl: int) -> torch.Tensor:
     check(load().sj_gemm_skinny(_dtype_code(a.dtype), impl, R, N, K, _ptr(a), _ptr(w), _ptr(y),
                                 C.c_void_p(torch.cuda.current_stream().cuda_stream)))
     return y
+
+
+def gemm_skinny_noalloc(a: torch.Tensor, w: torch.Tensor, y: torch.Tensor) -> None:
+    """``sj_gemm_skinny_noalloc``: y[R, N] fp32 = a[R, K] . w[N, K]^T (bf16 inputs) into the caller's ``y``.
+
+    For callers that cannot allocate device memory (their engine owns all of it, a capture is in progress
+    on another thread, or a cudaFree-induced device sync is unaffordable): the library's partial-sum
+    scratch is a fixed array inside the library image, so this wrapper allocates nothing either.
+    """
+    R, K = a.shape
+    N = w.shape[0]
+    assert a.dtype == torch.bfloat16 and w.dtype == torch.bfloat16 and y.dtype == torch.float32 and y.shape == (R, N)
+    check(load().sj_gemm_skinny_noalloc(R, N, K, _ptr(a), _ptr(w), _ptr(y),
+                                        C.c_void_p(torch.cuda.current_stream().cuda_stream)))

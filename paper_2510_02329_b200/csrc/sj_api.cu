@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <string>
 #include <tuple>
 #include <vector>
@@ -1032,6 +1033,107 @@ extern "C" sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, co
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   cleanup();
   if (e != cudaSuccess) { cudaGetLastError(); return fail(SJ_ERR_CUDA, "sj_gemm_skinny: %s", cudaGetErrorString(e)); }
+  if (hstatus != 0) return fail(SJ_ERR_TIMEOUT, "a bounded device-side wait ran out");
+  return SJ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// skinny GEMM that allocates nothing (see sj_gemm_skinny_noalloc in sj.h)
+// ---------------------------------------------------------------------------------------------
+// Scratch shared by every call on a device.  Layout: [0, 256) device status word; [256, slots_end)
+// the per-tile slot table; from slots_end (256-byte aligned) the fp32 partial sums [slot][R][N].
+// In host code `g_noalloc_scratch` is only a handle for cudaGetSymbolAddress(); the device address is
+// looked up once per device and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[SJ_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kNoAllocMaxDevices = 64;
+static unsigned char* g_noalloc_ptr[kNoAllocMaxDevices] = {nullptr};
+static int g_noalloc_sms[kNoAllocMaxDevices] = {0};
+static std::mutex g_noalloc_mu;
+
+// Same table as build_tile_slots(), computed on the device so that no host-to-device copy is needed.
+__global__ void k_noalloc_tile_slots(int2* __restrict__ slots, int n_tiles, int KB, int G) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n_tiles) return;
+  const long long U = (long long)n_tiles * KB, t_lo = (long long)t * KB, t_hi = t_lo + KB;
+  int first = -1, cnt = 0;
+  for (int c = 0; c < G; ++c) {
+    const long long lo = (long long)c * U / G, hi = (long long)(c + 1) * U / G;
+    if (hi <= lo || lo >= t_hi || hi <= t_lo) continue;
+    if (first < 0) first = c;
+    cnt = c - first + 1;
+  }
+  slots[t] = make_int2(first, cnt);
+}
+
+extern "C" sj_status sj_gemm_skinny_noalloc(int R, int N, int K, const void* a, const void* w, float* y,
+                                            void* cuda_stream) {
+  if (!a || !w || !y) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (R <= 0 || R > SJ_MAX_ROWS || N <= 0 || K <= 0 || K % kBK) return fail(SJ_ERR_SHAPE, "bad GEMM shape (K must be a multiple of 64)");
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  int dev = 0;
+  CU_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return fail(SJ_ERR_UNSUPPORTED, "device ordinal %d not supported", dev);
+  unsigned char* scratch = nullptr;
+  int sms = 0;
+  {
+    // first call on this device (which is current): resolve the scratch array's device address
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+      int major = 0;
+      CU_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+      if (major != 10) return fail(SJ_ERR_UNSUPPORTED, "built for sm_100a");
+      CU_TRY(cudaDeviceGetAttribute(&g_noalloc_sms[dev], cudaDevAttrMultiProcessorCount, dev));
+      void* p = nullptr;
+      CU_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+      if (!p) return fail(SJ_ERR_CUDA, "cudaGetSymbolAddress returned a null scratch address");
+      CU_TRY(cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+      g_noalloc_ptr[dev] = reinterpret_cast<unsigned char*>(p);
+    }
+    scratch = g_noalloc_ptr[dev];
+    sms = g_noalloc_sms[dev];
+  }
+  // work split, as in sj_gemm_skinny()
+  TcSite site;
+  site.nseg = 1; site.K = K; site.KB = K / kBK; site.lm = false; site.N = N;
+  site.n_tiles = (N + kTileN - 1) / kTileN;
+  site.seg_tile_end[0] = site.seg_tile_end[1] = site.seg_tile_end[2] = site.n_tiles;
+  site.G = (int)std::min<long long>((long long)site.n_tiles * site.KB, sms);
+  {
+    std::vector<int2> host_slots;  // host copy, only to learn the deepest split
+    build_tile_slots(site.n_tiles, site.KB, site.G, host_slots, site.max_slots);
+  }
+  const size_t slots_end = 256 + (((size_t)site.n_tiles * sizeof(int2) + 255) & ~(size_t)255);
+  const size_t need = slots_end + (size_t)site.max_slots * R * N * sizeof(float);
+  if (need > (size_t)SJ_NOALLOC_SCRATCH_BYTES)
+    return fail(SJ_ERR_SHAPE, "sj_gemm_skinny_noalloc: R=%d N=%d K=%d needs %zu bytes of scratch, the static array holds %zu",
+                R, N, K, need, (size_t)SJ_NOALLOC_SCRATCH_BYTES);
+  int* status = reinterpret_cast<int*>(scratch);
+  site.d_tile_slots = reinterpret_cast<int2*>(scratch + 256);
+  float* P = reinterpret_cast<float*>(scratch + slots_end);
+  // the array keeps the previous call's contents: the status word must start at zero; the slot table and
+  // every partial sum that is read are rewritten below before they are read
+  CU_TRY(cudaMemsetAsync(status, 0, 256, s));
+  CU_TRY(launch(k_noalloc_tile_slots, dim3((site.n_tiles + 127) / 128), dim3(128), 0, s, false, site.d_tile_slots,
+                site.n_tiles, site.KB, site.G));
+  sj_target tmp;  // borrowed for its plumbing fields only; owns nothing
+  tmp.stream = s;
+  tmp.sm_count = sms;
+  tmp.dm.V = N;
+  memset(&tmp.work, 0, sizeof(tmp.work));
+  tmp.work.P = P;
+  tmp.work.status = status;
+  CUtensorMap mA, mW;
+  RowGeom g = row_geom(R);
+  sj_status st;
+  if ((st = make_map(&mA, a, R, K, g.nblk)) != SJ_OK) return st;
+  if ((st = make_map(&mW, w, N, K, kTileN)) != SJ_OK) return st;
+  CU_TRY(launch_tc(&tmp, site, &mA, &mW, nullptr, nullptr, R, false, false));
+  CU_TRY(launch(k_sum_slots, dim3((unsigned)(((size_t)R * N + 255) / 256)), dim3(256), 0, s, false, (const float*)P,
+                SplitPlan{site.d_tile_slots, site.n_tiles}, (size_t)R * N, R, N, y));
+  int hstatus = 0;
+  CU_TRY(cudaMemcpyAsync(&hstatus, status, sizeof(int), cudaMemcpyDeviceToHost, s));
+  CU_TRY(cudaStreamSynchronize(s));
   if (hstatus != 0) return fail(SJ_ERR_TIMEOUT, "a bounded device-side wait ran out");
   return SJ_OK;
 }
