@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "../../include/sj.h"
+#include "sj_attn_tc.cuh"
 #include "sj_gemm_tc.cuh"
 
 using namespace sj;
@@ -194,6 +195,7 @@ struct sj_target {
   size_t p_elems = 0;
   size_t att_chunks_cap = 0;
   int att_rows_cap = 0;
+  size_t tc_part_cap = 0;   // floats in tc_m / tc_l
   size_t logits_rows = 0;
   std::map<StepKey, cudaGraphExec_t> graphs;
   std::map<int, CUtensorMap> mapA_d, mapA_q, mapA_f;  // activation maps per R
@@ -211,6 +213,8 @@ struct sj_kv {
   std::vector<char> exact;              // len_hi is the exact length
   int* d_block_table = nullptr;
   int* d_tmp = nullptr;                 // [2 * SJ_MAX_BATCH] staging for rollback / set_len
+  CUtensorMap tm_pool;                  // bf16 pool as a [rows, head_dim] matrix, box = 16 slots x 64 dims
+  bool has_tm_pool = false;
 };
 
 static void clear_graphs(sj_target* t) {
@@ -318,7 +322,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   }
   const bool tc = tc_shapes_ok(c);
   t->opt_gemm = tc ? 1 : 0;
-  t->opt_attn = 0;
+  t->opt_attn = t->bf ? 1 : 0;
   t->opt_graph = t->stream ? 1 : 0;  // the legacy default stream cannot be captured
 
   sj_status st = SJ_OK;
@@ -338,6 +342,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   const size_t act_rows = t->bf ? (size_t)2 * pad16(R) : (size_t)R;  // bf16: hi and lo planes
   ALLOC(tmp, uint8_t, act_rows * c.d_model * esz); W.A = tmp;
   ALLOC(W.Q, float, (size_t)R * qd);
+  if (t->bf) ALLOC(W.Qb, bf16, (size_t)R * qd);
   ALLOC(tmp, uint8_t, act_rows * qd * esz); W.ATT = tmp;
   ALLOC(tmp, uint8_t, act_rows * c.d_ffn * esz); W.H = tmp;
   ALLOC(W.Hf, float, (size_t)R * c.d_model);
@@ -393,6 +398,13 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   t->p_elems = p_elems;
   ALLOC(W.P, float, p_elems);
 #undef ALLOC
+  if (t->bf) {
+    const int att_smem = kAttStages * kAttStageBytes + (int)sizeof(AttSmemCtl) + 1024;
+    cudaError_t e = c.head_dim == 128
+                        ? cudaFuncSetAttribute(k_attn_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, att_smem)
+                        : cudaFuncSetAttribute(k_attn_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, att_smem);
+    if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "smem opt-in: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
+  }
   {
     cudaError_t e;
     if (t->bf) e = cudaFuncSetAttribute(k_attn_simt<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024);
@@ -434,7 +446,7 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     t->opt_gemm = value;
   } else if (n == "attn_impl") {
     if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "attn_impl must be 0 or 1");
-    if (value == 1) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention is not available in this build");
+    if (value == 1 && !t->bf) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention needs a bf16 model");
     t->opt_attn = value;
   } else if (n == "graph") {
     if (value && !t->stream) return fail(SJ_ERR_UNSUPPORTED, "the legacy default stream cannot be captured into a graph");
@@ -493,6 +505,20 @@ extern "C" sj_status sj_kv_create(sj_target* t, int max_seqs, long max_pages, in
                 cudaGetErrorString(e));
   }
   cudaMemset(meta, 0, sizeof(int) * ((size_t)max_seqs * (mpps + 2) + 2 * SJ_MAX_BATCH));
+  // Slots past a sequence's length are read (and masked) by the tensor-core attention: keep them finite.
+  e = cudaMemset(pool, 0, bytes);
+  if (e == cudaSuccess && t->bf) {
+    const long long rows_total = (long long)t->dm.n_layers * max_pages * 2 * t->dm.Hkv * page_size;
+    if (rows_total < 0x7fffffffLL && make_map(&kv->tm_pool, pool, rows_total, t->dm.hd, page_size) == SJ_OK)
+      kv->has_tm_pool = true;
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(pool);
+    cudaFree(meta);
+    delete kv;
+    return fail(SJ_ERR_CUDA, "KV pool clear: %s", cudaGetErrorString(e));
+  }
   kv->d_block_table = meta;
   kv->view.pool = pool;
   kv->view.block_table = meta;
@@ -728,9 +754,11 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   const int R = B * (gamma + 1), qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd;
   const bool timing = t->opt_timing != 0 && !t->opt_graph;
   const bool pdl = t->opt_pdl != 0 && !timing, tc = t->opt_gemm == 1;
+  const bool attn_tc = t->opt_attn == 1 && t->bf && kv->has_tm_pool;
   const StepArgs* args = t->d_args;
   Work W = t->work;
   if (!use_scratch) W.logits = nullptr;
+  if (!attn_tc) W.Qb = nullptr;
   cudaStream_t s = t->stream;
   const size_t row_smem = sizeof(float) * dm.d;
   SplitPlan one{nullptr, 0};
@@ -761,8 +789,22 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
     TIMED("qkv_rope", launch(k_qkv_rope<T>, dim3(R), dim3(256), 0, s, pdl, args, kv->view, W, dm, plan_of(t->s_qkv),
                   (size_t)R * (qd + 2 * kd), l, (const T*)L.bq, (const T*)L.bk, (const T*)L.bv));
     // attention
-    TIMED("attn", launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
-    TIMED("attn_combine", launch(k_attn_combine<T>, dim3(R * dm.Hq), dim3(std::min(dm.hd, 128)), 0, s, pdl, args, W, dm));
+    if (attn_tc) {
+      AttArgs aa{W.Qb, AttPartials{W.tc_m, W.tc_l, W.tc_o}, t->sm_count + B * dm.Hkv, l};
+      const size_t tc_smem = kAttStages * kAttStageBytes + sizeof(AttSmemCtl) + 1024;
+      const AttPartials parts{W.tc_m, W.tc_l, W.tc_o};
+      const int items = B * dm.Hkv * nq, cgrid = std::max(1, std::min(4 * t->sm_count, (items + 7) / 8));
+      if (dm.hd == 128) {
+        TIMED("attn", launch(k_attn_tc<128>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base));
+      } else {
+        TIMED("attn", launch(k_attn_tc<64>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
+        TIMED("attn_combine", launch(k_attn_combine_tc<64>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base));
+      }
+    } else {
+      TIMED("attn", launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
+      TIMED("attn_combine", launch(k_attn_combine<T>, dim3(R * dm.Hq), dim3(std::min(dm.hd, 128)), 0, s, pdl, args, W, dm));
+    }
     // O projection + residual + FFN norm
     if (tc) {
       TIMED("gemm_o", launch_tc(t, t->s_o, mA_q, &L.m_o, nullptr, nullptr, R, pdl, true));
@@ -902,6 +944,26 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
     if ((st = dev_alloc(t, &t->work.att_o, n_ml * t->dm.hd)) != SJ_OK) return st;
     t->att_chunks_cap = cap;
     t->att_rows_cap = rcap;
+  }
+  if (t->opt_attn == 1 && t->bf && kv->has_tm_pool) {
+    const size_t slots = (size_t)t->sm_count + 2 * (size_t)B * t->dm.Hkv;
+    const size_t need = slots * kAttMaxSub * (size_t)(group * rows);
+    if (need > t->tc_part_cap) {
+      CU_TRY(cudaStreamSynchronize(t->stream));
+      clear_graphs(t);
+      for (float** p : {&t->work.tc_m, &t->work.tc_l, &t->work.tc_o}) {
+        if (*p) {
+          cudaFree(*p);
+          t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)*p), t->owned.end());
+          *p = nullptr;
+        }
+      }
+      t->tc_part_cap = 0;
+      if ((st = dev_alloc(t, &t->work.tc_m, need)) != SJ_OK) return st;
+      if ((st = dev_alloc(t, &t->work.tc_l, need)) != SJ_OK) return st;
+      if ((st = dev_alloc(t, &t->work.tc_o, need * t->dm.hd)) != SJ_OK) return st;
+      t->tc_part_cap = need;
+    }
   }
   if (use_scratch && (size_t)R > t->logits_rows) {
     CU_TRY(cudaStreamSynchronize(t->stream));

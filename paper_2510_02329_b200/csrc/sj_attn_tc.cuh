@@ -1,0 +1,577 @@
+// Tensor-core attention of the verification step (bf16 models): causal grouped-query attention of the
+// gamma+1 block rows of every sequence over the paged cache, split along the keys over all SMs.
+//
+// Work decomposition.  The cached keys [0, L_b) of sequence b are cut into ring tiles of KPS keys
+// (one tile = 16 KiB: KPS keys of K and of V of one KV head; KPS = 32 for head_dim 128, 64 for head_dim
+// 64).  Tiles are ordered (sequence, KV head, tile) and block c owns tiles [c*T/G, (c+1)*T/G); every
+// maximal run of tiles of one (sequence, KV head) inside a block's range is a segment.  The block's own
+// gamma+1 new rows (positions L_b ..) are a separate "tail" segment per (sequence, KV head), read from
+// the pages with plain loads.  A segment's result is an unnormalised partial (running max m in the
+// log2 domain, sum l, output o) per query row; a combine pass merges the partials of a (sequence, KV
+// head) in a fixed order (deterministic).
+//
+// Per segment the query rows of the KV head's group (q = g*(gamma+1) + j, g = head inside the group)
+// form the M dimension of mma.sync.m16n8k16 tiles: warp (mi, ks) of a block owns m-tile mi (16 query
+// rows) and the ks-th share of the keys of every ring tile, with its own online-softmax state, so
+// warps never exchange data; each writes its own sub-partial.
+//
+// Ring tiles arrive by TMA (tensor map over the page pool, box = 16 slots x 64 dims, 128-byte swizzle)
+// into shared memory; K fragments are read with ldmatrix, V fragments with ldmatrix.trans.
+#pragma once
+
+#include <cuda.h>
+
+#include <type_traits>
+
+#include "sj_kernels.cuh"
+
+namespace sj {
+
+constexpr int kAttStageBytes = 16384;     // one ring tile: K part then V part, 8 KiB each
+constexpr int kAttMaxWarps = 8;           // consumer warps per block
+constexpr int kAttMaxSub = 4;             // sub-partials per segment (key shares)
+constexpr uint32_t kAttSpin = 1u << 22;
+
+__device__ __forceinline__ uint32_t att_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+               : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+__device__ __forceinline__ uint32_t ldcg_u32(const void* p) { return __ldcg(reinterpret_cast<const unsigned int*>(p)); }
+__device__ __forceinline__ uint32_t ldcg_u16(const void* p) { return (uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p)); }
+
+// Geometry shared by the attention pass, the combine pass and the host.
+struct AttGeom {
+  int HD, KPS, MT, KS, KW, nq, rows, group;
+};
+__host__ __device__ __forceinline__ AttGeom att_geom(int hd, int group, int rows) {
+  AttGeom g;
+  g.HD = hd;
+  g.KPS = kAttStageBytes / (4 * hd);          // keys per ring tile
+  g.rows = rows;
+  g.group = group;
+  g.nq = group * rows;
+  g.MT = (g.nq + 15) / 16;
+  int ks = g.KPS / 16, cap = kAttMaxWarps / g.MT;
+  if (ks > cap) ks = cap;
+  if (ks > kAttMaxSub) ks = kAttMaxSub;
+  if (ks < 1) ks = 1;
+  g.KS = ks == 3 ? 2 : ks;                    // power of two
+  g.KW = g.KPS / g.KS;                        // keys per warp per tile
+  return g;
+}
+
+// Which block owns ring tile t when T tiles are dealt to G blocks as [c*T/G, (c+1)*T/G).
+__device__ __forceinline__ int att_owner(long long t, long long T, int G) {
+  int c = (int)(t * G / T);
+  while ((long long)(c + 1) * T / G <= t) ++c;
+  return c;
+}
+
+// Partial storage: slot s, sub-partial ks, query row q.
+struct AttPartials {
+  float* m;   // [slots][kAttMaxSub][nq]
+  float* l;
+  float* o;   // [slots][kAttMaxSub][nq][hd]
+};
+
+// One warp's share of one segment.
+template <int HD, int NT>
+struct AttWarp {
+  uint32_t qa[HD / 16][4];
+  float o[HD / 8][4];
+  float m0, m1, l0, l1;
+
+  __device__ __forceinline__ void reset() {
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    m0 = m1 = -INFINITY;
+    l0 = l1 = 0.f;
+  }
+
+  // A fragments of this warp's 16 query rows.  Qb: [nq][HD] bf16 of one (sequence, KV head), already
+  // scaled by log2(e)/sqrt(HD).  Rows >= nq read as zero.
+  __device__ __forceinline__ void load_q(const bf16* __restrict__ Qb, int row0, int nq, int lane) {
+    const int r0 = row0 + (lane >> 2), r1 = r0 + 8, c = (lane & 3) * 2;
+#pragma unroll
+    for (int k = 0; k < HD / 16; ++k) {
+      qa[k][0] = r0 < nq ? ldcg_u32(Qb + (size_t)r0 * HD + k * 16 + c) : 0u;
+      qa[k][1] = r1 < nq ? ldcg_u32(Qb + (size_t)r1 * HD + k * 16 + c) : 0u;
+      qa[k][2] = r0 < nq ? ldcg_u32(Qb + (size_t)r0 * HD + k * 16 + c + 8) : 0u;
+      qa[k][3] = r1 < nq ? ldcg_u32(Qb + (size_t)r1 * HD + k * 16 + c + 8) : 0u;
+    }
+  }
+
+  // Online-softmax update from the score fragments s (log2 domain; masked entries are -inf), returning
+  // the probabilities in s.
+  __device__ __forceinline__ void softmax_update(float (*s)[4]) {
+    float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
+      mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float n0 = fmaxf(m0, mx0), n1 = fmaxf(m1, mx1);
+    const float a0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - n0);
+    const float a1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - n1);
+    m0 = n0;
+    m1 = n1;
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      s[n][0] = (s[n][0] == -INFINITY) ? 0.f : exp2f(s[n][0] - n0);
+      s[n][1] = (s[n][1] == -INFINITY) ? 0.f : exp2f(s[n][1] - n0);
+      s[n][2] = (s[n][2] == -INFINITY) ? 0.f : exp2f(s[n][2] - n1);
+      s[n][3] = (s[n][3] == -INFINITY) ? 0.f : exp2f(s[n][3] - n1);
+      s0 += s[n][0] + s[n][1];
+      s1 += s[n][2] + s[n][3];
+    }
+    l0 = l0 * a0 + s0;
+    l1 = l1 * a1 + s1;
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i) {
+      o[i][0] *= a0; o[i][1] *= a0;
+      o[i][2] *= a1; o[i][3] *= a1;
+    }
+  }
+
+  // One ring tile in shared memory.  `stage`: shared address of the tile (1024-byte aligned): K boxes
+  // [page][half] of 2 KiB (16 slots x 64 dims, 128-byte swizzle) then, 8 KiB in, the V boxes.
+  // kw0: first key of this warp's share inside the tile; key_abs0: absolute index of that key; L: keys
+  // >= L are masked.
+  __device__ __forceinline__ void tile(uint32_t stage, int kw0, int key_abs0, int L, int lane) {
+    constexpr int HB = HD / 64;
+    float s[NT][4];
+#pragma unroll
+    for (int n = 0; n < NT; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+    const int lr = lane & 7, mid = lane >> 3;
+#pragma unroll
+    for (int kp = 0; kp < HD / 32; ++kp) {
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        const int kk = kw0 + n * 8 + lr, page = kk >> 4, r = kk & 15;
+        const int d = kp * 32 + mid * 8, half = d >> 6, c = (d & 63) >> 3;
+        const uint32_t addr = stage + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4(addr, b0, b1, b2, b3);
+        mma_16816(s[n], qa[2 * kp], b0, b1);
+        mma_16816(s[n], qa[2 * kp + 1], b2, b3);
+      }
+    }
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+      const int k = key_abs0 + n * 8 + (lane & 3) * 2;
+      if (k >= L) { s[n][0] = -INFINITY; s[n][2] = -INFINITY; }
+      if (k + 1 >= L) { s[n][1] = -INFINITY; s[n][3] = -INFINITY; }
+    }
+    softmax_update(s);
+#pragma unroll
+    for (int kk2 = 0; kk2 < NT / 2; ++kk2) {
+      uint32_t pa[4];
+      pa[0] = pack_bf16(s[2 * kk2][0], s[2 * kk2][1]);
+      pa[1] = pack_bf16(s[2 * kk2][2], s[2 * kk2][3]);
+      pa[2] = pack_bf16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
+      pa[3] = pack_bf16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
+#pragma unroll
+      for (int dp = 0; dp < HD / 16; ++dp) {
+        const int kk = kw0 + kk2 * 16 + (mid & 1) * 8 + lr, page = kk >> 4, r = kk & 15;
+        const int d = (dp * 2 + (mid >> 1)) * 8, half = d >> 6, c = (d & 63) >> 3;
+        const uint32_t addr =
+            stage + 8192u + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
+        uint32_t v0, v1, v2, v3;
+        ldsm_x4_t(addr, v0, v1, v2, v3);
+        mma_16816(o[2 * dp], pa, v0, v1);
+        mma_16816(o[2 * dp + 1], pa, v2, v3);
+      }
+    }
+  }
+
+  // The block's own rows: keys kq = 0..rows-1 at positions L + kq, read from the pages with plain
+  // loads (they were written earlier in this step).  Query row q = g*rows + j sees kq <= j.
+  // krow(kq) / vrow(kq) return the bf16 row pointers [HD].
+  template <typename KFn, typename VFn>
+  __device__ __forceinline__ void tail(KFn krow, VFn vrow, int rows, int row0, int nq, int lane) {
+    const int q0 = row0 + (lane >> 2), q1 = q0 + 8;
+    const int j0 = q0 % rows, j1 = q1 % rows;
+    for (int kbase = 0; kbase < rows; kbase += NT * 8) {
+      float s[NT][4];
+#pragma unroll
+      for (int n = 0; n < NT; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        const int key = kbase + n * 8 + (lane >> 2);
+        if (kbase + n * 8 < rows) {   // warp-uniform
+          const bf16* kr = key < rows ? krow(key) : nullptr;
+#pragma unroll
+          for (int k = 0; k < HD / 16; ++k) {
+            uint32_t b0 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2) : 0u;
+            uint32_t b1 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2 + 8) : 0u;
+            mma_16816(s[n], qa[k], b0, b1);
+          }
+        }
+      }
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        const int k = kbase + n * 8 + (lane & 3) * 2;
+        if (k > j0 || k >= rows || q0 >= nq) s[n][0] = -INFINITY;
+        if (k + 1 > j0 || k + 1 >= rows || q0 >= nq) s[n][1] = -INFINITY;
+        if (k > j1 || k >= rows || q1 >= nq) s[n][2] = -INFINITY;
+        if (k + 1 > j1 || k + 1 >= rows || q1 >= nq) s[n][3] = -INFINITY;
+      }
+      softmax_update(s);
+#pragma unroll
+      for (int kk2 = 0; kk2 < NT / 2; ++kk2) {
+        if (kbase + kk2 * 16 >= rows) continue;   // warp-uniform
+        uint32_t pa[4];
+        pa[0] = pack_bf16(s[2 * kk2][0], s[2 * kk2][1]);
+        pa[1] = pack_bf16(s[2 * kk2][2], s[2 * kk2][3]);
+        pa[2] = pack_bf16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
+        pa[3] = pack_bf16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
+        const int ka = kbase + kk2 * 16 + (lane & 3) * 2;   // keys ka, ka+1 (b0) and ka+8, ka+9 (b1)
+        const bf16* v00 = ka < rows ? vrow(ka) : nullptr;
+        const bf16* v01 = ka + 1 < rows ? vrow(ka + 1) : nullptr;
+        const bf16* v10 = ka + 8 < rows ? vrow(ka + 8) : nullptr;
+        const bf16* v11 = ka + 9 < rows ? vrow(ka + 9) : nullptr;
+#pragma unroll
+        for (int dn = 0; dn < HD / 8; ++dn) {
+          const int d = dn * 8 + (lane >> 2);
+          uint32_t b0 = (v00 ? ldcg_u16(v00 + d) : 0u) | ((v01 ? ldcg_u16(v01 + d) : 0u) << 16);
+          uint32_t b1 = (v10 ? ldcg_u16(v10 + d) : 0u) | ((v11 ? ldcg_u16(v11 + d) : 0u) << 16);
+          mma_16816(o[dn], pa, b0, b1);
+        }
+      }
+    }
+  }
+
+  // Write this warp's sub-partial.
+  __device__ __forceinline__ void store(const AttPartials& P, size_t slot, int sub, int row0, int nq, int lane) {
+    float s0 = l0, s1 = l1;
+    s0 += __shfl_xor_sync(0xffffffffu, s0, 1);
+    s0 += __shfl_xor_sync(0xffffffffu, s0, 2);
+    s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
+    s1 += __shfl_xor_sync(0xffffffffu, s1, 2);
+    const int q0 = row0 + (lane >> 2), q1 = q0 + 8;
+    const size_t base = (slot * kAttMaxSub + sub) * (size_t)nq;
+    if ((lane & 3) == 0) {
+      if (q0 < nq) { P.m[base + q0] = m0; P.l[base + q0] = s0; }
+      if (q1 < nq) { P.m[base + q1] = m1; P.l[base + q1] = s1; }
+    }
+#pragma unroll
+    for (int dn = 0; dn < HD / 8; ++dn) {
+      const int d = dn * 8 + (lane & 3) * 2;
+      if (q0 < nq) *reinterpret_cast<float2*>(P.o + (base + q0) * HD + d) = make_float2(o[dn][0], o[dn][1]);
+      if (q1 < nq) *reinterpret_cast<float2*>(P.o + (base + q1) * HD + d) = make_float2(o[dn][2], o[dn][3]);
+    }
+  }
+};
+
+// Ring-tile bookkeeping of one block: sequence lengths, tile prefix, the block's tile range.
+struct AttPlan {
+  int L[kMaxBatch];          // cached keys per sequence
+  int pre[kMaxBatch + 1];    // ring tiles before sequence b (all KV heads)
+  long long T;               // total ring tiles
+};
+
+// Filled by one thread; callers synchronise afterwards.
+__device__ __forceinline__ void att_plan_fill(AttPlan* pl, const int* __restrict__ row_pos, int B, int rows, int Hkv,
+                                              int KPS) {
+  int acc = 0;
+  for (int b = 0; b < B; ++b) {
+    const int L = row_pos[b * rows];
+    pl->L[b] = L;
+    pl->pre[b] = acc;
+    acc += Hkv * ((L + KPS - 1) / KPS);
+  }
+  pl->pre[B] = acc;
+  pl->T = acc;
+}
+
+__device__ __forceinline__ int att_find_seq(const int* pre, int B, int t) {
+  int lo = 0, hi = B - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (pre[mid] <= t) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+struct AttArgs {
+  const bf16* Qb;          // [B][Hkv][nq][HD] scaled queries
+  AttPartials P;
+  int n_tail_base;         // slot of tail (b, h): n_tail_base + b*Hkv + h
+  int layer;
+};
+
+// ---------------------------------------------------------------------------------------------
+// stand-alone kernel (used by the multi-kernel step): warp 0 streams the ring, warps 1..8 consume
+// ---------------------------------------------------------------------------------------------
+struct AttSmemCtl {
+  uint64_t full[8];
+  uint64_t empty[8];
+  int cons_cnt[8];
+  int abort_flag;
+  AttPlan plan;
+};
+constexpr int kAttStages = 8;
+constexpr int kAttTcThreads = 32 * (1 + kAttMaxWarps);
+
+__device__ __forceinline__ void att_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void att_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void att_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool att_mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  for (uint32_t i = 0; i < kAttSpin; ++i) {
+    if (att_mbar_try(bar, parity)) return true;
+    if (i > 64) {
+      if (*abort_flag) return false;
+      __nanosleep(i > 4096 ? 128 : 20);
+    }
+  }
+  *abort_flag = 1;
+  atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+  return false;
+}
+__device__ __forceinline__ void att_tma_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// Issue the TMA loads of ring tile (sequence b, KV head h, tile index ti) into `stage`.
+__device__ __forceinline__ void att_issue_tile(const CUtensorMap* tmKV, const KvView& kv, int layer, int seq, int h, int ti,
+                                               int L, int KPS, int HD, uint32_t stage, uint32_t bar) {
+  const int HB = HD / 64, npg = KPS / 16;
+  const int last_page = (L - 1) / 16;   // L >= 1 for any ring tile
+  att_mbar_expect_tx(bar, kAttStageBytes);
+  for (int p = 0; p < npg; ++p) {
+    int pi = ti * npg + p;
+    if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
+    const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+    const long long rowK = ((((long long)layer * kv.n_pages + page) * 2 + 0) * kv.n_kv_heads + h) * 16;
+    const long long rowV = rowK + (long long)kv.n_kv_heads * 16;
+    for (int half = 0; half < HB; ++half) {
+      att_tma_2d(stage + (uint32_t)((p * HB + half) * 2048), tmKV, bar, half * 64, (int)rowK);
+      att_tma_2d(stage + 8192u + (uint32_t)((p * HB + half) * 2048), tmKV, bar, half * 64, (int)rowV);
+    }
+  }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kAttTcThreads, 1)
+k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__ args, KvView kv, Work w, Dims dm,
+          AttArgs a) {
+  extern __shared__ uint8_t att_smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(att_smem_raw) + 1023) & ~(uintptr_t)1023);
+  AttSmemCtl* ctl = reinterpret_cast<AttSmemCtl*>(ring + kAttStages * kAttStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_wait();
+  pdl_launch();
+  const int B = args->B, rows = args->gamma + 1, Hkv = dm.Hkv;
+  const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+  const int n_active = g.MT * g.KS;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kAttStages; ++i) {
+      att_mbar_init(att_smem_u32(&ctl->full[i]), 1);
+      att_mbar_init(att_smem_u32(&ctl->empty[i]), 1);
+      ctl->cons_cnt[i] = 0;
+    }
+    ctl->abort_flag = 0;
+    att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, g.KPS);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const AttPlan& pl = ctl->plan;
+  const long long T = pl.T;
+  const int G = gridDim.x, c = blockIdx.x;
+  const long long t_lo = (long long)c * T / G, t_hi = (long long)(c + 1) * T / G;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int it = 0;
+      for (long long t = t_lo; t < t_hi; ++t, ++it) {
+        const int s = it % kAttStages, round = it / kAttStages;
+        if (round > 0 && !att_mbar_wait(att_smem_u32(&ctl->empty[s]), (round - 1) & 1, abort_flag, w.status)) break;
+        const int b = att_find_seq(pl.pre, B, (int)t);
+        const int nt_b = (pl.L[b] + g.KPS - 1) / g.KPS;
+        const int rem = (int)t - pl.pre[b], h = rem / nt_b, ti = rem % nt_b;
+        att_issue_tile(&tmKV, kv, a.layer, args->seq_ids[b], h, ti, pl.L[b], g.KPS, HD,
+                       att_smem_u32(ring + (size_t)s * kAttStageBytes), att_smem_u32(&ctl->full[s]));
+      }
+    }
+  } else {
+    const int cw = warp - 1;
+    if (cw < n_active) {
+      const int mi = cw / g.KS, ks = cw % g.KS, row0 = mi * 16;
+      auto run = [&](auto tag) {
+        constexpr int NT = decltype(tag)::value;
+        AttWarp<HD, NT> st;
+        // ring segments
+        int it = 0;
+        long long t = t_lo;
+        bool alive = true;
+        while (t < t_hi && alive) {
+          const int b = att_find_seq(pl.pre, B, (int)t);
+          const int L = pl.L[b];
+          const int nt_b = (L + g.KPS - 1) / g.KPS;
+          const int rem = (int)t - pl.pre[b], h = rem / nt_b, ti0 = rem % nt_b;
+          const int n = (int)min((long long)(nt_b - ti0), t_hi - t);
+          st.reset();
+          st.load_q(a.Qb + ((size_t)b * Hkv + h) * g.nq * HD, row0, g.nq, lane);
+          for (int i = 0; i < n; ++i, ++it) {
+            const int s = it % kAttStages;
+            const uint32_t bar = att_smem_u32(&ctl->full[s]);
+            int ok = 1;
+            if (lane == 0) ok = att_mbar_wait(bar, (it / kAttStages) & 1, abort_flag, w.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { alive = false; break; }
+            att_mbar_try(bar, (it / kAttStages) & 1);   // every lane observes the completed phase
+            __syncwarp();
+            st.tile(att_smem_u32(ring + (size_t)s * kAttStageBytes), ks * g.KW, (ti0 + i) * g.KPS + ks * g.KW, L, lane);
+            __syncwarp();
+            if (lane == 0) {
+              __threadfence_block();
+              if (atomicAdd(&ctl->cons_cnt[s], 1) == n_active - 1) {
+                ctl->cons_cnt[s] = 0;
+                __threadfence_block();
+                att_mbar_arrive(att_smem_u32(&ctl->empty[s]));
+              }
+            }
+          }
+          if (!alive) break;
+          st.store(a.P, (size_t)c + (size_t)b * Hkv + h, ks, row0, g.nq, lane);
+          t += n;
+        }
+        // tail segments: (b, h) number x goes to block G-1-(x mod G), key share 0 only
+        if (alive && ks == 0) {
+          for (int x = G - 1 - c; x < B * Hkv; x += G) {
+            const int b = x / Hkv, h = x % Hkv;
+            const int L = pl.L[b], seq = args->seq_ids[b];
+            st.reset();
+            st.load_q(a.Qb + ((size_t)b * Hkv + h) * g.nq * HD, row0, g.nq, lane);
+            auto krow = [&](int kq) -> const bf16* {
+              const int pos = L + kq;
+              const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
+              return kv_row<bf16>(kv, a.layer, page, 0, h, pos % 16);
+            };
+            auto vrow = [&](int kq) -> const bf16* {
+              const int pos = L + kq;
+              const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
+              return kv_row<bf16>(kv, a.layer, page, 1, h, pos % 16);
+            };
+            st.tail(krow, vrow, rows, row0, g.nq, lane);
+            st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
+          }
+        }
+      };
+      if (g.KW == 16) run(std::integral_constant<int, 2>());
+      else if (g.KW == 32) run(std::integral_constant<int, 4>());
+      else if constexpr (HD == 64) run(std::integral_constant<int, 8>());
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) __nanosleep(20000);   // let copies in flight land before the block retires
+}
+
+// Merge the partials of one (sequence, KV head, query row): ring segments in block order, their
+// sub-partials in key-share order, then the tail.  One warp per item; writes the O-projection input.
+// G_att: grid of the attention pass.
+template <typename T, int HD>
+__device__ __forceinline__ void att_combine_item(const AttPartials& P, const AttPlan& pl, const AttGeom& g, int G_att,
+                                                 int n_tail_base, int Hkv, int item, int B, void* ATT, int R, int Hq,
+                                                 int lane) {
+  const int q = item % g.nq, bh = item / g.nq, b = bh / Hkv, h = bh % Hkv;
+  const int L = pl.L[b];
+  const int nt_b = (L + g.KPS - 1) / g.KPS;
+  int c_first = 0, c_last = -1;
+  if (nt_b > 0) {
+    const long long t0 = (long long)pl.pre[b] + (long long)h * nt_b;
+    c_first = att_owner(t0, pl.T, G_att);
+    c_last = att_owner(t0 + nt_b - 1, pl.T, G_att);
+  }
+  constexpr int DPL = HD / 32;   // dims per lane
+  float M = -INFINITY;
+  auto has_tiles = [&](int c) { return (long long)(c + 1) * pl.T / G_att > (long long)c * pl.T / G_att; };
+  for (int c = c_first; c <= c_last; ++c)
+    if (has_tiles(c))
+      for (int ks = 0; ks < g.KS; ++ks) M = fmaxf(M, __ldcg(P.m + (((size_t)c + bh) * kAttMaxSub + ks) * g.nq + q));
+  const size_t tail_idx = ((size_t)(n_tail_base + bh) * kAttMaxSub) * g.nq + q;
+  M = fmaxf(M, __ldcg(P.m + tail_idx));
+  float lsum = 0.f, acc[DPL];
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+  auto add = [&](size_t idx) {
+    const float m = __ldcg(P.m + idx);
+    if (m == -INFINITY) return;
+    const float wgt = exp2f(m - M);
+    lsum += __ldcg(P.l + idx) * wgt;
+    const float* op = P.o + idx * HD + lane * DPL;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] += __ldcg(op + i) * wgt;
+  };
+  for (int c = c_first; c <= c_last; ++c)
+    if (has_tiles(c))
+      for (int ks = 0; ks < g.KS; ++ks) add((((size_t)c + bh) * kAttMaxSub + ks) * g.nq + q);
+  add(tail_idx);
+  const int gq = q / g.rows, j = q % g.rows, r = b * g.rows + j, head = h * g.group + gq;
+  const float inv = 1.0f / lsum;
+#pragma unroll
+  for (int i = 0; i < DPL; ++i) store_act<T>(ATT, R, Hq * HD, r, head * HD + lane * DPL + i, acc[i] * inv);
+}
+
+template <int HD>
+__global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dims dm, AttPartials P, int G_att,
+                                  int n_tail_base) {
+  __shared__ AttPlan pl;
+  pdl_wait();
+  pdl_launch();
+  const int B = args->B, rows = args->gamma + 1;
+  const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+  if (threadIdx.x == 0) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS);
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
+  const int items = B * dm.Hkv * g.nq;
+  for (int item = blockIdx.x * wpb + warp; item < items; item += gridDim.x * wpb)
+    att_combine_item<bf16, HD>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, B, w.ATT, B * rows, dm.Hq, lane);
+}
+
+}  // namespace sj

@@ -15,6 +15,8 @@ struct Work {
   // in the fp32 accumulator's epilogue.
   void* A;           // normalised activations (input of QKV / gate-up / LM head), K = d
   float* Q;          // [R, Hq*hd]    fp32 rotated queries
+  bf16* Qb;          // [B, Hkv, group*(gamma+1), hd] bf16 rotated queries times log2(e)/sqrt(hd), query row
+                     // g*(gamma+1)+j of a KV head's group (tensor-core attention), or null
   void* ATT;         // attention output (input of the O projection), K = Hq*hd
   void* H;           // silu(gate)*up (input of the down projection), K = F
   float* P;          // partial sums of the current GEMM: [slot][R][N]
@@ -25,6 +27,9 @@ struct Work {
   float* att_m;      // [chunks, Hq, gamma+1]         running max of each partial
   float* att_l;      // same                           sum of exp
   float* att_o;      // [chunks, Hq, gamma+1, hd]      unnormalised partial outputs
+  float* tc_m;       // tensor-core attention partials: [slots][4][nq] running max (log2 domain)
+  float* tc_l;       // same                            sum of exp2
+  float* tc_o;       // [slots][4][nq][hd]              unnormalised outputs
   RowStat* stats;    // [vocab tiles, R]
   float* tgt_logit;  // [R]   logit of the drafted token d_{j+1} in row j
   RowStat* rowstat;  // [R]   merged statistics
@@ -177,6 +182,13 @@ __global__ void k_qkv_rope(const StepArgs* __restrict__ args, KvView kv, Work w,
       float* q = w.Q + (size_t)r * qd;
       q[n1] = y1;
       q[n2] = y2;
+      if (w.Qb) {
+        const int group = dm.Hq / dm.Hkv, j = r % rows;
+        const float qs = 1.4426950408889634f / sqrtf((float)dm.hd);
+        bf16* qb = w.Qb + ((((size_t)b * dm.Hkv + head / group) * group + head % group) * rows + j) * dm.hd;
+        qb[i] = __float2bfloat16_rn(y1 * qs);
+        qb[i + half] = __float2bfloat16_rn(y2 * qs);
+      }
     } else {
       T* krow = kv_row<T>(kv, layer, page, 0, head - dm.Hq, slot);
       krow[i] = from_f<T>(y1);
