@@ -962,6 +962,10 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
       if ((st = dev_alloc(t, &t->work.tc_m, need)) != SJ_OK) return st;
       if ((st = dev_alloc(t, &t->work.tc_l, need)) != SJ_OK) return st;
       if ((st = dev_alloc(t, &t->work.tc_o, need * t->dm.hd)) != SJ_OK) return st;
+      // slots of blocks that own no tile are read with weight zero: they must hold finite values
+      CU_TRY(cudaMemsetAsync(t->work.tc_m, 0, need * sizeof(float), t->stream));
+      CU_TRY(cudaMemsetAsync(t->work.tc_l, 0, need * sizeof(float), t->stream));
+      CU_TRY(cudaMemsetAsync(t->work.tc_o, 0, need * t->dm.hd * sizeof(float), t->stream));
       t->tc_part_cap = need;
     }
   }

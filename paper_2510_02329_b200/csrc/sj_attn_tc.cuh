@@ -324,18 +324,8 @@ struct AttArgs {
 };
 
 // ---------------------------------------------------------------------------------------------
-// stand-alone kernel (used by the multi-kernel step): warp 0 streams the ring, warps 1..8 consume
+// ring plumbing shared by the stand-alone kernel and the whole-step kernel
 // ---------------------------------------------------------------------------------------------
-struct AttSmemCtl {
-  uint64_t full[8];
-  uint64_t empty[8];
-  int cons_cnt[8];
-  int abort_flag;
-  AttPlan plan;
-};
-constexpr int kAttStages = 8;
-constexpr int kAttTcThreads = 32 * (1 + kAttMaxWarps);
-
 __device__ __forceinline__ void att_mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
@@ -356,15 +346,27 @@ __device__ __forceinline__ bool att_mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+// On a timeout with abort_g set, abort_g[1] records (where | block << 8) and abort_g[2] `extra`, for the
+// host's error message.
+__device__ __forceinline__ void att_note_timeout(volatile int* abort_g, int where, int extra) {
+  if (!abort_g) return;
+  if (atomicCAS(const_cast<int*>(abort_g) + 1, 0, where | ((int)blockIdx.x << 8)) == 0) abort_g[2] = extra;
+}
+// Bounded wait.  abort_flag: the block's flag (shared memory); abort_g: optional device-wide flag that
+// other blocks raise; status: device status word.
+__device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                              volatile int* abort_g = nullptr, int where = 0, int extra = 0) {
   for (uint32_t i = 0; i < kAttSpin; ++i) {
     if (att_mbar_try(bar, parity)) return true;
     if (i > 64) {
       if (*abort_flag) return false;
+      if (abort_g && (i & 255) == 0 && *abort_g) { *abort_flag = 1; return false; }
       __nanosleep(i > 4096 ? 128 : 20);
     }
   }
   *abort_flag = 1;
+  att_note_timeout(abort_g, where, extra);
+  if (abort_g) *abort_g = 1;
   atomicCAS(status, DEV_OK, DEV_TIMEOUT);
   return false;
 }
@@ -376,12 +378,12 @@ __device__ __forceinline__ void att_tma_2d(uint32_t dst, const CUtensorMap* tm, 
       : "memory");
 }
 
-// Issue the TMA loads of ring tile (sequence b, KV head h, tile index ti) into `stage`.
+// Issue the TMA loads of ring tile (sequence slot seq, KV head h, tile index ti) into `stage`; the
+// caller has already announced kAttStageBytes on `bar`.
 __device__ __forceinline__ void att_issue_tile(const CUtensorMap* tmKV, const KvView& kv, int layer, int seq, int h, int ti,
                                                int L, int KPS, int HD, uint32_t stage, uint32_t bar) {
   const int HB = HD / 64, npg = KPS / 16;
   const int last_page = (L - 1) / 16;   // L >= 1 for any ring tile
-  att_mbar_expect_tx(bar, kAttStageBytes);
   for (int p = 0; p < npg; ++p) {
     int pi = ti * npg + p;
     if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
@@ -395,6 +397,119 @@ __device__ __forceinline__ void att_issue_tile(const CUtensorMap* tmKV, const Kv
   }
 }
 
+// Map ring tile t to (sequence, KV head, tile index, tiles of that (sequence, head)).
+struct AttTile { int b, h, ti, nt_b, L; };
+__device__ __forceinline__ AttTile att_locate(const AttPlan& pl, int B, int KPS, int t) {
+  AttTile x;
+  x.b = att_find_seq(pl.pre, B, t);
+  x.L = pl.L[x.b];
+  x.nt_b = (x.L + KPS - 1) / KPS;
+  const int rem = t - pl.pre[x.b];
+  x.h = rem / x.nt_b;
+  x.ti = rem % x.nt_b;
+  return x;
+}
+
+// The consumer side of a ring shared with other traffic.
+struct AttRing {
+  uint64_t* full;        // [stages] shared memory barriers
+  uint64_t* empty;
+  int* cons_cnt;         // [stages] how many consumer warps are done with the stage
+  uint8_t* base;         // first stage
+  int stage_stride;      // bytes between stages
+  int stages;
+  volatile int* abort_flag;
+  volatile int* abort_g;
+  int* status;
+};
+
+// One consumer warp (cw of n_active = MT*KS) of block c of G: all ring segments of the block's tile
+// range [t_lo, t_hi) starting at ring position `it`, then the block's tail segments.
+template <int HD, int NT>
+__device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const AttPlan& pl, const AttGeom& g,
+                                            const StepArgs* __restrict__ args, const KvView& kv, const AttArgs& a, int Hkv,
+                                            int c, int G, int cw, int lane) {
+  const int B = args->B, rows = g.rows, n_active = g.MT * g.KS;
+  const int mi = cw / g.KS, ks = cw % g.KS, row0 = mi * 16;
+  const long long T = pl.T;
+  const long long t_lo = (long long)c * T / G, t_hi = (long long)(c + 1) * T / G;
+  AttWarp<HD, NT> st;
+  long long t = t_lo;
+  while (t < t_hi) {
+    const AttTile x = att_locate(pl, B, g.KPS, (int)t);
+    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    st.reset();
+    st.load_q(a.Qb + ((size_t)x.b * Hkv + x.h) * g.nq * HD, row0, g.nq, lane);
+    for (int i = 0; i < n; ++i, ++it) {
+      const int s = it % rg.stages;
+      const uint32_t bar = att_smem_u32(&rg.full[s]), par = (uint32_t)(it / rg.stages) & 1u;
+      int ok = 1;
+      if (lane == 0) ok = att_mbar_wait(bar, par, rg.abort_flag, rg.status, rg.abort_g, 9, it) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) return false;
+      att_mbar_try(bar, par);   // every lane observes the completed phase
+      __syncwarp();
+      st.tile(att_smem_u32(rg.base + (size_t)s * rg.stage_stride), ks * g.KW, (x.ti + i) * g.KPS + ks * g.KW, x.L, lane);
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence_block();
+        if (atomicAdd(&rg.cons_cnt[s], 1) == n_active - 1) {
+          rg.cons_cnt[s] = 0;
+          __threadfence_block();
+          att_mbar_arrive(att_smem_u32(&rg.empty[s]));
+        }
+      }
+    }
+    st.store(a.P, (size_t)c + (size_t)x.b * Hkv + x.h, ks, row0, g.nq, lane);
+    t += n;
+  }
+  // tail segments: (b, h) number x goes to block G-1-(x mod G), key share 0 only
+  if (ks == 0) {
+    for (int x = G - 1 - c; x < B * Hkv; x += G) {
+      const int b = x / Hkv, h = x % Hkv;
+      const int L = pl.L[b], seq = args->seq_ids[b];
+      st.reset();
+      st.load_q(a.Qb + ((size_t)b * Hkv + h) * g.nq * HD, row0, g.nq, lane);
+      auto krow = [&](int kq) -> const bf16* {
+        const int pos = L + kq;
+        const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
+        return kv_row<bf16>(kv, a.layer, page, 0, h, pos % 16);
+      };
+      auto vrow = [&](int kq) -> const bf16* {
+        const int pos = L + kq;
+        const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
+        return kv_row<bf16>(kv, a.layer, page, 1, h, pos % 16);
+      };
+      st.tail(krow, vrow, rows, row0, g.nq, lane);
+      st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
+    }
+  }
+  return true;
+}
+
+template <int HD>
+__device__ __forceinline__ bool att_consume_dispatch(const AttRing& rg, int& it, const AttPlan& pl, const AttGeom& g,
+                                                     const StepArgs* __restrict__ args, const KvView& kv, const AttArgs& a,
+                                                     int Hkv, int c, int G, int cw, int lane) {
+  if (g.KW == 16) return att_consume<HD, 2>(rg, it, pl, g, args, kv, a, Hkv, c, G, cw, lane);
+  if (g.KW == 32) return att_consume<HD, 4>(rg, it, pl, g, args, kv, a, Hkv, c, G, cw, lane);
+  if constexpr (HD == 64) return att_consume<HD, 8>(rg, it, pl, g, args, kv, a, Hkv, c, G, cw, lane);
+  return true;
+}
+
+// ---------------------------------------------------------------------------------------------
+// stand-alone kernel (used by the multi-kernel step): warp 0 streams the ring, warps 1..8 consume
+// ---------------------------------------------------------------------------------------------
+constexpr int kAttStages = 8;
+constexpr int kAttTcThreads = 32 * (1 + kAttMaxWarps);
+struct AttSmemCtl {
+  uint64_t full[kAttStages];
+  uint64_t empty[kAttStages];
+  int cons_cnt[kAttStages];
+  int abort_flag;
+  AttPlan plan;
+};
+
 template <int HD>
 __global__ void __launch_bounds__(kAttTcThreads, 1)
 k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__ args, KvView kv, Work w, Dims dm,
@@ -407,7 +522,6 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
   pdl_launch();
   const int B = args->B, rows = args->gamma + 1, Hkv = dm.Hkv;
   const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
-  const int n_active = g.MT * g.KS;
   if (threadIdx.x == 0) {
     for (int i = 0; i < kAttStages; ++i) {
       att_mbar_init(att_smem_u32(&ctl->full[i]), 1);
@@ -420,93 +534,26 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
   }
   __syncthreads();
   const AttPlan& pl = ctl->plan;
-  const long long T = pl.T;
   const int G = gridDim.x, c = blockIdx.x;
-  const long long t_lo = (long long)c * T / G, t_hi = (long long)(c + 1) * T / G;
   volatile int* abort_flag = &ctl->abort_flag;
-
   if (warp == 0) {
     if (lane == 0) {
+      const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
       int it = 0;
       for (long long t = t_lo; t < t_hi; ++t, ++it) {
         const int s = it % kAttStages, round = it / kAttStages;
         if (round > 0 && !att_mbar_wait(att_smem_u32(&ctl->empty[s]), (round - 1) & 1, abort_flag, w.status)) break;
-        const int b = att_find_seq(pl.pre, B, (int)t);
-        const int nt_b = (pl.L[b] + g.KPS - 1) / g.KPS;
-        const int rem = (int)t - pl.pre[b], h = rem / nt_b, ti = rem % nt_b;
-        att_issue_tile(&tmKV, kv, a.layer, args->seq_ids[b], h, ti, pl.L[b], g.KPS, HD,
-                       att_smem_u32(ring + (size_t)s * kAttStageBytes), att_smem_u32(&ctl->full[s]));
+        const AttTile x = att_locate(pl, B, g.KPS, (int)t);
+        const uint32_t bar = att_smem_u32(&ctl->full[s]);
+        att_mbar_expect_tx(bar, kAttStageBytes);
+        att_issue_tile(&tmKV, kv, a.layer, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD,
+                       att_smem_u32(ring + (size_t)s * kAttStageBytes), bar);
       }
     }
-  } else {
-    const int cw = warp - 1;
-    if (cw < n_active) {
-      const int mi = cw / g.KS, ks = cw % g.KS, row0 = mi * 16;
-      auto run = [&](auto tag) {
-        constexpr int NT = decltype(tag)::value;
-        AttWarp<HD, NT> st;
-        // ring segments
-        int it = 0;
-        long long t = t_lo;
-        bool alive = true;
-        while (t < t_hi && alive) {
-          const int b = att_find_seq(pl.pre, B, (int)t);
-          const int L = pl.L[b];
-          const int nt_b = (L + g.KPS - 1) / g.KPS;
-          const int rem = (int)t - pl.pre[b], h = rem / nt_b, ti0 = rem % nt_b;
-          const int n = (int)min((long long)(nt_b - ti0), t_hi - t);
-          st.reset();
-          st.load_q(a.Qb + ((size_t)b * Hkv + h) * g.nq * HD, row0, g.nq, lane);
-          for (int i = 0; i < n; ++i, ++it) {
-            const int s = it % kAttStages;
-            const uint32_t bar = att_smem_u32(&ctl->full[s]);
-            int ok = 1;
-            if (lane == 0) ok = att_mbar_wait(bar, (it / kAttStages) & 1, abort_flag, w.status) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) { alive = false; break; }
-            att_mbar_try(bar, (it / kAttStages) & 1);   // every lane observes the completed phase
-            __syncwarp();
-            st.tile(att_smem_u32(ring + (size_t)s * kAttStageBytes), ks * g.KW, (ti0 + i) * g.KPS + ks * g.KW, L, lane);
-            __syncwarp();
-            if (lane == 0) {
-              __threadfence_block();
-              if (atomicAdd(&ctl->cons_cnt[s], 1) == n_active - 1) {
-                ctl->cons_cnt[s] = 0;
-                __threadfence_block();
-                att_mbar_arrive(att_smem_u32(&ctl->empty[s]));
-              }
-            }
-          }
-          if (!alive) break;
-          st.store(a.P, (size_t)c + (size_t)b * Hkv + h, ks, row0, g.nq, lane);
-          t += n;
-        }
-        // tail segments: (b, h) number x goes to block G-1-(x mod G), key share 0 only
-        if (alive && ks == 0) {
-          for (int x = G - 1 - c; x < B * Hkv; x += G) {
-            const int b = x / Hkv, h = x % Hkv;
-            const int L = pl.L[b], seq = args->seq_ids[b];
-            st.reset();
-            st.load_q(a.Qb + ((size_t)b * Hkv + h) * g.nq * HD, row0, g.nq, lane);
-            auto krow = [&](int kq) -> const bf16* {
-              const int pos = L + kq;
-              const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
-              return kv_row<bf16>(kv, a.layer, page, 0, h, pos % 16);
-            };
-            auto vrow = [&](int kq) -> const bf16* {
-              const int pos = L + kq;
-              const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
-              return kv_row<bf16>(kv, a.layer, page, 1, h, pos % 16);
-            };
-            st.tail(krow, vrow, rows, row0, g.nq, lane);
-            st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
-          }
-        }
-      };
-      if (g.KW == 16) run(std::integral_constant<int, 2>());
-      else if (g.KW == 32) run(std::integral_constant<int, 4>());
-      else if constexpr (HD == 64) run(std::integral_constant<int, 8>());
-    }
+  } else if (warp - 1 < g.MT * g.KS) {
+    AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, kAttStageBytes, kAttStages, abort_flag, nullptr, w.status};
+    int it = 0;
+    att_consume_dispatch<HD>(rg, it, pl, g, args, kv, a, Hkv, c, G, warp - 1, lane);
   }
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) __nanosleep(20000);   // let copies in flight land before the block retires
@@ -514,44 +561,68 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
 
 // Merge the partials of one (sequence, KV head, query row): ring segments in block order, their
 // sub-partials in key-share order, then the tail.  One warp per item; writes the O-projection input.
-// G_att: grid of the attention pass.
+// G_att: number of blocks of the attention pass.  Partial buffers are zero-filled at allocation, so the
+// slots of blocks without tiles (weight 0) hold finite values.
 template <typename T, int HD>
 __device__ __forceinline__ void att_combine_item(const AttPartials& P, const AttPlan& pl, const AttGeom& g, int G_att,
-                                                 int n_tail_base, int Hkv, int item, int B, void* ATT, int R, int Hq,
-                                                 int lane) {
+                                                 int n_tail_base, int Hkv, int item, void* ATT, int R, int Hq, int lane) {
   const int q = item % g.nq, bh = item / g.nq, b = bh / Hkv, h = bh % Hkv;
   const int L = pl.L[b];
   const int nt_b = (L + g.KPS - 1) / g.KPS;
-  int c_first = 0, c_last = -1;
+  int c_first = 0, n_cta = 0;
   if (nt_b > 0) {
     const long long t0 = (long long)pl.pre[b] + (long long)h * nt_b;
     c_first = att_owner(t0, pl.T, G_att);
-    c_last = att_owner(t0 + nt_b - 1, pl.T, G_att);
+    n_cta = att_owner(t0 + nt_b - 1, pl.T, G_att) - c_first + 1;
   }
+  const int n_sub = n_cta * g.KS + 1;   // the last one is the tail
+  auto sub_index = [&](int k) -> size_t {
+    if (k >= n_sub - 1) return ((size_t)(n_tail_base + bh) * kAttMaxSub) * g.nq + q;
+    const int cc = c_first + k / g.KS, ks = k % g.KS;
+    return (((size_t)cc + bh) * kAttMaxSub + ks) * g.nq + q;
+  };
+  auto sub_live = [&](int k) -> bool {
+    if (k == n_sub - 1) return true;
+    const int cc = c_first + k / g.KS;
+    return (long long)(cc + 1) * pl.T / G_att > (long long)cc * pl.T / G_att;
+  };
   constexpr int DPL = HD / 32;   // dims per lane
-  float M = -INFINITY;
-  auto has_tiles = [&](int c) { return (long long)(c + 1) * pl.T / G_att > (long long)c * pl.T / G_att; };
-  for (int c = c_first; c <= c_last; ++c)
-    if (has_tiles(c))
-      for (int ks = 0; ks < g.KS; ++ks) M = fmaxf(M, __ldcg(P.m + (((size_t)c + bh) * kAttMaxSub + ks) * g.nq + q));
-  const size_t tail_idx = ((size_t)(n_tail_base + bh) * kAttMaxSub) * g.nq + q;
-  M = fmaxf(M, __ldcg(P.m + tail_idx));
-  float lsum = 0.f, acc[DPL];
+  float lsum = 0.f, Mrun = -INFINITY, acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-  auto add = [&](size_t idx) {
-    const float m = __ldcg(P.m + idx);
-    if (m == -INFINITY) return;
-    const float wgt = exp2f(m - M);
-    lsum += __ldcg(P.l + idx) * wgt;
-    const float* op = P.o + idx * HD + lane * DPL;
+  for (int k0 = 0; k0 < n_sub; k0 += 96) {   // 96 sub-partials at a time (three per lane)
+    float mk[3], Mb = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < DPL; ++i) acc[i] += __ldcg(op + i) * wgt;
-  };
-  for (int c = c_first; c <= c_last; ++c)
-    if (has_tiles(c))
-      for (int ks = 0; ks < g.KS; ++ks) add((((size_t)c + bh) * kAttMaxSub + ks) * g.nq + q);
-  add(tail_idx);
+    for (int u = 0; u < 3; ++u) {
+      const int k = k0 + u * 32 + lane;
+      mk[u] = (k < n_sub && sub_live(k)) ? __ldcg(P.m + sub_index(k)) : -INFINITY;
+      Mb = fmaxf(Mb, mk[u]);
+    }
+    Mb = warp_max(Mb);
+    const float Mnew = fmaxf(Mrun, Mb);
+    if (Mnew == -INFINITY) continue;   // warp-uniform: nothing live so far
+    const float rescale = (Mrun == -INFINITY) ? 0.f : exp2f(Mrun - Mnew);
+    lsum *= rescale;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] *= rescale;
+    Mrun = Mnew;
+    float wk[3], lpart = 0.f;
+#pragma unroll
+    for (int u = 0; u < 3; ++u) {
+      const int k = k0 + u * 32 + lane;
+      wk[u] = (mk[u] == -INFINITY) ? 0.f : exp2f(mk[u] - Mnew);
+      if (wk[u] != 0.f) lpart += __ldcg(P.l + sub_index(k)) * wk[u];
+    }
+    lsum += warp_sum(lpart);
+    const int kn = min(96, n_sub - k0);
+#pragma unroll 4
+    for (int k = 0; k < kn; ++k) {
+      const float wgt = __shfl_sync(0xffffffffu, k < 32 ? wk[0] : (k < 64 ? wk[1] : wk[2]), k & 31);
+      const float* op = P.o + sub_index(k0 + k) * HD + lane * DPL;
+#pragma unroll
+      for (int i = 0; i < DPL; ++i) acc[i] += __ldcg(op + i) * wgt;
+    }
+  }
   const int gq = q / g.rows, j = q % g.rows, r = b * g.rows + j, head = h * g.group + gq;
   const float inv = 1.0f / lsum;
 #pragma unroll
@@ -571,7 +642,7 @@ __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dim
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
   const int items = B * dm.Hkv * g.nq;
   for (int item = blockIdx.x * wpb + warp; item < items; item += gridDim.x * wpb)
-    att_combine_item<bf16, HD>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, B, w.ATT, B * rows, dm.Hq, lane);
+    att_combine_item<bf16, HD>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, w.ATT, B * rows, dm.Hq, lane);
 }
 
 }  // namespace sj
