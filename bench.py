@@ -329,6 +329,7 @@ def main():
     roofline = {"bound": "hbm", "achieved": None, "peak": peak, "unit": "GB/s", "frac": None, "traffic": None,
                 "peak_kind": peak_kind}
     breakdown = {}
+    mega_launches = 0
     if not args.no_breakdown:
         with torch.cuda.stream(stream):
             dw.target.set_option("graph", 0)
@@ -351,16 +352,28 @@ def main():
             breakdown["attn"] = {"launches_per_step": (n_a - n_c) // n_inst, "ms_per_step": (ms_a - ms_c) / n_inst}
             tot += (ms_a - ms_c) / n_inst
             for v in breakdown.values():
-                v["share"] = v["ms_per_step"] / tot
+                v["share"] = v["ms_per_step"] / tot if tot > 0 else 0.0
             g_ms, g_n = dw.target.kernel_time("gemm")
+            v_ms, v_n = dw.target.kernel_time("verify_step")
             dw.target.set_option("timing", 0)
             dw.target.set_option("graph", 1)
-        # k_gemm_tc: all projections + LM head; algorithmic bytes = every streamed weight byte once
-        per_launch_bytes = w_bytes / (g_n / n_inst)
-        per_launch_s = (g_ms / g_n) / 1e3
-        roofline.update({"kernel": "k_gemm_tc", "launches_per_step": g_n // n_inst,
-                         "achieved": per_launch_bytes / per_launch_s / 1e9,
-                         "avg_launch_us": per_launch_s * 1e6, "algorithmic_bytes_per_launch": per_launch_bytes})
+        if v_n:
+            # k_verify_mega: the whole step in one persistent kernel; algorithmic bytes = every streamed
+            # weight byte and every live cache byte once
+            mega_launches = v_n // n_inst
+            breakdown = {"verify_step": {"launches_per_step": mega_launches, "ms_per_step": v_ms / n_inst, "share": 1.0}}
+            per_launch_bytes = (w_bytes + kv_bytes) / mega_launches
+            per_launch_s = (v_ms / v_n) / 1e3
+            roofline.update({"kernel": "k_verify_mega", "launches_per_step": mega_launches,
+                             "achieved": per_launch_bytes / per_launch_s / 1e9,
+                             "avg_launch_us": per_launch_s * 1e6, "algorithmic_bytes_per_launch": per_launch_bytes})
+        else:
+            # k_gemm_tc: all projections + LM head; algorithmic bytes = every streamed weight byte once
+            per_launch_bytes = w_bytes / (g_n / n_inst)
+            per_launch_s = (g_ms / g_n) / 1e3
+            roofline.update({"kernel": "k_gemm_tc", "launches_per_step": g_n // n_inst,
+                             "achieved": per_launch_bytes / per_launch_s / 1e9,
+                             "avg_launch_us": per_launch_s * 1e6, "algorithmic_bytes_per_launch": per_launch_bytes})
         roofline["frac"] = roofline["achieved"] / peak
 
     cpu_baseline = None
@@ -384,7 +397,8 @@ def main():
         "algorithmic_bytes_per_step": w_bytes + kv_bytes,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e},
-        "gpu_launches": dw.launches_per_step(mode) * args.steps,
+        "gpu_launches": (mega_launches + 1 + (1 if mode == binding.MODE_SAMPLING else 0) if mega_launches
+                         else dw.launches_per_step(mode)) * args.steps,
         "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline, "kernel_breakdown": breakdown,
     }
     print(json.dumps(line))

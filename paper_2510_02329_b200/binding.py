@@ -24,7 +24,7 @@ MODE_GREEDY, MODE_SAMPLING = 0, 1
 EXPORTS = ["sj_create_target", "sj_destroy_target", "sj_load_judge_head", "sj_set_option", "sj_sync",
            "sj_kv_create", "sj_kv_destroy", "sj_kv_fill", "sj_kv_read", "sj_kv_set_len", "sj_kv_set_pending",
            "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_gemm_skinny_noalloc", "sj_last_error",
-           "sj_kernel_time"]
+           "sj_kernel_time", "sj_step_trace"]
 
 
 class SjError(RuntimeError):
@@ -97,6 +97,7 @@ def load(build_if_needed: bool = True) -> C.CDLL:
     lib.sj_rollback_kv.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int), C.c_int]
     lib.sj_gemm_skinny.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p]
+    lib.sj_step_trace.argtypes = [C.c_void_p, C.POINTER(C.c_ulonglong), C.c_int, C.POINTER(C.c_int)]
     lib.sj_gemm_skinny_noalloc.argtypes = [C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     _lib = lib
     return lib
@@ -163,6 +164,13 @@ class Target:
         ms, n = C.c_double(), C.c_long()
         check(self._lib.sj_kernel_time(self.handle, name.encode(), C.byref(ms), C.byref(n)))
         return ms.value, n.value
+
+    def step_trace(self, max_entries: int = 2048 + 8 * 512):
+        """Timeline (ns) of the last persistent-kernel step run with option ``trace`` = 1."""
+        buf = (C.c_ulonglong * max_entries)()
+        n = C.c_int()
+        check(self._lib.sj_step_trace(self.handle, buf, max_entries, C.byref(n)))
+        return list(buf[: n.value])
 
     def close(self) -> None:
         if self.handle:

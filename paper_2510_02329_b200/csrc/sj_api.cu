@@ -14,6 +14,7 @@
 #include "../../include/sj.h"
 #include "sj_attn_tc.cuh"
 #include "sj_gemm_tc.cuh"
+#include "sj_mega.cuh"
 
 using namespace sj;
 
@@ -163,6 +164,7 @@ static RowGeom row_geom(int R) {
 struct LayerW {
   const void *wq, *wk, *wv, *wo, *wg, *wu, *wd, *na, *nf, *bq, *bk, *bv;
   CUtensorMap m_q, m_k, m_v, m_o, m_g, m_u, m_d;
+  CUtensorMap m_g64, m_u64;   // gate / up with boxes of 64 rows (whole-step kernel)
 };
 
 struct StepKey {
@@ -188,7 +190,14 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0;
+  bool mega_shapes = false, coop = false;
+  MegaLayerPtrs* d_layer_ptrs = nullptr;
+  float* d_sumsq = nullptr;
+  float* d_pbuf = nullptr;
+  unsigned* d_sync = nullptr;      // [0] barrier counter, [1] abort word, [2..3] timeout note, [16 ..) split-K flags
+  unsigned long long* d_trace = nullptr;
+  std::vector<MegaMaps> mega_maps;  // one per launch chunk of kMegaMaxLayers layers
   struct Timed { const char* name; cudaEvent_t a, b; };
   std::vector<Timed> timed;
   TcSite s_qkv, s_o, s_gu, s_down, s_lm;
@@ -390,6 +399,8 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
       if ((st = make_map(&L.m_g, L.wg, c.d_ffn, c.d_model, kTileN)) != SJ_OK) return bail(st);
       if ((st = make_map(&L.m_u, L.wu, c.d_ffn, c.d_model, kTileN)) != SJ_OK) return bail(st);
       if ((st = make_map(&L.m_d, L.wd, c.d_model, c.d_ffn, kTileN)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_g64, L.wg, c.d_ffn, c.d_model, 64)) != SJ_OK) return bail(st);
+      if ((st = make_map(&L.m_u64, L.wu, c.d_ffn, c.d_model, 64)) != SJ_OK) return bail(st);
     }
     if ((st = make_map(&t->m_lm, t->lm_head, c.vocab, c.d_model, kTileN)) != SJ_OK) return bail(st);
     cudaError_t e = cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -397,6 +408,51 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   }
   t->p_elems = p_elems;
   ALLOC(W.P, float, p_elems);
+  {
+    int coop = 0;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    t->coop = coop != 0;
+  }
+  t->mega_shapes = tc && t->coop && c.d_ffn % 64 == 0;
+  if (t->mega_shapes) {
+    const int Rm = std::min(R, kMegaMaxRows);
+    ALLOC(t->d_layer_ptrs, MegaLayerPtrs, c.n_layers);
+    ALLOC(t->d_sumsq, float, (size_t)2 * (c.d_model / kTileN) * kMegaMaxRows);
+    ALLOC(t->d_pbuf, float, (size_t)t->sm_count * pad16(Rm) * kTileN);
+    ALLOC(t->d_sync, unsigned, 16 + t->sm_count);
+    std::vector<MegaLayerPtrs> lp(c.n_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+      const LayerW& L = t->layers[l];
+      lp[l].bq = (const bf16*)L.bq; lp[l].bk = (const bf16*)L.bk; lp[l].bv = (const bf16*)L.bv;
+      lp[l].gain_ffn = (const bf16*)L.nf;
+      lp[l].gain_next = (const bf16*)(l + 1 < c.n_layers ? t->layers[l + 1].na : t->final_norm);
+    }
+    cudaError_t e = cudaMemcpy(t->d_layer_ptrs, lp.data(), lp.size() * sizeof(MegaLayerPtrs), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(t->d_sumsq, 0, sizeof(float) * 2 * (c.d_model / kTileN) * kMegaMaxRows);
+    if (e == cudaSuccess) e = cudaMemset(t->d_pbuf, 0, sizeof(float) * (size_t)t->sm_count * pad16(Rm) * kTileN);
+    if (e == cudaSuccess) e = cudaMemset(t->d_sync, 0, sizeof(unsigned) * (16 + t->sm_count));
+    if (e == cudaSuccess)
+      e = c.head_dim == 128
+              ? cudaFuncSetAttribute(k_verify_mega<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+              : cudaFuncSetAttribute(k_verify_mega<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "whole-step kernel set-up: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
+    for (int l0 = 0; l0 < c.n_layers; l0 += kMegaMaxLayers) {
+      t->mega_maps.emplace_back();
+      MegaMaps& mm = t->mega_maps.back();
+      memset(&mm, 0, sizeof(mm));
+      for (int l = l0; l < std::min(c.n_layers, l0 + kMegaMaxLayers); ++l) {
+        const LayerW& L = t->layers[l];
+        mm.wq[l - l0] = L.m_q; mm.wk[l - l0] = L.m_k; mm.wv[l - l0] = L.m_v; mm.wo[l - l0] = L.m_o;
+        mm.wg[l - l0] = L.m_g64; mm.wu[l - l0] = L.m_u64; mm.wd[l - l0] = L.m_d;
+      }
+      mm.lm = t->m_lm;
+    }
+    // the activation planes are read as GEMM operands: rows past R must stay finite
+    cudaMemset(W.A, 0, act_rows * c.d_model * esz);
+    cudaMemset(W.ATT, 0, act_rows * qd * esz);
+    cudaMemset(W.H, 0, act_rows * c.d_ffn * esz);
+    t->opt_step = 1;
+  }
 #undef ALLOC
   if (t->bf) {
     const int att_smem = kAttStages * kAttStageBytes + (int)sizeof(AttSmemCtl) + 1024;
@@ -448,6 +504,18 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "attn_impl must be 0 or 1");
     if (value == 1 && !t->bf) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention needs a bf16 model");
     t->opt_attn = value;
+  } else if (n == "step_impl") {
+    if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "step_impl must be 0 or 1");
+    if (value == 1 && !t->mega_shapes) return fail(SJ_ERR_UNSUPPORTED, "the whole-step kernel needs bf16, 128-multiples and cooperative launch");
+    t->opt_step = value;
+  } else if (n == "trace") {
+    const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 8 * kMegaTraceSites;
+    if (value && !t->d_trace) {
+      sj_status st = dev_alloc(t, &t->d_trace, n_tr);
+      if (st != SJ_OK) return st;
+    }
+    if (t->d_trace) CU_TRY(cudaMemsetAsync(t->d_trace, 0, sizeof(unsigned long long) * n_tr, t->stream));
+    t->opt_trace = value ? 1 : 0;
   } else if (n == "graph") {
     if (value && !t->stream) return fail(SJ_ERR_UNSUPPORTED, "the legacy default stream cannot be captured into a graph");
     t->opt_graph = value ? 1 : 0;
@@ -471,6 +539,12 @@ extern "C" sj_status sj_sync(sj_target* t) {
   CU_TRY(cudaStreamSynchronize(t->stream));
   if (st != 0) {
     CU_TRY(cudaMemsetAsync(t->work.status, 0, sizeof(int), t->stream));
+    if (st == DEV_TIMEOUT && t->d_sync) {
+      unsigned info[4] = {0, 0, 0, 0};   // the whole-step kernel notes which wait gave up first
+      CU_TRY(cudaMemcpy(info, t->d_sync, sizeof(info), cudaMemcpyDeviceToHost));
+      return fail(SJ_ERR_TIMEOUT, "a bounded device-side wait ran out (barrier count %u, wait kind %u in block %u, detail %u)",
+                  info[0], info[2] & 255u, info[2] >> 8, info[3]);
+    }
     return fail((sj_status)st, st == DEV_TIMEOUT ? "a bounded device-side wait ran out"
                                                  : "device rejected a state change (rollback beyond the live length)");
   }
@@ -851,6 +925,96 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
 
 #undef TIMED
 
+// The whole step as one cooperative launch per chunk of kMegaMaxLayers layers.
+static bool mega_usable(const sj_target* t, const sj_kv* kv, int B, int gamma) {
+  const int rows = gamma + 1, R = B * rows, group = t->dm.Hq / t->dm.Hkv;
+  return t->opt_step == 1 && t->opt_gemm == 1 && t->mega_shapes && kv->has_tm_pool && R <= kMegaMaxRows &&
+         group * rows <= 16 * 6 && t->stream != nullptr;
+}
+
+static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode, bool use_scratch) {
+  const Dims& dm = t->dm;
+  const int rows = gamma + 1, R = B * rows, Rp = pad16(R), qd = dm.Hq * dm.hd;
+  cudaStream_t s = t->stream;
+  Work W = t->work;
+  if (!use_scratch) W.logits = nullptr;
+  const CUtensorMap *mA_d = nullptr, *mA_q = nullptr, *mA_f = nullptr;
+  sj_status st;
+  if ((st = activation_map(t, t->mapA_d, W.A, R, dm.d, &mA_d)) != SJ_OK) return st;
+  if ((st = activation_map(t, t->mapA_q, W.ATT, R, qd, &mA_q)) != SJ_OK) return st;
+  if ((st = activation_map(t, t->mapA_f, W.H, R, dm.F, &mA_f)) != SJ_OK) return st;
+  MegaParams p;
+  memset(&p, 0, sizeof(p));
+  p.B = B; p.rows = rows; p.R = R; p.Rp = Rp;
+  p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
+  const int budget = 227 * 1024 - 1024 - (int)sizeof(MegaCtl);
+  p.stages = std::min(kMegaMaxStages, budget / p.stage_bytes);
+  if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
+  uint32_t tc = 32;
+  while (tc < (uint32_t)(4 * Rp)) tc <<= 1;
+  p.tmem_cols = tc;
+  p.lp = t->d_layer_ptrs;
+  p.embed = (const bf16*)t->embed;
+  p.gain0 = (const bf16*)t->layers[0].na;
+  p.sumsq = t->d_sumsq;
+  p.pbuf = t->d_pbuf;
+  p.gbar = t->d_sync;
+  p.abort_g = reinterpret_cast<int*>(t->d_sync + 1);
+  p.flags = reinterpret_cast<int*>(t->d_sync + 16);
+  p.n_tail_base = t->sm_count + B * dm.Hkv;
+  p.trace = t->opt_trace ? t->d_trace : nullptr;
+  const size_t smem = (size_t)p.stages * p.stage_bytes + sizeof(MegaCtl) + 1024;
+  const bool timing = t->opt_timing != 0;
+  const int NL = dm.n_layers;
+  for (size_t ci = 0; ci < t->mega_maps.size(); ++ci) {
+    p.l0 = (int)ci * kMegaMaxLayers;
+    p.l1 = std::min(NL, p.l0 + kMegaMaxLayers);
+    p.do_embed = ci == 0 ? 1 : 0;
+    p.do_lm = p.l1 == NL ? 1 : 0;
+    MegaMaps mm = t->mega_maps[ci];
+    mm.pool = kv->tm_pool;
+    mm.a_d = *mA_d; mm.a_q = *mA_q; mm.a_f = *mA_f;
+    CU_TRY(cudaMemsetAsync(t->d_sync, 0, sizeof(unsigned) * (16 + t->sm_count), s));
+    cudaEvent_t ea = nullptr, eb = nullptr;
+    if (timing) {
+      CU_TRY(cudaEventCreate(&ea));
+      CU_TRY(cudaEventCreate(&eb));
+      CU_TRY(cudaEventRecord(ea, s));
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(t->sm_count);
+    cfg.blockDim = dim3(kMegaThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeCooperative;
+    at[0].val.cooperative = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    const StepArgs* args = t->d_args;
+    if (dm.hd == 128) CU_TRY(cudaLaunchKernelEx(&cfg, k_verify_mega<128>, mm, p, args, kv->view, W, dm));
+    else CU_TRY(cudaLaunchKernelEx(&cfg, k_verify_mega<64>, mm, p, args, kv->view, W, dm));
+    if (timing) {
+      CU_TRY(cudaEventRecord(eb, s));
+      t->timed.push_back({"verify_step", ea, eb});
+    }
+  }
+  if (mode == SJ_MODE_SAMPLING)
+    CU_TRY(launch(k_resample, dim3(B), dim3(1024), 0, s, false, (const StepArgs*)t->d_args, kv->view, W, dm));
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_step_trace(sj_target* t, unsigned long long* out_ns, int max_entries, int* n_entries) {
+  if (!t || !out_ns || !n_entries || max_entries <= 0) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (!t->d_trace) return fail(SJ_ERR_STATE, "tracing was never enabled (sj_set_option \"trace\")");
+  const int n = std::min(max_entries, 2 * kMegaTraceBarriers + 8 * kMegaTraceSites);
+  CU_TRY(cudaStreamSynchronize(t->stream));
+  CU_TRY(cudaMemcpy(out_ns, t->d_trace, sizeof(unsigned long long) * n, cudaMemcpyDeviceToHost));
+  *n_entries = n;
+  return SJ_OK;
+}
+
 extern "C" sj_status sj_kernel_time(sj_target* t, const char* name, double* total_ms, long* launches) {
   if (!t || !name || !total_ms || !launches) return fail(SJ_ERR_INVALID_ARG, "null argument");
   CU_TRY(cudaStreamSynchronize(t->stream));
@@ -924,7 +1088,8 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
   const int chunk_len = pick_chunk_len(t, total_keys);
   for (int i = 0; i < B; ++i) chunk_need_base += (size_t)(kv->len_hi[a->seq_ids[i]] + rows + chunk_len - 1) / chunk_len;
 
-  const bool use_scratch = a->mode == SJ_MODE_SAMPLING || t->opt_gemm == 0;
+  const bool use_mega = mega_usable(t, kv, B, gamma);
+  const bool use_scratch = a->mode == SJ_MODE_SAMPLING || (t->opt_gemm == 0 && !use_mega);
   // grow lazily-sized buffers (outside any capture)
   if (chunk_need_base > t->att_chunks_cap || rows > t->att_rows_cap) {
     CU_TRY(cudaStreamSynchronize(t->stream));
@@ -945,7 +1110,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
     t->att_chunks_cap = cap;
     t->att_rows_cap = rcap;
   }
-  if (t->opt_attn == 1 && t->bf && kv->has_tm_pool) {
+  if ((t->opt_attn == 1 || use_mega) && t->bf && kv->has_tm_pool) {
     const size_t slots = (size_t)t->sm_count + 2 * (size_t)B * t->dm.Hkv;
     const size_t need = slots * kAttMaxSub * (size_t)(group * rows);
     if (need > t->tc_part_cap) {
@@ -997,7 +1162,9 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
   CU_TRY(cudaMemcpyAsync(t->d_args, &h, sizeof(h), cudaMemcpyHostToDevice, t->stream));
 
   StepKey key{B, gamma, a->mode, chunk_len, t->opt_gemm, t->opt_attn, t->opt_pdl, use_scratch ? 1 : 0};
-  if (t->opt_graph) {
+  if (use_mega) {
+    if ((st = launch_mega(t, kv, B, gamma, a->mode, use_scratch)) != SJ_OK) return st;
+  } else if (t->opt_graph) {
     auto it = t->graphs.find(key);
     if (it == t->graphs.end()) {
       if (t->opt_gemm == 1) {  // encode activation maps before capturing

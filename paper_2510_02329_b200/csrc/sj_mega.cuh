@@ -1,0 +1,872 @@
+// The whole verification step as ONE persistent cooperative kernel (bf16 models, up to kMegaMaxRows
+// block rows): one thread block per SM, every phase of every layer executed by the same blocks with a
+// device-wide barrier between dependent phases.
+//
+// Why: at batch 1 the step is a chain of ~200 dependent phases of 10-100 us each, and the only thing
+// that takes time is streaming 15 GB of weights (plus the KV cache) from HBM.  Weights and cached K/V
+// do not depend on activations, so each block's producer warp streams ITS share of every phase's
+// weights and cache tiles through one shared-memory ring without ever stopping at a phase boundary;
+// consumers (the tcgen05 issuer, the attention warps) catch up after each barrier.  HBM stays busy
+// across barriers for as long as the ring has free stages.
+//
+// Roles per block (384 threads):
+//   warp 0      weight / cache-tile producer (TMA into the ring)
+//   warp 1      tcgen05.mma issuer, owns the TMEM allocation
+//   warp 2      activation producer: TMA of the activation K-slices, gated by the device-wide barrier
+//   warps 4..11 workers: the first four drain TMEM (fused epilogues), all eight run attention, the
+//               combine, the embedding and the final acceptance phase
+//
+// GEMM phases: work units are (128-feature tile, 64-wide K block) in tile-major order, dealt evenly to
+// the blocks (stream-K).  A block that holds the first K block of a tile owns the tile: other
+// contributors store fp32 partial sums to their slot and raise a flag; the owner adds them in block
+// order (deterministic) and runs the fused epilogue:
+//   QKV   -> scale by 1/rms, bias, rotary embedding; queries (bf16, pre-scaled) to the query buffer,
+//            K and V rows straight into the cache pages
+//   O     -> residual add, fp32 residual stream, next GEMM input planes (x * gain, hi/lo bf16), per-tile
+//            sum of squares (the 1/rms factor is applied by the consumer's epilogue: it is a row scalar)
+//   gate/up (tiles interleave 64 gate and 64 up features) -> silu(g) * u -> down-projection input planes
+//   down  -> as O
+//   LM head (whole tiles) -> softmax statistics per (vocabulary tile, row), logit of the drafted token
+// Attention: see sj_attn_tc.cuh; its cache tiles travel through the same ring.
+//
+// Every wait is bounded; the first one to run out raises a device-wide abort word that all other waits
+// poll, so that a logic error ends the kernel with SJ_ERR_TIMEOUT instead of hanging the GPU.
+#pragma once
+
+#include "sj_attn_tc.cuh"
+#include "sj_gemm_tc.cuh"
+
+namespace sj {
+
+constexpr int kMegaThreads = 384;
+constexpr int kMegaWorkers = 256;
+constexpr int kMegaMaxLayers = 32;   // per launch (tensor maps travel as kernel parameters)
+constexpr int kMegaMaxRows = 80;
+constexpr int kMegaMaxStages = 12;
+constexpr uint32_t kMegaSpin = 1u << 22;
+constexpr int kMegaTraceBarriers = 1024;
+constexpr int kMegaTraceSites = 512;
+
+enum MegaSite { SITE_QKV = 0, SITE_O = 1, SITE_GU = 2, SITE_DOWN = 3, SITE_LM = 4 };
+
+struct MegaMaps {
+  CUtensorMap wq[kMegaMaxLayers], wk[kMegaMaxLayers], wv[kMegaMaxLayers], wo[kMegaMaxLayers];
+  CUtensorMap wg[kMegaMaxLayers], wu[kMegaMaxLayers], wd[kMegaMaxLayers];   // wg, wu: boxes of 64 rows
+  CUtensorMap lm, pool, a_d, a_q, a_f;
+};
+
+struct MegaLayerPtrs {
+  const bf16 *bq, *bk, *bv;   // null without qkv_bias
+  const bf16* gain_ffn;       // RMSNorm gain applied to the O projection's output (input of gate/up)
+  const bf16* gain_next;      // gain applied to the down projection's output (next layer / final norm)
+};
+
+struct MegaParams {
+  int l0, l1, do_embed, do_lm;
+  int B, rows, R, Rp;
+  int stages, stage_bytes;
+  uint32_t tmem_cols;
+  const MegaLayerPtrs* lp;    // [n_layers], device
+  const bf16* embed;
+  const bf16* gain0;          // first layer's attention-norm gain
+  float* sumsq;               // [2][d/128][kMegaMaxRows]
+  float* pbuf;                // [blocks][Rp][128] split-K partial sums
+  unsigned* gbar;             // device-wide barrier counter   } zeroed before every launch
+  int* abort_g;               // device-wide abort word        }
+  int* flags;                 // [blocks] split-K flags        }
+  int n_tail_base;
+  // optional timeline of block 0 (global-timer nanoseconds):
+  //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
+  //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
+  //   load issued, 2 first stage ready at the MMA issuer, 3 last MMA committed, 4 last accumulator seen by the
+  //   epilogue, 5 split-K contributors' flags seen, 6 epilogue done, 7 weight producer issued the last load
+  unsigned long long* trace;
+};
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define MEGA_EV(sidx, k)                                                                             \
+  do {                                                                                               \
+    if (p.trace && blockIdx.x == 0 && (sidx) < kMegaTraceSites)                                      \
+      p.trace[2 * kMegaTraceBarriers + (sidx) * 8 + (k)] = global_timer_ns();                        \
+  } while (0)
+
+struct MegaCtl {
+  uint64_t full[kMegaMaxStages], empty[kMegaMaxStages], tmem_full[2], tmem_empty[2];
+  int cons_cnt[kMegaMaxStages];
+  uint32_t tmem_base;
+  int abort_flag;
+  int bars_passed;
+  int bcast[4];
+  float inv[kMegaMaxRows];
+  int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
+  float red[4][16];
+  RowStat wstat[4][16];
+  RowStat rs[kMaxGamma + 1];
+  float score[kMaxGamma + 1];
+  AttPlan plan;
+  union {
+    float exch[128][17];
+    RowStat sred[kMegaWorkers];
+  } u;
+};
+
+struct SiteInfo {
+  int n_tiles, KB;
+  long long u_lo, u_hi;
+};
+__host__ __device__ __forceinline__ SiteInfo site_info(int site, const Dims& dm, int c, int G) {
+  SiteInfo s;
+  const int qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd;
+  switch (site) {
+    case SITE_QKV: s.n_tiles = (qd + 2 * kd) / kTileN; s.KB = dm.d / kBK; break;
+    case SITE_O: s.n_tiles = dm.d / kTileN; s.KB = qd / kBK; break;
+    case SITE_GU: s.n_tiles = dm.F / 64; s.KB = dm.d / kBK; break;
+    case SITE_DOWN: s.n_tiles = dm.d / kTileN; s.KB = dm.F / kBK; break;
+    default: s.n_tiles = (dm.V + kTileN - 1) / kTileN; s.KB = dm.d / kBK; break;
+  }
+  const long long U = (long long)s.n_tiles * s.KB;
+  if (site == SITE_LM) {
+    s.u_lo = ((long long)c * s.n_tiles / G) * s.KB;
+    s.u_hi = ((long long)(c + 1) * s.n_tiles / G) * s.KB;
+  } else {
+    s.u_lo = (long long)c * U / G;
+    s.u_hi = (long long)(c + 1) * U / G;
+  }
+  return s;
+}
+// Block that owns unit u of a stream-K site.
+__device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
+  int c = (int)(u * G / U);
+  while ((long long)(c + 1) * U / G <= u) ++c;
+  return c;
+}
+
+template <typename FSite, typename FAtt>
+__device__ __forceinline__ void mega_walk(const MegaParams& p, FSite fsite, FAtt fatt) {
+  for (int l = p.l0; l < p.l1; ++l) {
+    fsite(SITE_QKV, l);
+    fatt(l);
+    fsite(SITE_O, l);
+    fsite(SITE_GU, l);
+    fsite(SITE_DOWN, l);
+  }
+  if (p.do_lm) fsite(SITE_LM, p.l1 - 1);
+}
+
+__device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_relaxed_add(unsigned* p, unsigned v) {
+  asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_s32(int* p, int v) {
+  asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Bounded wait on a shared-memory barrier that also watches the device-wide abort word.
+__device__ __forceinline__ bool mega_wait(uint32_t bar, uint32_t parity, MegaCtl* ctl, const MegaParams& p, int* status,
+                                          int where, int extra) {
+  return att_mbar_wait(bar, parity, &ctl->abort_flag, status, p.abort_g, where, extra);
+}
+// Bounded spin (relaxed polls; the caller fences after success) until *word (device memory, written by
+// other blocks) reaches `target`.
+__device__ __forceinline__ bool mega_spin_ge(const unsigned* word, unsigned target, MegaCtl* ctl, const MegaParams& p,
+                                             int* status, int where, int extra) {
+  volatile int* af = &ctl->abort_flag;
+  volatile int* ag = p.abort_g;
+  for (uint32_t i = 0; i < kMegaSpin; ++i) {
+    if (ld_relaxed_u32(word) >= target) return true;
+    if (i > 16) {
+      if (*af) return false;
+      if ((i & 63) == 0 && *ag) { *af = 1; return false; }
+      if (i > 4096) __nanosleep(64);
+    }
+  }
+  *af = 1;
+  att_note_timeout(ag, where, extra);
+  *ag = 1;
+  atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+  return false;
+}
+
+// Device-wide barrier for the 256 workers of every block.  Returns false once the step is aborting.
+// Block-level barrier, then one thread publishes (fence, arrive) and waits (poll, fence): the fences are
+// cumulative over what the block barrier ordered before them.
+__device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p, int* status, int& nbar, int wt) {
+  fence_proxy_async();   // this phase's generic-proxy stores are read by other blocks' TMA loads
+  bar_sync(1, kMegaWorkers);
+  ++nbar;
+  if (wt == 0) {
+    const bool tr = p.trace && blockIdx.x == 0 && nbar < kMegaTraceBarriers;
+    if (tr) p.trace[2 * nbar] = global_timer_ns();
+    if (!ctl->abort_flag) {
+      __threadfence();
+      red_relaxed_add(p.gbar, 1u);
+      mega_spin_ge(p.gbar, (unsigned)nbar * gridDim.x, ctl, p, status, 8, nbar);
+    }
+    __threadfence();
+    if (tr) p.trace[2 * nbar + 1] = global_timer_ns();
+    *reinterpret_cast<volatile int*>(&ctl->bars_passed) = nbar;
+  }
+  bar_sync(1, kMegaWorkers);
+  return *reinterpret_cast<volatile int*>(&ctl->abort_flag) == 0;
+}
+
+// TMA loads of one weight unit into a ring stage.
+__device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int li, const Dims& dm, long long u, int KB,
+                                             uint32_t dst, uint32_t bar, uint64_t pol) {
+  const int tile = (int)(u / KB), kb = (int)(u % KB);
+  switch (site) {
+    case SITE_QKV: {
+      const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
+      if (tile < tq) tma_load_2d(dst, &mp.wq[li], bar, kb * kBK, tile * kTileN, pol);
+      else if (tile < tq + tk) tma_load_2d(dst, &mp.wk[li], bar, kb * kBK, (tile - tq) * kTileN, pol);
+      else tma_load_2d(dst, &mp.wv[li], bar, kb * kBK, (tile - tq - tk) * kTileN, pol);
+      break;
+    }
+    case SITE_O: tma_load_2d(dst, &mp.wo[li], bar, kb * kBK, tile * kTileN, pol); break;
+    case SITE_GU:
+      tma_load_2d(dst, &mp.wg[li], bar, kb * kBK, tile * 64, pol);
+      tma_load_2d(dst + 8192u, &mp.wu[li], bar, kb * kBK, tile * 64, pol);
+      break;
+    case SITE_DOWN: tma_load_2d(dst, &mp.wd[li], bar, kb * kBK, tile * kTileN, pol); break;
+    default: tma_load_2d(dst, &mp.lm, bar, kb * kBK, tile * kTileN, pol); break;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// fused epilogues (the four epilogue warps: 128 threads, named barrier 2)
+// ---------------------------------------------------------------------------------------------
+template <int HD>
+__device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p,
+                                              const StepArgs* __restrict__ args, const KvView& kv, const Work& w,
+                                              const Dims& dm, int et) {
+  const int sidx = gseq - 1;
+  const int c = blockIdx.x, G = gridDim.x, R = p.R, Rp = p.Rp, rows = p.rows;
+  const int quarter = et >> 5, lane = et & 31;
+  const SiteInfo si = site_info(site, dm, c, G);
+  if (si.u_hi <= si.u_lo) return;
+  const long long U = (long long)si.n_tiles * si.KB;
+  const int nt128 = dm.d / kTileN;
+  const MegaLayerPtrs lp = p.lp[l];
+  // 1/rms of this phase's input rows (the planes hold x * gain; the scalar is applied here).  One warp
+  // per row, lanes over the column tiles, fixed shuffle tree: all loads of a row are in flight together.
+  if (site == SITE_QKV || site == SITE_GU || site == SITE_LM) {
+    const int buf = (site == SITE_GU) ? 1 : 0;
+    for (int r0 = quarter; r0 < R; r0 += 16) {
+      float part[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int r = r0 + 4 * k;
+        part[k] = 0.f;
+        if (r < R)
+          for (int t = lane; t < nt128; t += 32) part[k] += __ldcg(p.sumsq + ((size_t)buf * nt128 + t) * kMegaMaxRows + r);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int r = r0 + 4 * k;
+        const float s = warp_sum(part[k]);
+        if (lane == 0 && r < R) ctl->inv[r] = 1.0f / sqrtf(s / (float)dm.d + dm.eps);
+      }
+    }
+    bar_sync(2, 128);
+  }
+  const int qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd, tq = qd / kTileN, tk = kd / kTileN;
+  const float invT = (site == SITE_LM) ? args->inv_temperature : 1.f;
+  float* dbg_logits = (site == SITE_LM) ? args->dbg_logits : nullptr;
+  const float qscale = 1.4426950408889634f / sqrtf((float)HD);
+
+  long long u = si.u_lo;
+  while (u < si.u_hi) {
+    const int tile = (int)(u / si.KB), kb0 = (int)(u % si.KB);
+    const int len = (int)min((long long)(si.KB - kb0), si.u_hi - u);
+    const int acc = seg & 1, use = seg >> 1;
+    if (et == 0) ctl->bcast[seg & 1] = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
+    bar_sync(2, 128);
+    if (!ctl->bcast[seg & 1]) return;
+    tc_fence_after();
+    if (et == 0) MEGA_EV(sidx, 4);
+    const bool owner = (kb0 == 0), complete = owner && (len == si.KB);
+    int c_last = c;
+    if (owner && !complete) {
+      c_last = unit_owner((long long)(tile + 1) * si.KB - 1, U, G);
+      if (et < 32) {   // one lane per contributing block
+        int ok = 1;
+        for (int base = c + 1; base <= c_last; base += 32) {
+          const int c2 = base + lane;
+          int okl = 1;
+          if (c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G)   // blocks without units add nothing
+            okl = mega_spin_ge(reinterpret_cast<const unsigned*>(p.flags + c2), (unsigned)gseq, ctl, p, w.status, 7, gseq) ? 1 : 0;
+          ok &= __all_sync(0xffffffffu, okl);
+        }
+        __threadfence();
+        if (et == 0) ctl->bcast[2] = ok;
+      }
+      bar_sync(2, 128);
+      if (!ctl->bcast[2]) return;
+      if (et == 0) MEGA_EV(sidx, 5);
+    }
+    const uint32_t taddr = ctl->tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 2 * Rp);
+    const int fl = et;   // feature inside the tile == TMEM lane
+
+    // per-tile constants of the fused epilogues
+    int kind = 0, head = 0, dim = 0;
+    float bias = 0.f;
+    const bf16* gain = nullptr;
+    if (site == SITE_QKV) {
+      int fs;
+      if (tile < tq) { kind = 0; fs = tile * kTileN + fl; }
+      else if (tile < tq + tk) { kind = 1; fs = (tile - tq) * kTileN + fl; }
+      else { kind = 2; fs = (tile - tq - tk) * kTileN + fl; }
+      head = fs / HD;
+      dim = fs % HD;
+      const bf16* bp = kind == 0 ? lp.bq : (kind == 1 ? lp.bk : lp.bv);
+      if (bp) bias = __bfloat162float(bp[fs]);
+    } else if (site == SITE_O) {
+      gain = lp.gain_ffn;
+    } else if (site == SITE_DOWN) {
+      gain = lp.gain_next;
+    }
+
+    for (int c0 = 0; c0 < Rp; c0 += 16) {
+      float v[16], xs[16];
+      if (owner && (site == SITE_O || site == SITE_DOWN)) {   // residual rows: issue the loads before anything else
+        const int f = tile * kTileN + fl;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) xs[i] = (c0 + i < R) ? __ldcg(w.X + (size_t)(c0 + i) * dm.d + f) : 0.f;
+      }
+      {
+        float lo[16];
+        tc_ld16(taddr + c0, v);
+        tc_ld16(taddr + Rp + c0, lo);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] += lo[i];
+      }
+      if (!owner) {
+        float* dst = p.pbuf + ((size_t)c * Rp + c0) * kTileN + fl;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) dst[(size_t)i * kTileN] = v[i];
+        continue;
+      }
+      for (int cb = c + 1; cb <= c_last; cb += 4) {   // four contributors' loads in flight at a time, added in block order
+        float pv[4][16];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int c2 = cb + k;
+          const bool live = c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G;
+          const float* src = p.pbuf + ((size_t)(live ? c2 : c) * Rp + c0) * kTileN + fl;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) pv[k][i] = live ? __ldcg(src + (size_t)i * kTileN) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] += pv[k][i];
+      }
+      if (site == SITE_QKV) {
+        const int half = HD / 2;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int r = c0 + i;
+          v[i] = v[i] * (r < R ? ctl->inv[r] : 0.f) + bias;
+        }
+        if (kind < 2) {
+          const int ii = dim & (half - 1);
+          float2 cs[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) cs[i] = (c0 + i < R) ? __ldcg(w.rope + (size_t)(c0 + i) * half + ii) : make_float2(1.f, 0.f);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) ctl->u.exch[fl][i] = v[i];
+          bar_sync(2, 128);
+          const bool first = dim < half;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float xp = ctl->u.exch[fl ^ half][i];
+            v[i] = first ? v[i] * cs[i].x - xp * cs[i].y : v[i] * cs[i].x + xp * cs[i].y;
+          }
+          bar_sync(2, 128);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int r = c0 + i;
+          if (r < R) {
+            if (kind == 0) {
+              const int group = dm.Hq / dm.Hkv;
+              bf16* qb = w.Qb + ((((size_t)ctl->row_b[r] * dm.Hkv + head / group) * group + head % group) * rows +
+                                 ctl->row_j[r]) * HD;
+              qb[dim] = __float2bfloat16_rn(v[i] * qscale);
+            } else {
+              bf16* row = kv_row<bf16>(kv, l, ctl->row_page[r], kind - 1, head, ctl->row_slot[r]);
+              row[dim] = __float2bfloat16_rn(v[i]);
+            }
+          }
+        }
+      } else if (site == SITE_O || site == SITE_DOWN) {
+        const int f = tile * kTileN + fl;
+        const float gn = __bfloat162float(gain[f]);
+        const int buf = (site == SITE_O) ? 1 : 0;
+        float ss[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int r = c0 + i;
+          ss[i] = 0.f;
+          if (r < R) {
+            const float x = xs[i] + v[i];
+            w.X[(size_t)r * dm.d + f] = x;
+            store_act<bf16>(w.A, R, dm.d, r, f, x * gn);
+            ss[i] = x * x;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) ss[i] = warp_sum(ss[i]);
+        if (lane == 0) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) ctl->red[quarter][i] = ss[i];
+        }
+        bar_sync(2, 128);
+        if (et < 16 && c0 + et < R)
+          p.sumsq[((size_t)buf * nt128 + tile) * kMegaMaxRows + c0 + et] =
+              ctl->red[0][et] + ctl->red[1][et] + ctl->red[2][et] + ctl->red[3][et];
+        bar_sync(2, 128);
+      } else if (site == SITE_GU) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int r = c0 + i;
+          v[i] *= (r < R ? ctl->inv[r] : 0.f);
+        }
+        if (fl >= 64) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) ctl->u.exch[fl - 64][i] = v[i];
+        }
+        bar_sync(2, 128);
+        if (fl < 64) {
+          const int f = tile * 64 + fl;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int r = c0 + i;
+            if (r < R) {
+              const float g = v[i], up = ctl->u.exch[fl][i];
+              store_act<bf16>(w.H, R, dm.F, r, f, g / (1.0f + expf(-g)) * up);
+            }
+          }
+        }
+        bar_sync(2, 128);
+      } else {   // LM head
+        const int n = tile * kTileN + fl;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int r = c0 + i;
+          float z = -INFINITY;
+          if (r < R && n < dm.V) {
+            const float raw = v[i] * ctl->inv[r];
+            if (w.logits) w.logits[(size_t)r * dm.V + n] = raw;
+            if (dbg_logits) dbg_logits[(size_t)r * dm.V + n] = raw;
+            z = raw * invT;
+            if (n == ctl->tgt_tok[r]) w.tgt_logit[r] = z;
+          }
+          float m = z;
+          int arg = n;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, m, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+            if (om > m || (om == m && oa < arg)) { m = om; arg = oa; }
+          }
+          float e = (z == -INFINITY) ? 0.f : expf(z - m);
+          e = warp_sum(e);
+          if (lane == 0) {
+            RowStat st; st.m = m; st.s = e; st.arg = arg; st.pad = 0;
+            ctl->wstat[quarter][i] = st;
+          }
+        }
+        bar_sync(2, 128);
+        if (et < 16 && c0 + et < R) {
+          RowStat a = ctl->wstat[0][et];
+          a = stat_merge(a, ctl->wstat[1][et]);
+          a = stat_merge(a, ctl->wstat[2][et]);
+          a = stat_merge(a, ctl->wstat[3][et]);
+          w.stats[(size_t)tile * R + c0 + et] = a;
+        }
+        bar_sync(2, 128);
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+    if (!owner) {   // publish the partial: block barrier, then one cumulative fence and the flag
+      bar_sync(2, 128);
+      if (et == 0) {
+        __threadfence();
+        st_relaxed_s32(p.flags + c, gseq);
+      }
+    }
+    u += len;
+    ++seg;
+  }
+  if (et == 0) MEGA_EV(sidx, 6);
+}
+
+// a1 + first a2: embedding gather, fp32 residual stream, first GEMM input planes, sums of squares, and
+// this step's rotary table.  All 256 workers.
+__device__ __forceinline__ void mega_embed(MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args,
+                                           const KvView& kv, const Work& w, const Dims& dm, int wt) {
+  const int ww = wt >> 5, lane = wt & 31, R = p.R, nt = dm.d / kTileN, gamma = p.rows - 1;
+  for (int item = blockIdx.x * 8 + ww; item < R * nt; item += gridDim.x * 8) {
+    const int r = item / nt, tile = item % nt, b = ctl->row_b[r], j = ctl->row_j[r];
+    const int seq = args->seq_ids[b];
+    int tok = (j == 0) ? kv.pending[seq] : args->draft_ids[b * gamma + j - 1];
+    tok = min(max(tok, 0), dm.V - 1);
+    const int f = tile * kTileN + lane * 4;
+    const uint2 raw = *reinterpret_cast<const uint2*>(p.embed + (size_t)tok * dm.d + f);
+    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+    const float2 a = __bfloat1622float2(h2[0]), c2 = __bfloat1622float2(h2[1]);
+    const float x[4] = {a.x, a.y, c2.x, c2.y};
+    *reinterpret_cast<float4*>(w.X + (size_t)r * dm.d + f) = make_float4(x[0], x[1], x[2], x[3]);
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      store_act<bf16>(w.A, R, dm.d, r, f + i, x[i] * __bfloat162float(p.gain0[f + i]));
+      ss += x[i] * x[i];
+    }
+    ss = warp_sum(ss);
+    if (lane == 0) p.sumsq[(size_t)tile * kMegaMaxRows + r] = ss;
+  }
+  const int half = dm.hd / 2;
+  for (int idx = blockIdx.x * kMegaWorkers + wt; idx < R * half; idx += gridDim.x * kMegaWorkers) {
+    const int r = idx / half, i = idx % half;
+    const int pos = ctl->plan.L[ctl->row_b[r]] + ctl->row_j[r];
+    double s, c;
+    sincos((double)pos * w.inv_freq[i], &s, &c);
+    w.rope[idx] = make_float2((float)c, (float)s);
+  }
+}
+
+// a10 tail + a11..a15 for sequence b = blockIdx.x (256 workers, named barrier 1).
+__device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args,
+                                              const KvView& kv, const Work& w, const Dims& dm, int wt) {
+  const int b = blockIdx.x, gamma = p.rows - 1, rows = p.rows, R = p.R;
+  const int lane = wt & 31, warp = wt >> 5, nwarp = kMegaWorkers >> 5;
+  const int seq = args->seq_ids[b];
+  const int n_vtiles = (dm.V + kTileN - 1) / kTileN, nt128 = dm.d / kTileN;
+  const bf16* gainF = p.lp[p.l1 - 1].gain_next;
+  for (int j = 0; j < rows; ++j) {
+    const int r = b * rows + j;
+    RowStat a; a.m = -INFINITY; a.s = 0.f; a.arg = 0; a.pad = 0;
+    const int per = (n_vtiles + kMegaWorkers - 1) / kMegaWorkers;
+    const int t0 = wt * per, t1 = min(t0 + per, n_vtiles);
+    for (int t = t0; t < t1; ++t) {
+      RowStat x;
+      const float4 raw = __ldcg(reinterpret_cast<const float4*>(w.stats + (size_t)t * R + r));
+      x.m = raw.x; x.s = raw.y; x.arg = __float_as_int(raw.z); x.pad = 0;
+      a = stat_merge(a, x);
+    }
+    ctl->u.sred[wt] = a;
+    bar_sync(1, kMegaWorkers);
+    for (int stride = 1; stride < kMegaWorkers; stride <<= 1) {
+      if ((wt % (2 * stride)) == 0 && wt + stride < kMegaWorkers)
+        ctl->u.sred[wt] = stat_merge(ctl->u.sred[wt], ctl->u.sred[wt + stride]);
+      bar_sync(1, kMegaWorkers);
+    }
+    if (wt == 0) { ctl->rs[j] = ctl->u.sred[0]; w.rowstat[r] = ctl->u.sred[0]; }
+    bar_sync(1, kMegaWorkers);
+  }
+  // 1/rms of the final norm for this sequence's rows
+  if (wt < rows) {
+    float s = 0.f;
+    for (int t = 0; t < nt128; ++t) s += __ldcg(p.sumsq + (size_t)t * kMegaMaxRows + b * rows + wt);
+    ctl->inv[b * rows + wt] = 1.0f / sqrtf(s / (float)dm.d + dm.eps);
+  }
+  bar_sync(1, kMegaWorkers);
+  if (args->dbg_hidden) {
+    for (int idx = wt; idx < rows * dm.d; idx += kMegaWorkers) {
+      const int r = b * rows + idx / dm.d, i = idx % dm.d;
+      args->dbg_hidden[(size_t)r * dm.d + i] = __ldcg(w.X + (size_t)r * dm.d + i) * __bfloat162float(gainF[i]) * ctl->inv[r];
+    }
+  }
+  for (int j = 1 + warp; j <= gamma; j += nwarp) {
+    const int r = b * rows + j;
+    float a = 0.f;
+    if (args->has_judge)
+      for (int i = lane; i < dm.d; i += 32)
+        a = fmaf(__ldcg(w.X + (size_t)r * dm.d + i) * __bfloat162float(gainF[i]) * ctl->inv[r], w.judge_w[i], a);
+    a = warp_sum(a);
+    if (lane == 0) {
+      const float s = args->has_judge ? 1.0f / (1.0f + expf(-(a + args->judge_bias))) : 0.f;
+      ctl->score[j] = s;
+      args->judge_scores[b * gamma + j - 1] = s;
+    }
+  }
+  bar_sync(1, kMegaWorkers);
+  if (warp == 0) {
+    bool ok = true;
+    if (lane < gamma) {
+      const int j = lane + 1;
+      const int d = args->draft_ids[b * gamma + lane];
+      const RowStat st = ctl->rs[j - 1];
+      const float pr = expf(__ldcg(w.tgt_logit + b * rows + j - 1) - st.m) / st.s;
+      args->p_draft[b * gamma + lane] = pr;
+      bool align;
+      if (args->mode == 0) align = (d == st.arg);
+      else align = args->uniforms[b * rows + lane] * args->q_tok[b * gamma + lane] < pr;
+      const bool judge = args->has_judge && (ctl->score[j] > args->theta);
+      ok = (args->use_align && align) || (args->use_judge && judge);
+    }
+    const unsigned rej = __ballot_sync(0xffffffffu, !ok);
+    const int n = rej ? (__ffs(rej) - 1) : gamma;
+    if (lane == 0) {
+      const int L = ctl->plan.L[b];
+      args->accepted_len[b] = n;
+      args->new_kv_len[b] = L + 1 + n;
+      if (args->mode == 0) {
+        const int nxt = ctl->rs[n].arg;
+        args->next_token[b] = nxt;
+        if (args->commit) kv.pending[seq] = nxt;
+      }
+      if (args->commit) kv.kv_len[seq] = L + 1 + n;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// the kernel
+// ---------------------------------------------------------------------------------------------
+template <int HD>
+__global__ void __launch_bounds__(kMegaThreads, 1)
+k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const StepArgs* __restrict__ args, const KvView kv,
+              const Work w, const Dims dm) {
+  extern __shared__ uint8_t mega_smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(mega_smem_raw) + 1023) & ~(uintptr_t)1023);
+  MegaCtl* ctl = reinterpret_cast<MegaCtl*>(ring + (size_t)p.stages * p.stage_bytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int c = blockIdx.x, G = gridDim.x, NS = p.stages, B = p.B, R = p.R, Rp = p.Rp, rows = p.rows;
+  const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(smem_u32(&ctl->full[i]), 2);
+      mbar_init(smem_u32(&ctl->empty[i]), 1);
+      ctl->cons_cnt[i] = 0;
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
+      mbar_init(smem_u32(&ctl->tmem_empty[i]), 128);
+    }
+    ctl->abort_flag = 0;
+    ctl->bars_passed = 0;
+    int acc = 0;
+    for (int b = 0; b < B; ++b) {
+      const int L = kv.kv_len[args->seq_ids[b]];
+      ctl->plan.L[b] = L;
+      ctl->plan.pre[b] = acc;
+      acc += dm.Hkv * ((L + g.KPS - 1) / g.KPS);
+    }
+    ctl->plan.pre[B] = acc;
+    ctl->plan.T = acc;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                 "r"(p.tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (threadIdx.x < R) {
+    const int r = threadIdx.x, b = r / rows, j = r % rows, gamma = rows - 1;
+    const int pos = ctl->plan.L[b] + j;
+    ctl->row_b[r] = b;
+    ctl->row_j[r] = j;
+    ctl->row_page[r] = kv.block_table[(size_t)args->seq_ids[b] * kv.max_pages_per_seq + pos / kv.page_size];
+    ctl->row_slot[r] = pos % kv.page_size;
+    ctl->tgt_tok[r] = (j < gamma) ? args->draft_ids[b * gamma + j] : -1;
+  }
+  __syncthreads();
+
+  const AttPlan& pl = ctl->plan;
+  const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
+  const int n_att = (int)(t_hi - t_lo);
+  auto stage_addr = [&](int s) -> uint32_t { return smem_u32(ring + (size_t)s * p.stage_bytes); };
+
+  if (warp == 0) {
+    // ------------------------------ weight / cache-tile producer ------------------------------
+    if (lane == 0) {
+      const uint64_t pol_w = l2_policy_evict_first();
+      int it = 0, sidx = 0;
+      bool alive = true;
+      auto wait_slot = [&](int i) -> bool {
+        return i < NS || mega_wait(smem_u32(&ctl->empty[i % NS]), (uint32_t)((i / NS) - 1) & 1u, ctl, p, w.status, 1, i);
+      };
+      auto fsite = [&](int site, int l) {
+        if (!alive) return;
+        const SiteInfo si = site_info(site, dm, c, G);
+        for (long long u = si.u_lo; u < si.u_hi; ++u, ++it) {
+          if (!wait_slot(it)) { alive = false; return; }
+          const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+          mbar_expect_tx(bar, kWTileBytes);
+          mega_issue_w(mp, site, l - p.l0, dm, u, si.KB, stage_addr(it % NS), bar, pol_w);
+        }
+        MEGA_EV(sidx, 7);
+        ++sidx;
+      };
+      auto fatt = [&](int l) {
+        if (!alive) return;
+        for (long long t = t_lo; t < t_hi; ++t, ++it) {
+          if (!wait_slot(it)) { alive = false; return; }
+          const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+          mbar_expect_tx(bar, kAttStageBytes);
+          mbar_arrive(bar);   // stands in for the activation producer, which skips cache tiles
+          const AttTile x = att_locate(pl, B, g.KPS, (int)t);
+          att_issue_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD, stage_addr(it % NS), bar);
+        }
+      };
+      mega_walk(p, fsite, fatt);
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(2 * Rp);
+      const uint32_t tmem_base = ctl->tmem_base;
+      int it = 0, seg = 0, sidx = 0;
+      bool alive = true;
+      auto fsite = [&](int site, int l) {
+        if (!alive) return;
+        const SiteInfo si = site_info(site, dm, c, G);
+        bool first = true;
+        long long u = si.u_lo;
+        while (u < si.u_hi) {
+          const int kb0 = (int)(u % si.KB);
+          const int len = (int)min((long long)(si.KB - kb0), si.u_hi - u);
+          const int acc = seg & 1, use = seg >> 1;
+          if (use > 0 && !mega_wait(smem_u32(&ctl->tmem_empty[acc]), (uint32_t)(use - 1) & 1u, ctl, p, w.status, 4, seg)) {
+            alive = false;
+            return;
+          }
+          tc_fence_after();
+          for (int i = 0; i < len; ++i, ++it) {
+            const int s = it % NS;
+            if (!mega_wait(smem_u32(&ctl->full[s]), (uint32_t)(it / NS) & 1u, ctl, p, w.status, 5, it)) { alive = false; return; }
+            tc_fence_after();
+            if (first) { MEGA_EV(sidx, 2); first = false; }
+            const uint32_t wa = stage_addr(s);
+            const uint64_t dw = smem_desc_sw128(wa), da = smem_desc_sw128(wa + kWTileBytes);
+            const uint32_t dcol = tmem_base + (uint32_t)(acc * 2 * Rp);
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k) tc_mma_bf16(dcol, dw + 2 * k, da + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            tc_commit(smem_u32(&ctl->empty[s]));
+          }
+          tc_commit(smem_u32(&ctl->tmem_full[acc]));
+          u += len;
+          ++seg;
+        }
+        MEGA_EV(sidx, 3);
+        ++sidx;
+      };
+      auto fatt = [&](int l) { it += n_att; };
+      mega_walk(p, fsite, fatt);
+    }
+  } else if (warp == 2) {
+    // ------------------------------ activation producer ------------------------------
+    if (lane == 0) {
+      const uint64_t pol_a = l2_policy_evict_last();
+      const uint32_t a_tx = (uint32_t)(2 * Rp) * 128u;
+      int it = 0, nb = p.do_embed ? 1 : 0, sidx = 0;
+      bool alive = true;
+      auto fsite = [&](int site, int l) {
+        if (!alive) return;
+        const SiteInfo si = site_info(site, dm, c, G);
+        if (si.u_hi > si.u_lo) {
+          // inputs of this phase are complete once `nb` device-wide barriers have been passed
+          volatile int* bp = &ctl->bars_passed;
+          volatile int* af = &ctl->abort_flag;
+          uint32_t i = 0;
+          while (*bp < nb) {
+            if (*af || ++i > kMegaSpin) { alive = false; break; }
+            if (i > 64) __nanosleep(32);
+          }
+          if (i > kMegaSpin) { ctl->abort_flag = 1; att_note_timeout(p.abort_g, 3, nb); *p.abort_g = 1; atomicCAS(w.status, DEV_OK, DEV_TIMEOUT); }
+          if (!alive) return;
+          __threadfence();
+          fence_proxy_async();
+          MEGA_EV(sidx, 0);
+          const CUtensorMap* tm = (site == SITE_O) ? &mp.a_q : (site == SITE_DOWN ? &mp.a_f : &mp.a_d);
+          for (long long u = si.u_lo; u < si.u_hi; ++u, ++it) {
+            if (it >= NS && !mega_wait(smem_u32(&ctl->empty[it % NS]), (uint32_t)((it / NS) - 1) & 1u, ctl, p, w.status, 2, it)) {
+              alive = false;
+              return;
+            }
+            const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+            mbar_expect_tx(bar, a_tx);
+            tma_load_2d(stage_addr(it % NS) + kWTileBytes, tm, bar, (int)(u % si.KB) * kBK, 0, pol_a);
+          }
+          MEGA_EV(sidx, 1);
+        }
+        ++sidx;
+        nb += (site == SITE_QKV) ? 3 : 1;
+      };
+      auto fatt = [&](int l) { it += n_att; };
+      mega_walk(p, fsite, fatt);
+    }
+  } else if (warp >= 4) {
+    // ------------------------------ workers ------------------------------
+    const int wt = threadIdx.x - 128, ww = wt >> 5;
+    int nbar = 0, gseq = 0, seg = 0, it = 0;
+    bool alive = true;
+    if (p.do_embed) {
+      mega_embed(ctl, p, args, kv, w, dm, wt);
+      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+    }
+    auto units = [&](int site) -> int {
+      const SiteInfo si = site_info(site, dm, c, G);
+      return (int)(si.u_hi - si.u_lo);
+    };
+    auto gemm_phase = [&](int site, int l) {
+      ++gseq;
+      if (alive && ww < 4) mega_epilogue<HD>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
+      it += units(site);
+      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+    };
+    for (int l = p.l0; l < p.l1; ++l) {
+      gemm_phase(SITE_QKV, l);
+      if (alive && ww < g.MT * g.KS) {
+        AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status};
+        AttArgs aa{w.Qb, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
+        int it2 = it;
+        att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
+      }
+      it += n_att;
+      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+      if (alive) {
+        const AttPartials P{w.tc_m, w.tc_l, w.tc_o};
+        const int items = B * dm.Hkv * g.nq;
+        for (int item = c * 8 + ww; item < items; item += G * 8)
+          att_combine_item<bf16, HD>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane);
+      }
+      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+      gemm_phase(SITE_O, l);
+      gemm_phase(SITE_GU, l);
+      gemm_phase(SITE_DOWN, l);
+    }
+    if (p.do_lm) {
+      gemm_phase(SITE_LM, p.l1 - 1);
+      if (alive && c < B) mega_finalize(ctl, p, args, kv, w, dm, wt);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    if (*reinterpret_cast<volatile int*>(&ctl->abort_flag)) __nanosleep(20000);   // let copies in flight land
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(ctl->tmem_base), "r"(p.tmem_cols) : "memory");
+  }
+}
+
+}  // namespace sj

@@ -66,8 +66,10 @@ CFG1_VARIANTS = [
     ("f32", torch.float32, {}),
     ("f32-nograph-nopdl", torch.float32, {"graph": 0, "pdl": 0}),
     ("bf16-cudacore", torch.bfloat16, {"gemm_impl": 0}),
-    ("bf16-tcgen05", torch.bfloat16, {"gemm_impl": 1}),
-    ("bf16-tcgen05-nograph", torch.bfloat16, {"gemm_impl": 1, "graph": 0, "pdl": 0}),
+    ("bf16-persistent", torch.bfloat16, {"gemm_impl": 1, "step_impl": 1}),
+    ("bf16-tcgen05", torch.bfloat16, {"gemm_impl": 1, "step_impl": 0}),
+    ("bf16-tcgen05-simt-attn", torch.bfloat16, {"gemm_impl": 1, "step_impl": 0, "attn_impl": 0}),
+    ("bf16-tcgen05-nograph", torch.bfloat16, {"gemm_impl": 1, "step_impl": 0, "graph": 0, "pdl": 0}),
 ]
 
 
@@ -88,7 +90,9 @@ def test_config1_tiny_target(name, dtype, options):
 
 
 @pytest.mark.parametrize("dtype,options", [(torch.float32, {}), (torch.bfloat16, {"gemm_impl": 0}),
-                                            (torch.bfloat16, {"gemm_impl": 1})], ids=["f32", "bf16-cudacore", "bf16-tcgen05"])
+                                            (torch.bfloat16, {"gemm_impl": 1, "step_impl": 0}),
+                                            (torch.bfloat16, {"gemm_impl": 1, "step_impl": 1})],
+                         ids=["f32", "bf16-cudacore", "bf16-tcgen05", "bf16-persistent"])
 @pytest.mark.parametrize("kv_lens,gamma", [([5, 37, 130], 3), ([15, 16, 17, 0], 5), ([200], 1), ([63, 64], 16)])
 def test_ragged_batches_and_page_edges(dtype, options, kv_lens, gamma):
     case = harness.Case(GQA, dtype, kv_lens, gamma, seed=3).gpu_setup()
@@ -100,7 +104,8 @@ def test_ragged_batches_and_page_edges(dtype, options, kv_lens, gamma):
         case.close()
 
 
-@pytest.mark.parametrize("options", [{"gemm_impl": 0}, {"gemm_impl": 1}], ids=["cudacore", "tcgen05"])
+@pytest.mark.parametrize("options", [{"gemm_impl": 0}, {"gemm_impl": 1, "step_impl": 0}, {"gemm_impl": 1, "step_impl": 1}],
+                         ids=["cudacore", "tcgen05", "persistent"])
 def test_head_dim_128_with_qkv_bias(options):
     case = harness.Case(GQA128, torch.bfloat16, [70, 300], 8, seed=4).gpu_setup()
     try:
