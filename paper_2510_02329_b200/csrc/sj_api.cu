@@ -190,7 +190,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_l2_ahead = 0;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -508,8 +508,14 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "step_impl must be 0 or 1");
     if (value == 1 && !t->mega_shapes) return fail(SJ_ERR_UNSUPPORTED, "the whole-step kernel needs bf16, 128-multiples and cooperative launch");
     t->opt_step = value;
+  } else if (n == "ring_stages") {
+    if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
+    t->opt_ring = value;
+  } else if (n == "l2_ahead") {
+    if (value < 0 || value > 4096) return fail(SJ_ERR_INVALID_ARG, "l2_ahead must be in [0, 4096]");
+    t->opt_l2_ahead = value;
   } else if (n == "trace") {
-    const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 8 * kMegaTraceSites;
+    const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 16 * kMegaTraceSites;
     if (value && !t->d_trace) {
       sj_status st = dev_alloc(t, &t->d_trace, n_tr);
       if (st != SJ_OK) return st;
@@ -950,6 +956,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   const int budget = 227 * 1024 - 1024 - (int)sizeof(MegaCtl);
   p.stages = std::min(kMegaMaxStages, budget / p.stage_bytes);
   if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
+  if (t->opt_ring) p.stages = std::min(p.stages, t->opt_ring);
   uint32_t tc = 32;
   while (tc < (uint32_t)(4 * Rp)) tc <<= 1;
   p.tmem_cols = tc;
@@ -963,6 +970,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.flags = reinterpret_cast<int*>(t->d_sync + 16);
   p.n_tail_base = t->sm_count + B * dm.Hkv;
   p.trace = t->opt_trace ? t->d_trace : nullptr;
+  p.l2_ahead = t->opt_l2_ahead;
   const size_t smem = (size_t)p.stages * p.stage_bytes + sizeof(MegaCtl) + 1024;
   const bool timing = t->opt_timing != 0;
   const int NL = dm.n_layers;
@@ -1008,7 +1016,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
 extern "C" sj_status sj_step_trace(sj_target* t, unsigned long long* out_ns, int max_entries, int* n_entries) {
   if (!t || !out_ns || !n_entries || max_entries <= 0) return fail(SJ_ERR_INVALID_ARG, "null argument");
   if (!t->d_trace) return fail(SJ_ERR_STATE, "tracing was never enabled (sj_set_option \"trace\")");
-  const int n = std::min(max_entries, 2 * kMegaTraceBarriers + 8 * kMegaTraceSites);
+  const int n = std::min(max_entries, 2 * kMegaTraceBarriers + 16 * kMegaTraceSites);
   CU_TRY(cudaStreamSynchronize(t->stream));
   CU_TRY(cudaMemcpy(out_ns, t->d_trace, sizeof(unsigned long long) * n, cudaMemcpyDeviceToHost));
   *n_entries = n;

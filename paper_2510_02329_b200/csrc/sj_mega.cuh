@@ -13,6 +13,7 @@
 //   warp 0      weight / cache-tile producer (TMA into the ring)
 //   warp 1      tcgen05.mma issuer, owns the TMEM allocation
 //   warp 2      activation producer: TMA of the activation K-slices, gated by the device-wide barrier
+//   warp 3      L2 prefetcher: requests the producer's upcoming boxes into L2 beyond the ring
 //   warps 4..11 workers: the first four drain TMEM (fused epilogues), all eight run attention, the
 //               combine, the embedding and the final acceptance phase
 //
@@ -75,6 +76,7 @@ struct MegaParams {
   int* abort_g;               // device-wide abort word        }
   int* flags;                 // [blocks] split-K flags        }
   int n_tail_base;
+  int l2_ahead;               // units beyond the ring that the producer keeps requested into L2 (0: none)
   // optional timeline of block 0 (global-timer nanoseconds):
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
   //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
@@ -94,12 +96,21 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
       p.trace[2 * kMegaTraceBarriers + (sidx) * 8 + (k)] = global_timer_ns();                        \
   } while (0)
 
+// second event set (fine-grained epilogue timing): block 1 records its contributor-side events, block 0 its
+// owner-side ones, at [2*kMegaTraceBarriers + 8*kMegaTraceSites + 8*s + e]
+#define MEGA_EV2(blk, sidx, k)                                                                       \
+  do {                                                                                               \
+    if (p.trace && blockIdx.x == (blk) && (sidx) < kMegaTraceSites)                                  \
+      p.trace[2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (sidx) * 8 + (k)] = global_timer_ns();  \
+  } while (0)
+
 struct MegaCtl {
   uint64_t full[kMegaMaxStages], empty[kMegaMaxStages], tmem_full[2], tmem_empty[2];
   int cons_cnt[kMegaMaxStages];
   uint32_t tmem_base;
   int abort_flag;
   int bars_passed;
+  int w_issued;            // units the weight producer has issued so far (read by the L2 prefetcher)
   int bcast[4];
   float inv[kMegaMaxRows];
   int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
@@ -220,6 +231,22 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
   return *reinterpret_cast<volatile int*>(&ctl->abort_flag) == 0;
 }
 
+// Bounded wait (shared-memory polling) until the block's workers have passed `need` device-wide barriers.
+__device__ __forceinline__ bool mega_wait_bars(int need, MegaCtl* ctl, const MegaParams& p, int* status, int where) {
+  volatile int* bp = &ctl->bars_passed;
+  volatile int* af = &ctl->abort_flag;
+  for (uint32_t i = 0; i < kMegaSpin; ++i) {
+    if (*bp >= need) return true;
+    if (*af) return false;
+    if (i > 64) __nanosleep(32);
+  }
+  ctl->abort_flag = 1;
+  att_note_timeout(p.abort_g, where, need);
+  *p.abort_g = 1;
+  atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+  return false;
+}
+
 // TMA loads of one weight unit into a ring stage.
 __device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int li, const Dims& dm, long long u, int KB,
                                              uint32_t dst, uint32_t bar, uint64_t pol) {
@@ -239,6 +266,48 @@ __device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int l
       break;
     case SITE_DOWN: tma_load_2d(dst, &mp.wd[li], bar, kb * kBK, tile * kTileN, pol); break;
     default: tma_load_2d(dst, &mp.lm, bar, kb * kBK, tile * kTileN, pol); break;
+  }
+}
+
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tm, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(c0),
+               "r"(c1)
+               : "memory");
+}
+// L2 prefetch of one weight unit (same boxes as mega_issue_w).
+__device__ __forceinline__ void mega_prefetch_w(const MegaMaps& mp, int site, int li, const Dims& dm, long long u, int KB) {
+  const int tile = (int)(u / KB), kb = (int)(u % KB);
+  switch (site) {
+    case SITE_QKV: {
+      const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
+      if (tile < tq) tma_prefetch_2d(&mp.wq[li], kb * kBK, tile * kTileN);
+      else if (tile < tq + tk) tma_prefetch_2d(&mp.wk[li], kb * kBK, (tile - tq) * kTileN);
+      else tma_prefetch_2d(&mp.wv[li], kb * kBK, (tile - tq - tk) * kTileN);
+      break;
+    }
+    case SITE_O: tma_prefetch_2d(&mp.wo[li], kb * kBK, tile * kTileN); break;
+    case SITE_GU:
+      tma_prefetch_2d(&mp.wg[li], kb * kBK, tile * 64);
+      tma_prefetch_2d(&mp.wu[li], kb * kBK, tile * 64);
+      break;
+    case SITE_DOWN: tma_prefetch_2d(&mp.wd[li], kb * kBK, tile * kTileN); break;
+    default: tma_prefetch_2d(&mp.lm, kb * kBK, tile * kTileN); break;
+  }
+}
+// L2 prefetch of one cache tile (same boxes as att_issue_tile).
+__device__ __forceinline__ void mega_prefetch_tile(const CUtensorMap* tmKV, const KvView& kv, int layer, int seq, int h, int ti,
+                                                   int L, int KPS, int HD) {
+  const int HB = HD / 64, npg = KPS / 16, last_page = (L - 1) / 16;
+  for (int pg = 0; pg < npg; ++pg) {
+    const int pi = ti * npg + pg;
+    if (pi > last_page) break;
+    const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+    const long long rowK = ((((long long)layer * kv.n_pages + page) * 2 + 0) * kv.n_kv_heads + h) * 16;
+    const long long rowV = rowK + (long long)kv.n_kv_heads * 16;
+    for (int half = 0; half < HB; ++half) {
+      tma_prefetch_2d(tmKV, half * 64, (int)rowK);
+      tma_prefetch_2d(tmKV, half * 64, (int)rowV);
+    }
   }
 }
 
@@ -294,6 +363,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     if (!ctl->bcast[seg & 1]) return;
     tc_fence_after();
     if (et == 0) MEGA_EV(sidx, 4);
+    if (et == 0 && kb0 != 0) MEGA_EV2(1, sidx, 0);
     const bool owner = (kb0 == 0), complete = owner && (len == si.KB);
     int c_last = c;
     if (owner && !complete) {
@@ -371,6 +441,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] += pv[k][i];
       }
+      if (et == 0) MEGA_EV2(0, sidx, 5);
       if (site == SITE_QKV) {
         const int half = HD / 2;
 #pragma unroll
@@ -498,12 +569,16 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         bar_sync(2, 128);
       }
     }
+    if (et == 0) MEGA_EV2(0, sidx, 7);
     tc_fence_before();
     mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
     if (!owner) {   // publish the partial: block barrier, then one cumulative fence and the flag
+      if (et == 0) MEGA_EV2(1, sidx, 1);
       bar_sync(2, 128);
       if (et == 0) {
+        MEGA_EV2(1, sidx, 2);
         __threadfence();
+        MEGA_EV2(1, sidx, 3);
         st_relaxed_s32(p.flags + c, gseq);
       }
     }
@@ -660,6 +735,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     }
     ctl->abort_flag = 0;
     ctl->bars_passed = 0;
+    ctl->w_issued = 0;
     int acc = 0;
     for (int b = 0; b < B; ++b) {
       const int L = kv.kv_len[args->seq_ids[b]];
@@ -702,6 +778,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       const uint64_t pol_w = l2_policy_evict_first();
       int it = 0, sidx = 0;
       bool alive = true;
+      volatile int* w_issued = &ctl->w_issued;
       auto wait_slot = [&](int i) -> bool {
         return i < NS || mega_wait(smem_u32(&ctl->empty[i % NS]), (uint32_t)((i / NS) - 1) & 1u, ctl, p, w.status, 1, i);
       };
@@ -713,6 +790,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           const uint32_t bar = smem_u32(&ctl->full[it % NS]);
           mbar_expect_tx(bar, kWTileBytes);
           mega_issue_w(mp, site, l - p.l0, dm, u, si.KB, stage_addr(it % NS), bar, pol_w);
+          *w_issued = it + 1;
         }
         MEGA_EV(sidx, 7);
         ++sidx;
@@ -726,7 +804,43 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           mbar_arrive(bar);   // stands in for the activation producer, which skips cache tiles
           const AttTile x = att_locate(pl, B, g.KPS, (int)t);
           att_issue_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD, stage_addr(it % NS), bar);
+          *w_issued = it + 1;
         }
+      };
+      mega_walk(p, fsite, fatt);
+    }
+  } else if (warp == 3) {
+    // ------------------------------ L2 prefetcher ------------------------------
+    // Walks the same unit sequence ahead of the producer and requests the boxes into L2 only, so that HBM
+    // keeps streaming while every block waits at a barrier with a full ring; the real loads then hit L2.
+    // It stays at most l2_ahead units ahead of the producer's issue point.
+    if (lane == 0 && p.l2_ahead > 0) {
+      volatile int* w_issued = &ctl->w_issued;
+      volatile int* af = &ctl->abort_flag;
+      const int D = p.l2_ahead;
+      int pf = 0;
+      bool alive = true;
+      auto gate = [&]() -> bool {   // true: prefetch unit pf; false: skip it (the real load is imminent)
+        uint32_t i = 0;
+        while (pf >= *w_issued + D) {
+          if (*af || ++i > kMegaSpin) { alive = false; return false; }
+          __nanosleep(100);
+        }
+        return pf >= *w_issued + 2;
+      };
+      auto fsite = [&](int site, int l) {
+        if (!alive) return;
+        const SiteInfo si = site_info(site, dm, c, G);
+        for (long long u = si.u_lo; u < si.u_hi && alive; ++u, ++pf)
+          if (gate()) mega_prefetch_w(mp, site, l - p.l0, dm, u, si.KB);
+      };
+      auto fatt = [&](int l) {
+        if (!alive) return;
+        for (long long t = t_lo; t < t_hi && alive; ++t, ++pf)
+          if (gate()) {
+            const AttTile x = att_locate(pl, B, g.KPS, (int)t);
+            mega_prefetch_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD);
+          }
       };
       mega_walk(p, fsite, fatt);
     }
@@ -735,13 +849,18 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(2 * Rp);
       const uint32_t tmem_base = ctl->tmem_base;
-      int it = 0, seg = 0, sidx = 0;
+      int it = 0, seg = 0, sidx = 0, nb = p.do_embed ? 1 : 0;
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
         const SiteInfo si = site_info(site, dm, c, G);
         bool first = true;
         long long u = si.u_lo;
+        // Do not look at this phase's stages before the phase has begun: the attention phase in between
+        // may reuse a stage several times, and a parity wait started two uses early would be satisfied by
+        // the wrong one.
+        if (u < si.u_hi && !mega_wait_bars(nb, ctl, p, w.status, 10)) { alive = false; return; }
+        nb += (site == SITE_QKV) ? 3 : 1;
         while (u < si.u_hi) {
           const int kb0 = (int)(u % si.KB);
           const int len = (int)min((long long)(si.KB - kb0), si.u_hi - u);
@@ -785,15 +904,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         const SiteInfo si = site_info(site, dm, c, G);
         if (si.u_hi > si.u_lo) {
           // inputs of this phase are complete once `nb` device-wide barriers have been passed
-          volatile int* bp = &ctl->bars_passed;
-          volatile int* af = &ctl->abort_flag;
-          uint32_t i = 0;
-          while (*bp < nb) {
-            if (*af || ++i > kMegaSpin) { alive = false; break; }
-            if (i > 64) __nanosleep(32);
-          }
-          if (i > kMegaSpin) { ctl->abort_flag = 1; att_note_timeout(p.abort_g, 3, nb); *p.abort_g = 1; atomicCAS(w.status, DEV_OK, DEV_TIMEOUT); }
-          if (!alive) return;
+          if (!mega_wait_bars(nb, ctl, p, w.status, 3)) { alive = false; return; }
           __threadfence();
           fence_proxy_async();
           MEGA_EV(sidx, 0);
