@@ -80,6 +80,12 @@ __host__ __device__ __forceinline__ AttGeom att_geom(int hd, int group, int rows
 
 // Which block owns ring tile t when T tiles are dealt to G blocks as [c*T/G, (c+1)*T/G).
 __device__ __forceinline__ int att_owner(long long t, long long T, int G) {
+  if (T < (1 << 22) && G < 512) {   // 32-bit arithmetic (64-bit division is slow): t*G and (c+1)*T stay below 2^31
+    const unsigned tt = (unsigned)t, TT = (unsigned)T, GG = (unsigned)G;
+    unsigned c = tt * GG / TT;
+    while ((c + 1) * TT / GG <= tt) ++c;
+    return (int)c;
+  }
   int c = (int)(t * G / T);
   while ((long long)(c + 1) * T / G <= t) ++c;
   return c;
@@ -581,8 +587,9 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     const int cc = c_first + k / g.KS, ks = k % g.KS;
     return (((size_t)cc + bh) * kAttMaxSub + ks) * g.nq + q;
   };
+  const bool all_live = pl.T >= G_att;   // every block of the attention pass owns at least one tile
   auto sub_live = [&](int k) -> bool {
-    if (k == n_sub - 1) return true;
+    if (all_live || k == n_sub - 1) return true;
     const int cc = c_first + k / g.KS;
     return (long long)(cc + 1) * pl.T / G_att > (long long)cc * pl.T / G_att;
   };

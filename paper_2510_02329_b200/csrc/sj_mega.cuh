@@ -13,7 +13,6 @@
 //   warp 0      weight / cache-tile producer (TMA into the ring)
 //   warp 1      tcgen05.mma issuer, owns the TMEM allocation
 //   warp 2      activation producer: TMA of the activation K-slices, gated by the device-wide barrier
-//   warp 3      L2 prefetcher: requests the producer's upcoming boxes into L2 beyond the ring
 //   warps 4..11 workers: the first four drain TMEM (fused epilogues), all eight run attention, the
 //               combine, the embedding and the final acceptance phase
 //
@@ -28,6 +27,14 @@
 //   gate/up (tiles interleave 64 gate and 64 up features) -> silu(g) * u -> down-projection input planes
 //   down  -> as O
 //   LM head (whole tiles) -> softmax statistics per (vocabulary tile, row), logit of the drafted token
+// The three projections with few tiles (QKV, O, down: 32..48 tiles for 148 SMs) would have every tile split
+// over 3..5 blocks that all finish at the same moment, so that the owner's wait for its contributors, through
+// L2 (about 2 us per round trip while the weight stream runs), sits on the critical path of every phase.
+// With thread-block clusters of four the stream-K deal is made over CLUSTERS for these three sites and each
+// segment's K range is cut in four inside the cluster; the three other blocks push their partial sums into
+// the first block's shared memory (distributed shared memory + a cluster-scope mbarrier), which then acts for
+// the cluster.  Across clusters a tile is shared by at most two clusters whose shares sit at opposite ends of
+// their ranges, so the contributor has published long before the owner asks.
 // Attention: see sj_attn_tc.cuh; its cache tiles travel through the same ring.
 //
 // Every wait is bounded; the first one to run out raises a device-wide abort word that all other waits
@@ -45,6 +52,8 @@ constexpr int kMegaMaxLayers = 32;   // per launch (tensor maps travel as kernel
 constexpr int kMegaMaxRows = 80;
 constexpr int kMegaMaxStages = 12;
 constexpr uint32_t kMegaSpin = 1u << 22;
+constexpr int kMegaRegsLight = 64;    // registers per thread of warps 0..3 after reallocation
+constexpr int kMegaRegsHeavy = 216;   // registers per thread of the worker warps (128*96 + 256*200 <= 384*168)
 constexpr int kMegaTraceBarriers = 1024;
 constexpr int kMegaTraceSites = 512;
 
@@ -76,7 +85,7 @@ struct MegaParams {
   int* abort_g;               // device-wide abort word        }
   int* flags;                 // [blocks] split-K flags        }
   int n_tail_base;
-  int l2_ahead;               // units beyond the ring that the producer keeps requested into L2 (0: none)
+  int cluster;                // blocks per cluster (1 or 4)
   // optional timeline of block 0 (global-timer nanoseconds):
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
   //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
@@ -87,7 +96,7 @@ struct MegaParams {
 
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
   return t;
 }
 #define MEGA_EV(sidx, k)                                                                             \
@@ -110,10 +119,13 @@ struct MegaCtl {
   uint32_t tmem_base;
   int abort_flag;
   int bars_passed;
-  int w_issued;            // units the weight producer has issued so far (read by the L2 prefetcher)
   int bcast[4];
+  uint64_t xfull;          // cluster exchange: the contributors' partial sums have landed (first block of a cluster)
+  uint64_t xfree;          // cluster exchange: the first block has consumed this block's previous partial sums
   float inv[kMegaMaxRows];
   int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
+  int row_qoff[kMegaMaxRows];         // element offset of row r's queries in the query buffer, without the head part
+  long long row_kvoff[kMegaMaxRows];  // element offset of row r's slot in its cache page, without layer / K|V / head part
   float red[4][16];
   RowStat wstat[4][16];
   RowStat rs[kMaxGamma + 1];
@@ -154,6 +166,79 @@ __device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
   int c = (int)(u * G / U);
   while ((long long)(c + 1) * U / G <= u) ++c;
   return c;
+}
+
+// How a site's units are dealt.  A "group" is a cluster for the sites whose tiles are split inside a cluster
+// (QKV, O, down when clusters are on) and a single block otherwise.  Groups take [g*U/n, (g+1)*U/n); every
+// maximal run of units of one tile inside a group's range is a segment, and block `rank` of the group takes
+// the K blocks [kb0 + rank*len/CS, kb0 + (rank+1)*len/CS) of it.
+struct SiteSplit {
+  int n_tiles, KB, CS, rank, grp, ngrp;
+  long long U, g_lo, g_hi;
+};
+__device__ __forceinline__ SiteSplit site_split(int site, const Dims& dm, int c, int G, int cluster) {
+  SiteSplit s;
+  const SiteInfo t = site_info(site, dm, 0, 1);
+  s.n_tiles = t.n_tiles;
+  s.KB = t.KB;
+  s.CS = (cluster > 1 && (site == SITE_QKV || site == SITE_O || site == SITE_DOWN)) ? cluster : 1;
+  s.ngrp = G / s.CS;
+  s.grp = c / s.CS;
+  s.rank = c % s.CS;
+  s.U = (long long)s.n_tiles * s.KB;
+  if (site == SITE_LM) {
+    s.g_lo = ((long long)s.grp * s.n_tiles / s.ngrp) * s.KB;
+    s.g_hi = ((long long)(s.grp + 1) * s.n_tiles / s.ngrp) * s.KB;
+  } else {
+    s.g_lo = (long long)s.grp * s.U / s.ngrp;
+    s.g_hi = (long long)(s.grp + 1) * s.U / s.ngrp;
+  }
+  return s;
+}
+struct Seg { int tile, kb0, len, a, b; };
+__device__ __forceinline__ bool seg_next(const SiteSplit& s, long long& u, Seg& g) {
+  if (u >= s.g_hi) return false;
+  g.tile = (int)(u / s.KB);
+  g.kb0 = (int)(u % s.KB);
+  g.len = (int)min((long long)(s.KB - g.kb0), s.g_hi - u);
+  g.a = g.kb0 + s.rank * g.len / s.CS;
+  g.b = g.kb0 + (s.rank + 1) * g.len / s.CS;
+  u += g.len;
+  return true;
+}
+__device__ __forceinline__ int site_units(const SiteSplit& s) {
+  long long u = s.g_lo;
+  Seg g;
+  int n = 0;
+  while (seg_next(s, u, g)) n += g.b - g.a;
+  return n;
+}
+
+// cluster plumbing
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t local_addr, int rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t remote_addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 template <typename FSite, typename FAtt>
@@ -248,9 +333,8 @@ __device__ __forceinline__ bool mega_wait_bars(int need, MegaCtl* ctl, const Meg
 }
 
 // TMA loads of one weight unit into a ring stage.
-__device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int li, const Dims& dm, long long u, int KB,
+__device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int li, const Dims& dm, int tile, int kb,
                                              uint32_t dst, uint32_t bar, uint64_t pol) {
-  const int tile = (int)(u / KB), kb = (int)(u % KB);
   switch (site) {
     case SITE_QKV: {
       const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
@@ -269,66 +353,48 @@ __device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int l
   }
 }
 
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tm, int c0, int c1) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(tm)), "r"(c0),
-               "r"(c1)
-               : "memory");
-}
-// L2 prefetch of one weight unit (same boxes as mega_issue_w).
-__device__ __forceinline__ void mega_prefetch_w(const MegaMaps& mp, int site, int li, const Dims& dm, long long u, int KB) {
-  const int tile = (int)(u / KB), kb = (int)(u % KB);
-  switch (site) {
-    case SITE_QKV: {
-      const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
-      if (tile < tq) tma_prefetch_2d(&mp.wq[li], kb * kBK, tile * kTileN);
-      else if (tile < tq + tk) tma_prefetch_2d(&mp.wk[li], kb * kBK, (tile - tq) * kTileN);
-      else tma_prefetch_2d(&mp.wv[li], kb * kBK, (tile - tq - tk) * kTileN);
-      break;
-    }
-    case SITE_O: tma_prefetch_2d(&mp.wo[li], kb * kBK, tile * kTileN); break;
-    case SITE_GU:
-      tma_prefetch_2d(&mp.wg[li], kb * kBK, tile * 64);
-      tma_prefetch_2d(&mp.wu[li], kb * kBK, tile * 64);
-      break;
-    case SITE_DOWN: tma_prefetch_2d(&mp.wd[li], kb * kBK, tile * kTileN); break;
-    default: tma_prefetch_2d(&mp.lm, kb * kBK, tile * kTileN); break;
-  }
-}
-// L2 prefetch of one cache tile (same boxes as att_issue_tile).
-__device__ __forceinline__ void mega_prefetch_tile(const CUtensorMap* tmKV, const KvView& kv, int layer, int seq, int h, int ti,
-                                                   int L, int KPS, int HD) {
-  const int HB = HD / 64, npg = KPS / 16, last_page = (L - 1) / 16;
-  for (int pg = 0; pg < npg; ++pg) {
-    const int pi = ti * npg + pg;
-    if (pi > last_page) break;
-    const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
-    const long long rowK = ((((long long)layer * kv.n_pages + page) * 2 + 0) * kv.n_kv_heads + h) * 16;
-    const long long rowV = rowK + (long long)kv.n_kv_heads * 16;
-    for (int half = 0; half < HB; ++half) {
-      tma_prefetch_2d(tmKV, half * 64, (int)rowK);
-      tma_prefetch_2d(tmKV, half * 64, (int)rowV);
-    }
-  }
-}
-
 // ---------------------------------------------------------------------------------------------
 // fused epilogues (the four epilogue warps: 128 threads, named barrier 2)
 // ---------------------------------------------------------------------------------------------
+// Bounded wait on a cluster-scope barrier in this block's shared memory (one thread).
+__device__ __forceinline__ bool mega_wait_cluster(uint32_t bar, uint32_t parity, MegaCtl* ctl, const MegaParams& p, int* status,
+                                                  int where, int extra) {
+  volatile int* af = &ctl->abort_flag;
+  volatile int* ag = p.abort_g;
+  for (uint32_t i = 0; i < kMegaSpin; ++i) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (i > 64) {
+      if (*af) return false;
+      if ((i & 255) == 0 && *ag) { *af = 1; return false; }
+      __nanosleep(i > 4096 ? 128 : 20);
+    }
+  }
+  *af = 1;
+  att_note_timeout(ag, where, extra);
+  *ag = 1;
+  atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+  return false;
+}
+
+// xbuf: the first block's landing area for its cluster's partial sums, [CS-1][16][128] fp32 (clusters only;
+// one chunk of 16 columns, i.e. at most 16 block rows).  xseq counts this cluster's exchanges so far.
 template <int HD>
-__device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p,
-                                              const StepArgs* __restrict__ args, const KvView& kv, const Work& w,
-                                              const Dims& dm, int et) {
+__device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, int& xseq, MegaCtl* ctl, float* xbuf,
+                                              const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
+                                              const Work& w, const Dims& dm, int et) {
   const int sidx = gseq - 1;
-  const int c = blockIdx.x, G = gridDim.x, R = p.R, Rp = p.Rp, rows = p.rows;
+  const int R = p.R, Rp = p.Rp, rows = p.rows;
   const int quarter = et >> 5, lane = et & 31;
-  const SiteInfo si = site_info(site, dm, c, G);
-  if (si.u_hi <= si.u_lo) return;
-  const long long U = (long long)si.n_tiles * si.KB;
+  const SiteSplit ss = site_split(site, dm, blockIdx.x, gridDim.x, p.cluster);
+  if (ss.g_hi <= ss.g_lo) return;   // the whole group (cluster) is idle in this phase
+  const int c = ss.grp, G = ss.ngrp;   // split-K partners across groups are addressed by group
+  const long long U = ss.U;
   const int nt128 = dm.d / kTileN;
   const MegaLayerPtrs lp = p.lp[l];
+  const bool contributor = ss.CS > 1 && ss.rank > 0;
   // 1/rms of this phase's input rows (the planes hold x * gain; the scalar is applied here).  One warp
   // per row, lanes over the column tiles, fixed shuffle tree: all loads of a row are in flight together.
-  if (site == SITE_QKV || site == SITE_GU || site == SITE_LM) {
+  if (!contributor && (site == SITE_QKV || site == SITE_GU || site == SITE_LM)) {
     const int buf = (site == SITE_GU) ? 1 : 0;
     for (int r0 = quarter; r0 < R; r0 += 16) {
       float part[4];
@@ -352,45 +418,57 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
   const float invT = (site == SITE_LM) ? args->inv_temperature : 1.f;
   float* dbg_logits = (site == SITE_LM) ? args->dbg_logits : nullptr;
   const float qscale = 1.4426950408889634f / sqrtf((float)HD);
+  const int fl = et;   // feature inside the tile == TMEM lane
 
-  long long u = si.u_lo;
-  while (u < si.u_hi) {
-    const int tile = (int)(u / si.KB), kb0 = (int)(u % si.KB);
-    const int len = (int)min((long long)(si.KB - kb0), si.u_hi - u);
+  long long u = ss.g_lo;
+  Seg sg;
+  int segno = 0;
+  while (seg_next(ss, u, sg)) {
+    const int tile = sg.tile, kb0 = sg.kb0;
+    ++segno;
+    const bool mine = sg.b > sg.a;   // this block computed a share of the segment
     const int acc = seg & 1, use = seg >> 1;
-    if (et == 0) ctl->bcast[seg & 1] = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
-    bar_sync(2, 128);
-    if (!ctl->bcast[seg & 1]) return;
-    tc_fence_after();
-    if (et == 0) MEGA_EV(sidx, 4);
-    if (et == 0 && kb0 != 0) MEGA_EV2(1, sidx, 0);
-    const bool owner = (kb0 == 0), complete = owner && (len == si.KB);
-    int c_last = c;
-    if (owner && !complete) {
-      c_last = unit_owner((long long)(tile + 1) * si.KB - 1, U, G);
-      if (et < 32) {   // one lane per contributing block
+    const uint32_t taddr = ctl->tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 2 * Rp);
+
+    if (contributor) {
+      // ---- a cluster's second..fourth block: push the partial sums into the first block's shared memory
+      float v[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) v[i] = 0.f;
+      if (et == 0) {
         int ok = 1;
-        for (int base = c + 1; base <= c_last; base += 32) {
-          const int c2 = base + lane;
-          int okl = 1;
-          if (c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G)   // blocks without units add nothing
-            okl = mega_spin_ge(reinterpret_cast<const unsigned*>(p.flags + c2), (unsigned)gseq, ctl, p, w.status, 7, gseq) ? 1 : 0;
-          ok &= __all_sync(0xffffffffu, okl);
-        }
-        __threadfence();
-        if (et == 0) ctl->bcast[2] = ok;
+        if (mine) ok = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
+        // the landing area is free once the first block has consumed the previous exchange
+        if (ok && xseq > 0) ok = mega_wait_cluster(smem_u32(&ctl->xfree), (uint32_t)(xseq - 1) & 1u, ctl, p, w.status, 11, xseq) ? 1 : 0;
+        ctl->bcast[seg & 1] = ok;
       }
       bar_sync(2, 128);
-      if (!ctl->bcast[2]) return;
-      if (et == 0) MEGA_EV(sidx, 5);
+      if (!ctl->bcast[seg & 1]) return;
+      if (et == 0) MEGA_EV2(1, sidx, segno == 1 ? 0 : 2);
+      if (mine) {
+        tc_fence_after();
+        float lo[16];
+        tc_ld16(taddr, v);
+        tc_ld16(taddr + Rp, lo);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] += lo[i];
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+        const uint32_t dst = mapa_u32(smem_u32(xbuf + ((size_t)(ss.rank - 1) * 16) * kTileN + fl), 0);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) st_cluster_f32(dst + (uint32_t)(i * kTileN * 4), v[i]);
+        ++seg;
+      }
+      bar_sync(2, 128);   // every thread's remote stores precede the (cumulative) release below
+      if (et == 0) mbar_arrive_remote(mapa_u32(smem_u32(&ctl->xfull), 0));
+      if (et == 0) MEGA_EV2(1, sidx, segno == 1 ? 1 : 3);
+      ++xseq;
+      continue;
     }
-    const uint32_t taddr = ctl->tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 2 * Rp);
-    const int fl = et;   // feature inside the tile == TMEM lane
 
-    // per-tile constants of the fused epilogues
+    // per-tile constants of the fused epilogues; their global loads are issued before any wait
     int kind = 0, head = 0, dim = 0;
-    float bias = 0.f;
-    const bf16* gain = nullptr;
+    float bias = 0.f, gn = 1.f;
     if (site == SITE_QKV) {
       int fs;
       if (tile < tq) { kind = 0; fs = tile * kTileN + fl; }
@@ -401,32 +479,90 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       const bf16* bp = kind == 0 ? lp.bq : (kind == 1 ? lp.bk : lp.bv);
       if (bp) bias = __bfloat162float(bp[fs]);
     } else if (site == SITE_O) {
-      gain = lp.gain_ffn;
+      gn = __bfloat162float(lp.gain_ffn[tile * kTileN + fl]);
     } else if (site == SITE_DOWN) {
-      gain = lp.gain_next;
+      gn = __bfloat162float(lp.gain_next[tile * kTileN + fl]);
     }
+
+    const bool owner = (kb0 == 0), complete = owner && (sg.len == ss.KB);
+    int c_last = c;
+    // An owner first makes sure the other groups that share the tile have published (with clusters they did
+    // long ago: their share of this tile was the first thing they computed), then waits for its own sums.
+    if (owner && !complete) {
+      c_last = unit_owner((long long)(tile + 1) * ss.KB - 1, U, G);
+      if (et < 32) {   // one lane per contributing group
+        int ok = 1;
+        for (int base = c + 1; base <= c_last; base += 32) {
+          const int c2 = base + lane;
+          int okl = 1;
+          if (c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G)   // groups without units add nothing
+            okl = mega_spin_ge(reinterpret_cast<const unsigned*>(p.flags + c2), (unsigned)gseq, ctl, p, w.status, 7, gseq) ? 1 : 0;
+          ok &= __all_sync(0xffffffffu, okl);
+        }
+        __threadfence();
+        if (et == 0) ctl->bcast[2] = ok;
+      }
+      bar_sync(2, 128);
+      if (!ctl->bcast[2]) return;
+      if (et == 0) MEGA_EV(sidx, 5);
+    }
+    if (et == 0) {
+      int ok = 1;
+      if (mine) ok = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
+      if (ok && ss.CS > 1) ok = mega_wait_cluster(smem_u32(&ctl->xfull), (uint32_t)xseq & 1u, ctl, p, w.status, 12, xseq) ? 1 : 0;
+      ctl->bcast[seg & 1] = ok;
+    }
+    bar_sync(2, 128);
+    if (!ctl->bcast[seg & 1]) return;
+    tc_fence_after();
+    if (et == 0) MEGA_EV(sidx, 4);
+    if (et == 0 && segno == 1) MEGA_EV2(4, sidx, 4);
 
     for (int c0 = 0; c0 < Rp; c0 += 16) {
       float v[16], xs[16];
-      if (owner && (site == SITE_O || site == SITE_DOWN)) {   // residual rows: issue the loads before anything else
+      float2 cs[16];
+      // every global load of this chunk is issued before anything waits on one of them
+      if (owner && (site == SITE_O || site == SITE_DOWN)) {   // residual rows
         const int f = tile * kTileN + fl;
 #pragma unroll
         for (int i = 0; i < 16; ++i) xs[i] = (c0 + i < R) ? __ldcg(w.X + (size_t)(c0 + i) * dm.d + f) : 0.f;
       }
-      {
+      if (owner && site == SITE_QKV && kind < 2) {            // rotary table rows
+        const int ii = dim & (HD / 2 - 1);
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          cs[i] = (c0 + i < R) ? __ldcg(w.rope + (size_t)(c0 + i) * (HD / 2) + ii) : make_float2(1.f, 0.f);
+      }
+      if (mine) {
         float lo[16];
         tc_ld16(taddr + c0, v);
         tc_ld16(taddr + Rp + c0, lo);
 #pragma unroll
         for (int i = 0; i < 16; ++i) v[i] += lo[i];
+      } else {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+      }
+      if (ss.CS > 1) {   // the cluster's other shares, in block order (single chunk: Rp == 16)
+        for (int r = 1; r < ss.CS; ++r) {
+          const int ar = kb0 + r * sg.len / ss.CS, br = kb0 + (r + 1) * sg.len / ss.CS;
+          if (br > ar) {
+            const float* src = xbuf + ((size_t)(r - 1) * 16) * kTileN + fl;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] += src[(size_t)i * kTileN];
+          }
+        }
+        bar_sync(2, 128);   // the landing area has been read by everyone
+        if (et >= 1 && et < ss.CS) mbar_arrive_remote(mapa_u32(smem_u32(&ctl->xfree), et));
       }
       if (!owner) {
         float* dst = p.pbuf + ((size_t)c * Rp + c0) * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) dst[(size_t)i * kTileN] = v[i];
+        for (int i = 0; i < 16; ++i)
+          if (c0 + i < R) dst[(size_t)i * kTileN] = v[i];
         continue;
       }
-      for (int cb = c + 1; cb <= c_last; cb += 4) {   // four contributors' loads in flight at a time, added in block order
+      for (int cb = c + 1; cb <= c_last; cb += 4) {   // four contributing groups' loads in flight at a time, added in group order
         float pv[4][16];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -434,7 +570,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           const bool live = c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G;
           const float* src = p.pbuf + ((size_t)(live ? c2 : c) * Rp + c0) * kTileN + fl;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) pv[k][i] = live ? __ldcg(src + (size_t)i * kTileN) : 0.f;
+          for (int i = 0; i < 16; ++i) pv[k][i] = (live && c0 + i < R) ? __ldcg(src + (size_t)i * kTileN) : 0.f;
         }
 #pragma unroll
         for (int k = 0; k < 4; ++k)
@@ -450,10 +586,6 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           v[i] = v[i] * (r < R ? ctl->inv[r] : 0.f) + bias;
         }
         if (kind < 2) {
-          const int ii = dim & (half - 1);
-          float2 cs[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) cs[i] = (c0 + i < R) ? __ldcg(w.rope + (size_t)(c0 + i) * half + ii) : make_float2(1.f, 0.f);
 #pragma unroll
           for (int i = 0; i < 16; ++i) ctl->u.exch[fl][i] = v[i];
           bar_sync(2, 128);
@@ -465,24 +597,23 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           }
           bar_sync(2, 128);
         }
+        if (et == 0) MEGA_EV2(0, sidx, 6);
+        // query row (b, kvh, g, j) sits at ((b*Hq + head)*rows + j)*HD; a cache row at
+        // ((((layer*n_pages + page)*2 + K|V)*Hkv + head)*page_size + slot)*HD: the per-row parts are tabulated
+        if (kind == 0) {
+          bf16* qb = w.Qb + (size_t)head * rows * HD + dim;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int r = c0 + i;
-          if (r < R) {
-            if (kind == 0) {
-              const int group = dm.Hq / dm.Hkv;
-              bf16* qb = w.Qb + ((((size_t)ctl->row_b[r] * dm.Hkv + head / group) * group + head % group) * rows +
-                                 ctl->row_j[r]) * HD;
-              qb[dim] = __float2bfloat16_rn(v[i] * qscale);
-            } else {
-              bf16* row = kv_row<bf16>(kv, l, ctl->row_page[r], kind - 1, head, ctl->row_slot[r]);
-              row[dim] = __float2bfloat16_rn(v[i]);
-            }
-          }
+          for (int i = 0; i < 16; ++i)
+            if (c0 + i < R) qb[ctl->row_qoff[c0 + i]] = __float2bfloat16_rn(v[i] * qscale);
+        } else {
+          bf16* kvb = reinterpret_cast<bf16*>(kv.pool) +
+                      ((size_t)l * kv.n_pages * 2 * dm.Hkv + (size_t)(kind - 1) * dm.Hkv + head) * kv.page_size * HD + dim;
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (c0 + i < R) kvb[ctl->row_kvoff[c0 + i]] = __float2bfloat16_rn(v[i]);
         }
       } else if (site == SITE_O || site == SITE_DOWN) {
         const int f = tile * kTileN + fl;
-        const float gn = __bfloat162float(gain[f]);
         const int buf = (site == SITE_O) ? 1 : 0;
         float ss[16];
 #pragma unroll
@@ -497,7 +628,8 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           }
         }
 #pragma unroll
-        for (int i = 0; i < 16; ++i) ss[i] = warp_sum(ss[i]);
+        for (int i = 0; i < 16; ++i)
+          if (c0 + i < R) ss[i] = warp_sum(ss[i]);   // block-uniform
         if (lane == 0) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) ctl->red[quarter][i] = ss[i];
@@ -570,20 +702,20 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       }
     }
     if (et == 0) MEGA_EV2(0, sidx, 7);
-    tc_fence_before();
-    mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+    if (mine) {
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+      ++seg;
+    }
+    if (ss.CS > 1) ++xseq;
     if (!owner) {   // publish the partial: block barrier, then one cumulative fence and the flag
-      if (et == 0) MEGA_EV2(1, sidx, 1);
       bar_sync(2, 128);
       if (et == 0) {
-        MEGA_EV2(1, sidx, 2);
         __threadfence();
-        MEGA_EV2(1, sidx, 3);
         st_relaxed_s32(p.flags + c, gseq);
+        MEGA_EV2(4, sidx, 5);
       }
     }
-    u += len;
-    ++seg;
   }
   if (et == 0) MEGA_EV(sidx, 6);
 }
@@ -719,6 +851,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   extern __shared__ uint8_t mega_smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(mega_smem_raw) + 1023) & ~(uintptr_t)1023);
   MegaCtl* ctl = reinterpret_cast<MegaCtl*>(ring + (size_t)p.stages * p.stage_bytes);
+  float* xbuf = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(ctl) + ((sizeof(MegaCtl) + 127) & ~(size_t)127));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x, NS = p.stages, B = p.B, R = p.R, Rp = p.Rp, rows = p.rows;
   const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
@@ -735,7 +868,8 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     }
     ctl->abort_flag = 0;
     ctl->bars_passed = 0;
-    ctl->w_issued = 0;
+    mbar_init(smem_u32(&ctl->xfull), (uint32_t)max(p.cluster - 1, 1));
+    mbar_init(smem_u32(&ctl->xfree), 1);
     int acc = 0;
     for (int b = 0; b < B; ++b) {
       const int L = kv.kv_len[args->seq_ids[b]];
@@ -756,6 +890,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (p.cluster > 1) cluster_sync_all();   // every block's barriers exist before any block arrives on them
   if (threadIdx.x < R) {
     const int r = threadIdx.x, b = r / rows, j = r % rows, gamma = rows - 1;
     const int pos = ctl->plan.L[b] + j;
@@ -764,6 +899,8 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     ctl->row_page[r] = kv.block_table[(size_t)args->seq_ids[b] * kv.max_pages_per_seq + pos / kv.page_size];
     ctl->row_slot[r] = pos % kv.page_size;
     ctl->tgt_tok[r] = (j < gamma) ? args->draft_ids[b * gamma + j] : -1;
+    ctl->row_qoff[r] = (b * dm.Hq * rows + j) * dm.hd;
+    ctl->row_kvoff[r] = ((long long)ctl->row_page[r] * 2 * dm.Hkv * kv.page_size + ctl->row_slot[r]) * dm.hd;
   }
   __syncthreads();
 
@@ -772,25 +909,33 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   const int n_att = (int)(t_hi - t_lo);
   auto stage_addr = [&](int s) -> uint32_t { return smem_u32(ring + (size_t)s * p.stage_bytes); };
 
+  // Register reallocation between warpgroups: the single-thread roles need few registers, the workers
+  // (fused epilogues, attention fragments) many.  Under the 384-thread launch bound of 168 registers per
+  // thread the workers spill, and with 227 KB of the SM's memory configured as shared memory a spill reload
+  // rarely hits L1: it costs an L2 round trip.
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kMegaRegsLight));
   if (warp == 0) {
     // ------------------------------ weight / cache-tile producer ------------------------------
     if (lane == 0) {
       const uint64_t pol_w = l2_policy_evict_first();
       int it = 0, sidx = 0;
       bool alive = true;
-      volatile int* w_issued = &ctl->w_issued;
       auto wait_slot = [&](int i) -> bool {
         return i < NS || mega_wait(smem_u32(&ctl->empty[i % NS]), (uint32_t)((i / NS) - 1) & 1u, ctl, p, w.status, 1, i);
       };
       auto fsite = [&](int site, int l) {
         if (!alive) return;
-        const SiteInfo si = site_info(site, dm, c, G);
-        for (long long u = si.u_lo; u < si.u_hi; ++u, ++it) {
-          if (!wait_slot(it)) { alive = false; return; }
-          const uint32_t bar = smem_u32(&ctl->full[it % NS]);
-          mbar_expect_tx(bar, kWTileBytes);
-          mega_issue_w(mp, site, l - p.l0, dm, u, si.KB, stage_addr(it % NS), bar, pol_w);
-          *w_issued = it + 1;
+        const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
+        long long u = ss.g_lo;
+        Seg sg;
+        while (seg_next(ss, u, sg)) {
+          for (int kb = sg.a; kb < sg.b; ++kb, ++it) {
+            if (!wait_slot(it)) { alive = false; return; }
+            const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+            mbar_expect_tx(bar, kWTileBytes);
+            mega_issue_w(mp, site, l - p.l0, dm, sg.tile, kb, stage_addr(it % NS), bar, pol_w);
+          }
         }
         MEGA_EV(sidx, 7);
         ++sidx;
@@ -804,43 +949,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           mbar_arrive(bar);   // stands in for the activation producer, which skips cache tiles
           const AttTile x = att_locate(pl, B, g.KPS, (int)t);
           att_issue_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD, stage_addr(it % NS), bar);
-          *w_issued = it + 1;
         }
-      };
-      mega_walk(p, fsite, fatt);
-    }
-  } else if (warp == 3) {
-    // ------------------------------ L2 prefetcher ------------------------------
-    // Walks the same unit sequence ahead of the producer and requests the boxes into L2 only, so that HBM
-    // keeps streaming while every block waits at a barrier with a full ring; the real loads then hit L2.
-    // It stays at most l2_ahead units ahead of the producer's issue point.
-    if (lane == 0 && p.l2_ahead > 0) {
-      volatile int* w_issued = &ctl->w_issued;
-      volatile int* af = &ctl->abort_flag;
-      const int D = p.l2_ahead;
-      int pf = 0;
-      bool alive = true;
-      auto gate = [&]() -> bool {   // true: prefetch unit pf; false: skip it (the real load is imminent)
-        uint32_t i = 0;
-        while (pf >= *w_issued + D) {
-          if (*af || ++i > kMegaSpin) { alive = false; return false; }
-          __nanosleep(100);
-        }
-        return pf >= *w_issued + 2;
-      };
-      auto fsite = [&](int site, int l) {
-        if (!alive) return;
-        const SiteInfo si = site_info(site, dm, c, G);
-        for (long long u = si.u_lo; u < si.u_hi && alive; ++u, ++pf)
-          if (gate()) mega_prefetch_w(mp, site, l - p.l0, dm, u, si.KB);
-      };
-      auto fatt = [&](int l) {
-        if (!alive) return;
-        for (long long t = t_lo; t < t_hi && alive; ++t, ++pf)
-          if (gate()) {
-            const AttTile x = att_locate(pl, B, g.KPS, (int)t);
-            mega_prefetch_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD);
-          }
       };
       mega_walk(p, fsite, fatt);
     }
@@ -853,17 +962,18 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
-        const SiteInfo si = site_info(site, dm, c, G);
+        const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
         bool first = true;
-        long long u = si.u_lo;
+        long long u = ss.g_lo;
         // Do not look at this phase's stages before the phase has begun: the attention phase in between
         // may reuse a stage several times, and a parity wait started two uses early would be satisfied by
         // the wrong one.
-        if (u < si.u_hi && !mega_wait_bars(nb, ctl, p, w.status, 10)) { alive = false; return; }
+        if (u < ss.g_hi && !mega_wait_bars(nb, ctl, p, w.status, 10)) { alive = false; return; }
         nb += (site == SITE_QKV) ? 3 : 1;
-        while (u < si.u_hi) {
-          const int kb0 = (int)(u % si.KB);
-          const int len = (int)min((long long)(si.KB - kb0), si.u_hi - u);
+        Seg sg;
+        while (seg_next(ss, u, sg)) {
+          const int len = sg.b - sg.a;
+          if (len == 0) continue;   // no share of this segment: no accumulator is used
           const int acc = seg & 1, use = seg >> 1;
           if (use > 0 && !mega_wait(smem_u32(&ctl->tmem_empty[acc]), (uint32_t)(use - 1) & 1u, ctl, p, w.status, 4, seg)) {
             alive = false;
@@ -883,7 +993,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
             tc_commit(smem_u32(&ctl->empty[s]));
           }
           tc_commit(smem_u32(&ctl->tmem_full[acc]));
-          u += len;
           ++seg;
         }
         MEGA_EV(sidx, 3);
@@ -901,22 +1010,26 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
-        const SiteInfo si = site_info(site, dm, c, G);
-        if (si.u_hi > si.u_lo) {
+        const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
+        if (ss.g_hi > ss.g_lo) {
           // inputs of this phase are complete once `nb` device-wide barriers have been passed
           if (!mega_wait_bars(nb, ctl, p, w.status, 3)) { alive = false; return; }
           __threadfence();
           fence_proxy_async();
           MEGA_EV(sidx, 0);
           const CUtensorMap* tm = (site == SITE_O) ? &mp.a_q : (site == SITE_DOWN ? &mp.a_f : &mp.a_d);
-          for (long long u = si.u_lo; u < si.u_hi; ++u, ++it) {
-            if (it >= NS && !mega_wait(smem_u32(&ctl->empty[it % NS]), (uint32_t)((it / NS) - 1) & 1u, ctl, p, w.status, 2, it)) {
-              alive = false;
-              return;
+          long long u = ss.g_lo;
+          Seg sg;
+          while (seg_next(ss, u, sg)) {
+            for (int kb = sg.a; kb < sg.b; ++kb, ++it) {
+              if (it >= NS && !mega_wait(smem_u32(&ctl->empty[it % NS]), (uint32_t)((it / NS) - 1) & 1u, ctl, p, w.status, 2, it)) {
+                alive = false;
+                return;
+              }
+              const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+              mbar_expect_tx(bar, a_tx);
+              tma_load_2d(stage_addr(it % NS) + kWTileBytes, tm, bar, kb * kBK, 0, pol_a);
             }
-            const uint32_t bar = smem_u32(&ctl->full[it % NS]);
-            mbar_expect_tx(bar, a_tx);
-            tma_load_2d(stage_addr(it % NS) + kWTileBytes, tm, bar, (int)(u % si.KB) * kBK, 0, pol_a);
           }
           MEGA_EV(sidx, 1);
         }
@@ -926,22 +1039,21 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       auto fatt = [&](int l) { it += n_att; };
       mega_walk(p, fsite, fatt);
     }
-  } else if (warp >= 4) {
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kMegaRegsHeavy));
     // ------------------------------ workers ------------------------------
     const int wt = threadIdx.x - 128, ww = wt >> 5;
-    int nbar = 0, gseq = 0, seg = 0, it = 0;
+    int nbar = 0, gseq = 0, seg = 0, it = 0, xseq = 0;
     bool alive = true;
     if (p.do_embed) {
       mega_embed(ctl, p, args, kv, w, dm, wt);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     }
-    auto units = [&](int site) -> int {
-      const SiteInfo si = site_info(site, dm, c, G);
-      return (int)(si.u_hi - si.u_lo);
-    };
+    auto units = [&](int site) -> int { return site_units(site_split(site, dm, c, G, p.cluster)); };
     auto gemm_phase = [&](int site, int l) {
       ++gseq;
-      if (alive && ww < 4) mega_epilogue<HD>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
+      if (alive && ww < 4) mega_epilogue<HD>(site, l, gseq, seg, xseq, ctl, xbuf, p, args, kv, w, dm, wt);
       it += units(site);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     };
@@ -973,6 +1085,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   }
   tc_fence_before();
   __syncthreads();
+  if (p.cluster > 1) cluster_sync_all();   // no block leaves while another may still write into its shared memory
   if (warp == 1) {
     if (*reinterpret_cast<volatile int*>(&ctl->abort_flag)) __nanosleep(20000);   // let copies in flight land
     tc_fence_after();
