@@ -168,10 +168,11 @@ struct AttWarp {
   // >= L are masked.
   __device__ __forceinline__ void tile(uint32_t stage, int kw0, int key_abs0, int L, int lane) {
     constexpr int HB = HD / 64;
-    float s[NT][4];
-#pragma unroll
-    for (int n = 0; n < NT; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
     const int lr = lane & 7, mid = lane >> 3;
+    // All K fragments of this warp's keys first (the ldmatrix results are not needed until the MMA chain
+    // reaches them; issued one by one in front of their MMA they would serialise the chain), then the V
+    // fragments, whose latency hides behind the score MMAs and the softmax arithmetic.
+    uint32_t kf[HD / 32][NT][4];
 #pragma unroll
     for (int kp = 0; kp < HD / 32; ++kp) {
 #pragma unroll
@@ -179,10 +180,30 @@ struct AttWarp {
         const int kk = kw0 + n * 8 + lr, page = kk >> 4, r = kk & 15;
         const int d = kp * 32 + mid * 8, half = d >> 6, c = (d & 63) >> 3;
         const uint32_t addr = stage + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(addr, b0, b1, b2, b3);
-        mma_16816(s[n], qa[2 * kp], b0, b1);
-        mma_16816(s[n], qa[2 * kp + 1], b2, b3);
+        ldsm_x4(addr, kf[kp][n][0], kf[kp][n][1], kf[kp][n][2], kf[kp][n][3]);
+      }
+    }
+    uint32_t vf[NT / 2][HD / 16][4];
+#pragma unroll
+    for (int kk2 = 0; kk2 < NT / 2; ++kk2) {
+#pragma unroll
+      for (int dp = 0; dp < HD / 16; ++dp) {
+        const int kk = kw0 + kk2 * 16 + (mid & 1) * 8 + lr, page = kk >> 4, r = kk & 15;
+        const int d = (dp * 2 + (mid >> 1)) * 8, half = d >> 6, c = (d & 63) >> 3;
+        const uint32_t addr =
+            stage + 8192u + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
+        ldsm_x4_t(addr, vf[kk2][dp][0], vf[kk2][dp][1], vf[kk2][dp][2], vf[kk2][dp][3]);
+      }
+    }
+    float s[NT][4];
+#pragma unroll
+    for (int n = 0; n < NT; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+    for (int kp = 0; kp < HD / 32; ++kp) {
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {   // the NT chains are independent: interleaved, they overlap each other's latency
+        mma_16816(s[n], qa[2 * kp], kf[kp][n][0], kf[kp][n][1]);
+        mma_16816(s[n], qa[2 * kp + 1], kf[kp][n][2], kf[kp][n][3]);
       }
     }
 #pragma unroll
@@ -201,14 +222,8 @@ struct AttWarp {
       pa[3] = pack_bf16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
 #pragma unroll
       for (int dp = 0; dp < HD / 16; ++dp) {
-        const int kk = kw0 + kk2 * 16 + (mid & 1) * 8 + lr, page = kk >> 4, r = kk & 15;
-        const int d = (dp * 2 + (mid >> 1)) * 8, half = d >> 6, c = (d & 63) >> 3;
-        const uint32_t addr =
-            stage + 8192u + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
-        uint32_t v0, v1, v2, v3;
-        ldsm_x4_t(addr, v0, v1, v2, v3);
-        mma_16816(o[2 * dp], pa, v0, v1);
-        mma_16816(o[2 * dp + 1], pa, v2, v3);
+        mma_16816(o[2 * dp], pa, vf[kk2][dp][0], vf[kk2][dp][1]);
+        mma_16816(o[2 * dp + 1], pa, vf[kk2][dp][2], vf[kk2][dp][3]);
       }
     }
   }
@@ -386,14 +401,17 @@ __device__ __forceinline__ void att_tma_2d(uint32_t dst, const CUtensorMap* tm, 
 
 // Issue the TMA loads of ring tile (sequence slot seq, KV head h, tile index ti) into `stage`; the
 // caller has already announced kAttStageBytes on `bar`.
+// pages: optional shared-memory copy of this tile's page ids (npg entries, already clamped to the
+// sequence's last page); without it each id costs the issuing thread a dependent global load.
 __device__ __forceinline__ void att_issue_tile(const CUtensorMap* tmKV, const KvView& kv, int layer, int seq, int h, int ti,
-                                               int L, int KPS, int HD, uint32_t stage, uint32_t bar) {
+                                               int L, int KPS, int HD, uint32_t stage, uint32_t bar,
+                                               const int* pages = nullptr) {
   const int HB = HD / 64, npg = KPS / 16;
   const int last_page = (L - 1) / 16;   // L >= 1 for any ring tile
   for (int p = 0; p < npg; ++p) {
     int pi = ti * npg + p;
     if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
-    const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+    const int page = pages ? pages[p] : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
     const long long rowK = ((((long long)layer * kv.n_pages + page) * 2 + 0) * kv.n_kv_heads + h) * 16;
     const long long rowV = rowK + (long long)kv.n_kv_heads * 16;
     for (int half = 0; half < HB; ++half) {
@@ -427,7 +445,13 @@ struct AttRing {
   volatile int* abort_flag;
   volatile int* abort_g;
   int* status;
+  unsigned long long* ev;   // optional: consumer warp 0 stamps [0] queries loaded, [1] last tile done, [2] partial stored
 };
+__device__ __forceinline__ unsigned long long att_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
+  return t;
+}
 
 // One consumer warp (cw of n_active = MT*KS) of block c of G: all ring segments of the block's tile
 // range [t_lo, t_hi) starting at ring position `it`, then the block's tail segments.
@@ -446,6 +470,7 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
     const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
     st.reset();
     st.load_q(a.Qb + ((size_t)x.b * Hkv + x.h) * g.nq * HD, row0, g.nq, lane);
+    if (rg.ev && cw == 0 && lane == 0) { rg.ev[3] = st.qa[0][0]; rg.ev[0] = att_timer_ns(); }
     for (int i = 0; i < n; ++i, ++it) {
       const int s = it % rg.stages;
       const uint32_t bar = att_smem_u32(&rg.full[s]), par = (uint32_t)(it / rg.stages) & 1u;
@@ -466,7 +491,9 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
         }
       }
     }
+    if (rg.ev && cw == 0 && lane == 0) rg.ev[1] = att_timer_ns();
     st.store(a.P, (size_t)c + (size_t)x.b * Hkv + x.h, ks, row0, g.nq, lane);
+    if (rg.ev && cw == 0 && lane == 0) rg.ev[2] = att_timer_ns();
     t += n;
   }
   // tail segments: (b, h) number x goes to block G-1-(x mod G), key share 0 only
@@ -508,13 +535,28 @@ __device__ __forceinline__ bool att_consume_dispatch(const AttRing& rg, int& it,
 // ---------------------------------------------------------------------------------------------
 constexpr int kAttStages = 8;
 constexpr int kAttTcThreads = 32 * (1 + kAttMaxWarps);
+constexpr int kAttPageCache = 1024;   // page ids of a block's first tiles kept in shared memory
 struct AttSmemCtl {
   uint64_t full[kAttStages];
   uint64_t empty[kAttStages];
   int cons_cnt[kAttStages];
   int abort_flag;
   AttPlan plan;
+  int pages[kAttPageCache];
 };
+// Page ids of the block's ring tiles [t_lo, t_hi), npg per tile, as many as fit; all threads of the caller.
+__device__ __forceinline__ void att_fill_pages(int* pages, const AttPlan& pl, const KvView& kv, const StepArgs* args, int B,
+                                               int KPS, long long t_lo, long long t_hi, int tid, int nthreads) {
+  const int npg = KPS / 16;
+  const long long n = min((t_hi - t_lo) * npg, (long long)kAttPageCache);
+  for (int i = tid; i < n; i += nthreads) {
+    const AttTile x = att_locate(pl, B, KPS, (int)(t_lo + i / npg));
+    int pi = x.ti * npg + i % npg;
+    const int last_page = (x.L - 1) / 16;
+    if (pi > last_page) pi = last_page;
+    pages[i] = __ldg(kv.block_table + (size_t)args->seq_ids[x.b] * kv.max_pages_per_seq + pi);
+  }
+}
 
 template <int HD>
 __global__ void __launch_bounds__(kAttTcThreads, 1)
@@ -542,9 +584,15 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
   const AttPlan& pl = ctl->plan;
   const int G = gridDim.x, c = blockIdx.x;
   volatile int* abort_flag = &ctl->abort_flag;
+  {
+    const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
+    att_fill_pages(ctl->pages, pl, kv, args, B, g.KPS, t_lo, t_hi, threadIdx.x, blockDim.x);
+  }
+  __syncthreads();
   if (warp == 0) {
     if (lane == 0) {
       const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
+      const int npg = g.KPS / 16;
       int it = 0;
       for (long long t = t_lo; t < t_hi; ++t, ++it) {
         const int s = it % kAttStages, round = it / kAttStages;
@@ -553,11 +601,12 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         const uint32_t bar = att_smem_u32(&ctl->full[s]);
         att_mbar_expect_tx(bar, kAttStageBytes);
         att_issue_tile(&tmKV, kv, a.layer, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD,
-                       att_smem_u32(ring + (size_t)s * kAttStageBytes), bar);
+                       att_smem_u32(ring + (size_t)s * kAttStageBytes), bar,
+                       (it + 1) * npg <= kAttPageCache ? ctl->pages + it * npg : nullptr);
       }
     }
   } else if (warp - 1 < g.MT * g.KS) {
-    AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, kAttStageBytes, kAttStages, abort_flag, nullptr, w.status};
+    AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, kAttStageBytes, kAttStages, abort_flag, nullptr, w.status, nullptr};
     int it = 0;
     att_consume_dispatch<HD>(rg, it, pl, g, args, kv, a, Hkv, c, G, warp - 1, lane);
   }
@@ -569,9 +618,23 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
 // sub-partials in key-share order, then the tail.  One warp per item; writes the O-projection input.
 // G_att: number of blocks of the attention pass.  Partial buffers are zero-filled at allocation, so the
 // slots of blocks without tiles (weight 0) hold finite values.
+// 128-bit / 64-bit loads of a lane's share of an output row
+template <int DPL> struct AttVec;
+template <> struct AttVec<4> {
+  typedef float4 type;
+  static __device__ __forceinline__ void fma(float* acc, const float4& v, float w) {
+    acc[0] += v.x * w; acc[1] += v.y * w; acc[2] += v.z * w; acc[3] += v.w * w;
+  }
+};
+template <> struct AttVec<2> {
+  typedef float2 type;
+  static __device__ __forceinline__ void fma(float* acc, const float2& v, float w) { acc[0] += v.x * w; acc[1] += v.y * w; }
+};
+
 template <typename T, int HD>
 __device__ __forceinline__ void att_combine_item(const AttPartials& P, const AttPlan& pl, const AttGeom& g, int G_att,
-                                                 int n_tail_base, int Hkv, int item, void* ATT, int R, int Hq, int lane) {
+                                                 int n_tail_base, int Hkv, int item, void* ATT, int R, int Hq, int lane,
+                                                 unsigned long long* ev = nullptr) {
   const int q = item % g.nq, bh = item / g.nq, b = bh / Hkv, h = bh % Hkv;
   const int L = pl.L[b];
   const int nt_b = (L + g.KPS - 1) / g.KPS;
@@ -582,29 +645,44 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     n_cta = att_owner(t0 + nt_b - 1, pl.T, G_att) - c_first + 1;
   }
   const int n_sub = n_cta * g.KS + 1;   // the last one is the tail
-  auto sub_index = [&](int k) -> size_t {
-    if (k >= n_sub - 1) return ((size_t)(n_tail_base + bh) * kAttMaxSub) * g.nq + q;
-    const int cc = c_first + k / g.KS, ks = k % g.KS;
-    return (((size_t)cc + bh) * kAttMaxSub + ks) * g.nq + q;
+  // sub-partial k of the ring: block c_first + k / KS, key share k % KS (KS is a power of two); row index in
+  // the partial arrays = base + (k / KS) * 4 * nq + (k % KS) * nq
+  const int ks_shift = g.KS == 4 ? 2 : (g.KS == 2 ? 1 : 0), ks_mask = g.KS - 1;
+  const int base = ((c_first + bh) * kAttMaxSub) * g.nq + q, step_c = kAttMaxSub * g.nq;
+  const int tail_idx = ((n_tail_base + bh) * kAttMaxSub) * g.nq + q;
+  auto sub_index = [&](int k) -> int {
+    return k >= n_sub - 1 ? tail_idx : base + (k >> ks_shift) * step_c + (k & ks_mask) * g.nq;
   };
   const bool all_live = pl.T >= G_att;   // every block of the attention pass owns at least one tile
   auto sub_live = [&](int k) -> bool {
     if (all_live || k == n_sub - 1) return true;
-    const int cc = c_first + k / g.KS;
+    const int cc = c_first + (k >> ks_shift);
     return (long long)(cc + 1) * pl.T / G_att > (long long)cc * pl.T / G_att;
   };
   constexpr int DPL = HD / 32;   // dims per lane
+  constexpr int OB = 24;         // output rows whose loads one lane keeps in flight
+  typedef typename AttVec<DPL>::type V;
+  const V* Po = reinterpret_cast<const V*>(P.o) + lane;   // row r of the outputs starts at Po + r * 32
   float lsum = 0.f, Mrun = -INFINITY, acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
-  for (int k0 = 0; k0 < n_sub; k0 += 96) {   // 96 sub-partials at a time (three per lane)
-    float mk[3], Mb = -INFINITY;
+  for (int k0 = 0; k0 < n_sub; k0 += 96) {   // 96 sub-partials at a time (three per lane); one pass in practice
+    // Everything this pass reads is requested before anything is used: maxima, sums, and the first OB
+    // output rows (their weights are not needed to issue the loads).
+    float mk[3], lk[3];
 #pragma unroll
     for (int u = 0; u < 3; ++u) {
       const int k = k0 + u * 32 + lane;
-      mk[u] = (k < n_sub && sub_live(k)) ? __ldcg(P.m + sub_index(k)) : -INFINITY;
-      Mb = fmaxf(Mb, mk[u]);
+      const bool live = k < n_sub && sub_live(k);
+      mk[u] = live ? __ldcg(P.m + sub_index(k)) : -INFINITY;
+      lk[u] = live ? __ldcg(P.l + sub_index(k)) : 0.f;
     }
+    const int kn = min(96, n_sub - k0);
+    V ob[OB];
+#pragma unroll
+    for (int k = 0; k < OB; ++k) ob[k] = __ldcg(Po + (size_t)sub_index(k0 + min(k, kn - 1)) * 32);
+    float Mb = fmaxf(fmaxf(mk[0], mk[1]), mk[2]);
+    if (ev && lane == 0) ev[0] = att_timer_ns();
     Mb = warp_max(Mb);
     const float Mnew = fmaxf(Mrun, Mb);
     if (Mnew == -INFINITY) continue;   // warp-uniform: nothing live so far
@@ -616,20 +694,29 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     float wk[3], lpart = 0.f;
 #pragma unroll
     for (int u = 0; u < 3; ++u) {
-      const int k = k0 + u * 32 + lane;
       wk[u] = (mk[u] == -INFINITY) ? 0.f : exp2f(mk[u] - Mnew);
-      if (wk[u] != 0.f) lpart += __ldcg(P.l + sub_index(k)) * wk[u];
+      lpart += lk[u] * wk[u];
     }
     lsum += warp_sum(lpart);
-    const int kn = min(96, n_sub - k0);
-#pragma unroll 4
-    for (int k = 0; k < kn; ++k) {
-      const float wgt = __shfl_sync(0xffffffffu, k < 32 ? wk[0] : (k < 64 ? wk[1] : wk[2]), k & 31);
-      const float* op = P.o + sub_index(k0 + k) * HD + lane * DPL;
+    if (ev && lane == 0) ev[1] = att_timer_ns();
 #pragma unroll
-      for (int i = 0; i < DPL; ++i) acc[i] += __ldcg(op + i) * wgt;
+    for (int k = 0; k < OB; ++k) {
+      const float wgt = k < kn ? __shfl_sync(0xffffffffu, wk[0], k) : 0.f;   // OB <= 32: the first weight register
+      AttVec<DPL>::fma(acc, ob[k], wgt);
+    }
+    for (int kb = OB; kb < kn; kb += OB) {   // further output rows, OB at a time, added in order
+#pragma unroll
+      for (int k = 0; k < OB; ++k) ob[k] = __ldcg(Po + (size_t)sub_index(k0 + min(kb + k, kn - 1)) * 32);
+#pragma unroll
+      for (int k = 0; k < OB; ++k) {
+        const int kk = kb + k;
+        const float wsel = kk < 32 ? wk[0] : (kk < 64 ? wk[1] : wk[2]);
+        const float wgt = kk < kn ? __shfl_sync(0xffffffffu, wsel, kk & 31) : 0.f;
+        AttVec<DPL>::fma(acc, ob[k], wgt);
+      }
     }
   }
+  if (ev && lane == 0) { ev[3] = (unsigned long long)__float_as_uint(acc[0]); ev[2] = att_timer_ns(); }
   const int gq = q / g.rows, j = q % g.rows, r = b * g.rows + j, head = h * g.group + gq;
   const float inv = 1.0f / lsum;
 #pragma unroll
@@ -648,7 +735,7 @@ __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dim
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
   const int items = B * dm.Hkv * g.nq;
-  for (int item = blockIdx.x * wpb + warp; item < items; item += gridDim.x * wpb)
+  for (int item = warp * gridDim.x + blockIdx.x; item < items; item += gridDim.x * wpb)   // spread over blocks first
     att_combine_item<bf16, HD>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, w.ATT, B * rows, dm.Hq, lane);
 }
 

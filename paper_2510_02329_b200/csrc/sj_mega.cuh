@@ -131,6 +131,7 @@ struct MegaCtl {
   RowStat rs[kMaxGamma + 1];
   float score[kMaxGamma + 1];
   AttPlan plan;
+  int att_pages[kAttPageCache];   // page ids of this block's first ring tiles (the same in every layer)
   union {
     float exch[128][17];
     RowStat sred[kMegaWorkers];
@@ -241,8 +242,22 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// The step as a list of phases: per layer QKV, attention (+ combine, which streams nothing), O, gate/up,
+// down; then the LM head.  One call site per callback: the callbacks are large and get inlined, and the
+// kernel has to fit the instruction cache.
+__device__ __forceinline__ int mega_n_phases(const MegaParams& p) { return 5 * (p.l1 - p.l0) + (p.do_lm ? 1 : 0); }
+// phase index -> (site or -1 for attention, layer)
+__device__ __forceinline__ void mega_phase(const MegaParams& p, int ph, int& site, int& l) {
+  const int nl = p.l1 - p.l0;
+  if (ph >= 5 * nl) { site = SITE_LM; l = p.l1 - 1; return; }
+  l = p.l0 + ph / 5;
+  const int k = ph % 5;
+  site = k == 0 ? SITE_QKV : k == 1 ? -1 : k == 2 ? SITE_O : k == 3 ? SITE_GU : SITE_DOWN;
+}
+// The same walk with one call site per site kind: the single-thread loops (producers, MMA issuer) are small
+// and their per-unit instruction count bounds the streaming rate, so they get a copy specialised per site.
 template <typename FSite, typename FAtt>
-__device__ __forceinline__ void mega_walk(const MegaParams& p, FSite fsite, FAtt fatt) {
+__device__ __forceinline__ void mega_walk_spec(const MegaParams& p, FSite fsite, FAtt fatt) {
   for (int l = p.l0; l < p.l1; ++l) {
     fsite(SITE_QKV, l);
     fatt(l);
@@ -251,6 +266,27 @@ __device__ __forceinline__ void mega_walk(const MegaParams& p, FSite fsite, FAtt
     fsite(SITE_DOWN, l);
   }
   if (p.do_lm) fsite(SITE_LM, p.l1 - 1);
+}
+// Position in the ring: stage index and how many times the ring has wrapped, advanced without divisions.
+struct RingPos {
+  int s, r, NS;
+  __device__ __forceinline__ void advance(int n) {   // n may exceed NS (skipping a phase's stages)
+    s += n;
+    if (s >= NS) { r += s / NS; s %= NS; }
+  }
+  __device__ __forceinline__ void next() {
+    if (++s == NS) { s = 0; ++r; }
+  }
+};
+template <typename FSite, typename FAtt>
+__device__ __forceinline__ void mega_walk(const MegaParams& p, FSite fsite, FAtt fatt) {
+  const int n = mega_n_phases(p);
+  for (int ph = 0; ph < n; ++ph) {
+    int site, l;
+    mega_phase(p, ph, site, l);
+    if (site < 0) fatt(l);
+    else fsite(site, l);
+  }
 }
 
 __device__ __forceinline__ void bar_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
@@ -907,6 +943,8 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   const AttPlan& pl = ctl->plan;
   const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
   const int n_att = (int)(t_hi - t_lo);
+  att_fill_pages(ctl->att_pages, pl, kv, args, B, g.KPS, t_lo, t_hi, threadIdx.x, blockDim.x);
+  __syncthreads();
   auto stage_addr = [&](int s) -> uint32_t { return smem_u32(ring + (size_t)s * p.stage_bytes); };
 
   // Register reallocation between warpgroups: the single-thread roles need few registers, the workers
@@ -919,22 +957,39 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     // ------------------------------ weight / cache-tile producer ------------------------------
     if (lane == 0) {
       const uint64_t pol_w = l2_policy_evict_first();
-      int it = 0, sidx = 0;
+      RingPos rp{0, 0, NS};
+      int sidx = 0;
       bool alive = true;
-      auto wait_slot = [&](int i) -> bool {
-        return i < NS || mega_wait(smem_u32(&ctl->empty[i % NS]), (uint32_t)((i / NS) - 1) & 1u, ctl, p, w.status, 1, i);
+      auto wait_slot = [&]() -> bool {
+        return rp.r == 0 || mega_wait(smem_u32(&ctl->empty[rp.s]), (uint32_t)(rp.r - 1) & 1u, ctl, p, w.status, 1, rp.r);
       };
       auto fsite = [&](int site, int l) {
         if (!alive) return;
         const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
+        const int li = l - p.l0;
+        const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
         long long u = ss.g_lo;
         Seg sg;
         while (seg_next(ss, u, sg)) {
-          for (int kb = sg.a; kb < sg.b; ++kb, ++it) {
-            if (!wait_slot(it)) { alive = false; return; }
-            const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+          // the tensor map(s) and row of this segment's tile; only the K coordinate changes per unit
+          const CUtensorMap* tm0;
+          const CUtensorMap* tm1 = nullptr;
+          int row = sg.tile * kTileN;
+          if (site == SITE_QKV) {
+            if (sg.tile < tq) tm0 = &mp.wq[li];
+            else if (sg.tile < tq + tk) { tm0 = &mp.wk[li]; row = (sg.tile - tq) * kTileN; }
+            else { tm0 = &mp.wv[li]; row = (sg.tile - tq - tk) * kTileN; }
+          } else if (site == SITE_O) tm0 = &mp.wo[li];
+          else if (site == SITE_GU) { tm0 = &mp.wg[li]; tm1 = &mp.wu[li]; row = sg.tile * 64; }
+          else if (site == SITE_DOWN) tm0 = &mp.wd[li];
+          else tm0 = &mp.lm;
+          for (int kb = sg.a; kb < sg.b; ++kb) {
+            if (!wait_slot()) { alive = false; return; }
+            const uint32_t bar = smem_u32(&ctl->full[rp.s]), dst = stage_addr(rp.s);
             mbar_expect_tx(bar, kWTileBytes);
-            mega_issue_w(mp, site, l - p.l0, dm, sg.tile, kb, stage_addr(it % NS), bar, pol_w);
+            tma_load_2d(dst, tm0, bar, kb * kBK, row, pol_w);
+            if (site == SITE_GU) tma_load_2d(dst + 8192u, tm1, bar, kb * kBK, row, pol_w);
+            rp.next();
           }
         }
         MEGA_EV(sidx, 7);
@@ -942,23 +997,27 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       };
       auto fatt = [&](int l) {
         if (!alive) return;
-        for (long long t = t_lo; t < t_hi; ++t, ++it) {
-          if (!wait_slot(it)) { alive = false; return; }
-          const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+        for (long long t = t_lo; t < t_hi; ++t) {
+          if (!wait_slot()) { alive = false; return; }
+          const uint32_t bar = smem_u32(&ctl->full[rp.s]);
           mbar_expect_tx(bar, kAttStageBytes);
           mbar_arrive(bar);   // stands in for the activation producer, which skips cache tiles
           const AttTile x = att_locate(pl, B, g.KPS, (int)t);
-          att_issue_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD, stage_addr(it % NS), bar);
+          const int ai = (int)(t - t_lo) * (g.KPS / 16);
+          att_issue_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD, stage_addr(rp.s), bar,
+                         ai + g.KPS / 16 <= kAttPageCache ? ctl->att_pages + ai : nullptr);
+          rp.next();
         }
       };
-      mega_walk(p, fsite, fatt);
+      mega_walk_spec(p, fsite, fatt);
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(2 * Rp);
       const uint32_t tmem_base = ctl->tmem_base;
-      int it = 0, seg = 0, sidx = 0, nb = p.do_embed ? 1 : 0;
+      RingPos rp{0, 0, NS};
+      int seg = 0, sidx = 0, nb = p.do_embed ? 1 : 0;
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
@@ -980,17 +1039,17 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
             return;
           }
           tc_fence_after();
-          for (int i = 0; i < len; ++i, ++it) {
-            const int s = it % NS;
-            if (!mega_wait(smem_u32(&ctl->full[s]), (uint32_t)(it / NS) & 1u, ctl, p, w.status, 5, it)) { alive = false; return; }
+          const uint32_t dcol = tmem_base + (uint32_t)(acc * 2 * Rp);
+          for (int i = 0; i < len; ++i) {
+            if (!mega_wait(smem_u32(&ctl->full[rp.s]), (uint32_t)rp.r & 1u, ctl, p, w.status, 5, rp.r)) { alive = false; return; }
             tc_fence_after();
             if (first) { MEGA_EV(sidx, 2); first = false; }
-            const uint32_t wa = stage_addr(s);
+            const uint32_t wa = stage_addr(rp.s);
             const uint64_t dw = smem_desc_sw128(wa), da = smem_desc_sw128(wa + kWTileBytes);
-            const uint32_t dcol = tmem_base + (uint32_t)(acc * 2 * Rp);
 #pragma unroll
             for (int k = 0; k < kBK / 16; ++k) tc_mma_bf16(dcol, dw + 2 * k, da + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-            tc_commit(smem_u32(&ctl->empty[s]));
+            tc_commit(smem_u32(&ctl->empty[rp.s]));
+            rp.next();
           }
           tc_commit(smem_u32(&ctl->tmem_full[acc]));
           ++seg;
@@ -998,15 +1057,16 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         MEGA_EV(sidx, 3);
         ++sidx;
       };
-      auto fatt = [&](int l) { it += n_att; };
-      mega_walk(p, fsite, fatt);
+      auto fatt = [&](int l) { rp.advance(n_att); };
+      mega_walk_spec(p, fsite, fatt);
     }
   } else if (warp == 2) {
     // ------------------------------ activation producer ------------------------------
     if (lane == 0) {
       const uint64_t pol_a = l2_policy_evict_last();
       const uint32_t a_tx = (uint32_t)(2 * Rp) * 128u;
-      int it = 0, nb = p.do_embed ? 1 : 0, sidx = 0;
+      RingPos rp{0, 0, NS};
+      int nb = p.do_embed ? 1 : 0, sidx = 0;
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
@@ -1021,14 +1081,15 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           long long u = ss.g_lo;
           Seg sg;
           while (seg_next(ss, u, sg)) {
-            for (int kb = sg.a; kb < sg.b; ++kb, ++it) {
-              if (it >= NS && !mega_wait(smem_u32(&ctl->empty[it % NS]), (uint32_t)((it / NS) - 1) & 1u, ctl, p, w.status, 2, it)) {
+            for (int kb = sg.a; kb < sg.b; ++kb) {
+              if (rp.r > 0 && !mega_wait(smem_u32(&ctl->empty[rp.s]), (uint32_t)(rp.r - 1) & 1u, ctl, p, w.status, 2, rp.r)) {
                 alive = false;
                 return;
               }
-              const uint32_t bar = smem_u32(&ctl->full[it % NS]);
+              const uint32_t bar = smem_u32(&ctl->full[rp.s]);
               mbar_expect_tx(bar, a_tx);
-              tma_load_2d(stage_addr(it % NS) + kWTileBytes, tm, bar, kb * kBK, 0, pol_a);
+              tma_load_2d(stage_addr(rp.s) + kWTileBytes, tm, bar, kb * kBK, 0, pol_a);
+              rp.next();
             }
           }
           MEGA_EV(sidx, 1);
@@ -1036,8 +1097,8 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         ++sidx;
         nb += (site == SITE_QKV) ? 3 : 1;
       };
-      auto fatt = [&](int l) { it += n_att; };
-      mega_walk(p, fsite, fatt);
+      auto fatt = [&](int l) { rp.advance(n_att); };
+      mega_walk_spec(p, fsite, fatt);
     }
   }
   } else {
@@ -1057,10 +1118,21 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       it += units(site);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     };
-    for (int l = p.l0; l < p.l1; ++l) {
-      gemm_phase(SITE_QKV, l);
+    const int n_ph = mega_n_phases(p);
+    for (int ph = 0; ph < n_ph; ++ph) {
+      int site, l;
+      mega_phase(p, ph, site, l);
+      if (site >= 0) {
+        gemm_phase(site, l);
+        continue;
+      }
+      // attention over the cache tiles of the ring, then the combine
       if (alive && ww < g.MT * g.KS) {
-        AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status};
+        // attention events of block 0 go to the second event set of the layer's QKV phase
+        unsigned long long* ev = (p.trace && c == 0 && (l - p.l0) * 4 < kMegaTraceSites)
+                                     ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8
+                                     : nullptr;
+        AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status, ev};
         AttArgs aa{w.Qb, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
         int it2 = it;
         att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
@@ -1070,18 +1142,15 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       if (alive) {
         const AttPartials P{w.tc_m, w.tc_l, w.tc_o};
         const int items = B * dm.Hkv * g.nq;
-        for (int item = c * 8 + ww; item < items; item += G * 8)
-          att_combine_item<bf16, HD>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane);
+        for (int item = ww * G + c; item < items; item += G * 8)   // spread over blocks first
+          att_combine_item<bf16, HD>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane,
+                                     (p.trace && c == 0 && ww == 0 && (l - p.l0) * 4 < kMegaTraceSites)
+                                         ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8 + 4
+                                         : nullptr);
       }
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
-      gemm_phase(SITE_O, l);
-      gemm_phase(SITE_GU, l);
-      gemm_phase(SITE_DOWN, l);
     }
-    if (p.do_lm) {
-      gemm_phase(SITE_LM, p.l1 - 1);
-      if (alive && c < B) mega_finalize(ctl, p, args, kv, w, dm, wt);
-    }
+    if (p.do_lm && alive && c < B) mega_finalize(ctl, p, args, kv, w, dm, wt);
   }
   tc_fence_before();
   __syncthreads();
