@@ -103,10 +103,6 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *   "step_impl"  1 = the whole step as one persistent cooperative kernel (bf16, tcgen05 GEMMs, at most 80
  *                block rows; default when the shape allows), 0 = one kernel per stage
  *   "ring_stages" persistent kernel: cap on the shared-memory ring depth (0 = as many as fit, the default)
- *   "cluster"    persistent kernel: 1 = launch as clusters of four blocks that split the K range of the QKV, O
- *                and down projections' tiles among themselves through distributed shared memory (only for steps
- *                of at most 16 block rows; a B200 holds 33 such clusters, i.e. 132 of its 148 SMs, which costs
- *                more streaming rate than the cheaper exchange saves), 0 = independent blocks (default)
  *   "trace"      1 = the persistent kernel's block 0 stamps its arrival at and release from every device-wide
  *                barrier, and eight events per GEMM phase, with the nanosecond global timer (sj_step_trace())
  *   "graph"      1 = replay the step as a CUDA graph (default unless the stream is NULL, which

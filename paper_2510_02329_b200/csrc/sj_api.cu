@@ -190,8 +190,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_cluster = 0;
-  int cluster_blocks = 0;          // blocks of the largest grid of 4-block clusters that fits the device (0: unknown / none)
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -512,9 +511,6 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
   } else if (n == "ring_stages") {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
-  } else if (n == "cluster") {
-    if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "cluster must be 0 or 1");
-    t->opt_cluster = value;
   } else if (n == "trace") {
     const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 16 * kMegaTraceSites;
     if (value && !t->d_trace) {
@@ -954,8 +950,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   memset(&p, 0, sizeof(p));
   p.B = B; p.rows = rows; p.R = R; p.Rp = Rp;
   p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
-  const int xbuf_bytes = 3 * 16 * kTileN * (int)sizeof(float);   // cluster landing area (reserved in either mode)
-  const int ctl_bytes = (((int)sizeof(MegaCtl) + 127) & ~127) + xbuf_bytes;
+  const int ctl_bytes = ((int)sizeof(MegaCtl) + 127) & ~127;
   const int budget = 227 * 1024 - 1024 - ctl_bytes;
   p.stages = std::min(kMegaMaxStages, budget / p.stage_bytes);
   if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
@@ -973,27 +968,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.flags = reinterpret_cast<int*>(t->d_sync + 16);
   p.n_tail_base = t->sm_count + B * dm.Hkv;
   p.trace = t->opt_trace ? t->d_trace : nullptr;
-  // Clusters of four blocks for the projections with few tiles: needs one chunk of 16 accumulator columns and
-  // a device that can hold enough clusters at once.
-  if (t->opt_cluster && Rp == 16 && t->cluster_blocks == 0) {
-    cudaLaunchConfig_t q;
-    memset(&q, 0, sizeof(q));
-    q.gridDim = dim3((t->sm_count / 4) * 4);
-    q.blockDim = dim3(kMegaThreads);
-    q.dynamicSmemBytes = 220 * 1024;
-    cudaLaunchAttribute qa[1];
-    qa[0].id = cudaLaunchAttributeClusterDimension;
-    qa[0].val.clusterDim.x = 4; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-    q.attrs = qa;
-    q.numAttrs = 1;
-    int nc = 0;
-    cudaError_t e = dm.hd == 128 ? cudaOccupancyMaxActiveClusters(&nc, k_verify_mega<128>, &q)
-                                 : cudaOccupancyMaxActiveClusters(&nc, k_verify_mega<64>, &q);
-    if (e != cudaSuccess) { cudaGetLastError(); nc = 0; }
-    t->cluster_blocks = nc >= 16 ? std::min(nc * 4, (t->sm_count / 4) * 4) : -1;
-  }
-  p.cluster = (t->opt_cluster && Rp == 16 && t->cluster_blocks > 0) ? 4 : 1;
-  const int grid = p.cluster > 1 ? t->cluster_blocks : t->sm_count;
+  const int grid = t->sm_count;
   const size_t smem = (size_t)p.stages * p.stage_bytes + ctl_bytes + 1024;
   const bool timing = t->opt_timing != 0;
   const int NL = dm.n_layers;
@@ -1018,13 +993,11 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
     cfg.blockDim = dim3(kMegaThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute at[2];
+    cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeCooperative;
     at[0].val.cooperative = 1;
-    at[1].id = cudaLaunchAttributeClusterDimension;
-    at[1].val.clusterDim.x = 4; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
     cfg.attrs = at;
-    cfg.numAttrs = p.cluster > 1 ? 2 : 1;
+    cfg.numAttrs = 1;
     const StepArgs* args = t->d_args;
     if (dm.hd == 128) CU_TRY(cudaLaunchKernelEx(&cfg, k_verify_mega<128>, mm, p, args, kv->view, W, dm));
     else CU_TRY(cudaLaunchKernelEx(&cfg, k_verify_mega<64>, mm, p, args, kv->view, W, dm));

@@ -375,8 +375,11 @@ __device__ __forceinline__ void att_note_timeout(volatile int* abort_g, int wher
 }
 // Bounded wait.  abort_flag: the block's flag (shared memory); abort_g: optional device-wide flag that
 // other blocks raise; status: device status word.
-__device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                              volatile int* abort_g = nullptr, int where = 0, int extra = 0) {
+// (Kept inline on purpose: an out-of-line call makes the caller save its live registers to local memory,
+// and with almost all of the SM's memory configured as shared memory a local-memory access costs an L2
+// round trip.)
+__device__ __forceinline__ bool att_mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                volatile int* abort_g, int where, int extra) {
   for (uint32_t i = 0; i < kAttSpin; ++i) {
     if (att_mbar_try(bar, parity)) return true;
     if (i > 64) {
@@ -390,6 +393,11 @@ __device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, vol
   if (abort_g) *abort_g = 1;
   atomicCAS(status, DEV_OK, DEV_TIMEOUT);
   return false;
+}
+__device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                              volatile int* abort_g = nullptr, int where = 0, int extra = 0) {
+  if (att_mbar_try(bar, parity)) return true;
+  return att_mbar_wait_slow(bar, parity, abort_flag, status, abort_g, where, extra);
 }
 __device__ __forceinline__ void att_tma_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
   asm volatile(
@@ -453,6 +461,10 @@ __device__ __forceinline__ unsigned long long att_timer_ns() {
   return t;
 }
 
+template <int HD, int NT>
+__device__ __forceinline__ void att_tails(AttWarp<HD, NT>& st, const AttPlan& pl, const AttGeom& g, const StepArgs* __restrict__ args,
+                                       const KvView& kv, const AttArgs& a, int Hkv, int c, int G, int row0, int lane);
+
 // One consumer warp (cw of n_active = MT*KS) of block c of G: all ring segments of the block's tile
 // range [t_lo, t_hi) starting at ring position `it`, then the block's tail segments.
 template <int HD, int NT>
@@ -497,7 +509,15 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
     t += n;
   }
   // tail segments: (b, h) number x goes to block G-1-(x mod G), key share 0 only
-  if (ks == 0) {
+  if (ks == 0 && G - 1 - c < B * Hkv) att_tails<HD, NT>(st, pl, g, args, kv, a, Hkv, c, G, row0, lane);
+  return true;
+}
+
+template <int HD, int NT>
+__device__ __forceinline__ void att_tails(AttWarp<HD, NT>& st, const AttPlan& pl, const AttGeom& g, const StepArgs* __restrict__ args,
+                                       const KvView& kv, const AttArgs& a, int Hkv, int c, int G, int row0, int lane) {
+  const int B = args->B, rows = g.rows;
+  {
     for (int x = G - 1 - c; x < B * Hkv; x += G) {
       const int b = x / Hkv, h = x % Hkv;
       const int L = pl.L[b], seq = args->seq_ids[b];
@@ -517,7 +537,6 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
       st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
     }
   }
-  return true;
 }
 
 template <int HD>

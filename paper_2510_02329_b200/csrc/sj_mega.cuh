@@ -27,14 +27,6 @@
 //   gate/up (tiles interleave 64 gate and 64 up features) -> silu(g) * u -> down-projection input planes
 //   down  -> as O
 //   LM head (whole tiles) -> softmax statistics per (vocabulary tile, row), logit of the drafted token
-// The three projections with few tiles (QKV, O, down: 32..48 tiles for 148 SMs) would have every tile split
-// over 3..5 blocks that all finish at the same moment, so that the owner's wait for its contributors, through
-// L2 (about 2 us per round trip while the weight stream runs), sits on the critical path of every phase.
-// With thread-block clusters of four the stream-K deal is made over CLUSTERS for these three sites and each
-// segment's K range is cut in four inside the cluster; the three other blocks push their partial sums into
-// the first block's shared memory (distributed shared memory + a cluster-scope mbarrier), which then acts for
-// the cluster.  Across clusters a tile is shared by at most two clusters whose shares sit at opposite ends of
-// their ranges, so the contributor has published long before the owner asks.
 // Attention: see sj_attn_tc.cuh; its cache tiles travel through the same ring.
 //
 // Every wait is bounded; the first one to run out raises a device-wide abort word that all other waits
@@ -85,7 +77,6 @@ struct MegaParams {
   int* abort_g;               // device-wide abort word        }
   int* flags;                 // [blocks] split-K flags        }
   int n_tail_base;
-  int cluster;                // blocks per cluster (1 or 4)
   // optional timeline of block 0 (global-timer nanoseconds):
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
   //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
@@ -120,8 +111,6 @@ struct MegaCtl {
   int abort_flag;
   int bars_passed;
   int bcast[4];
-  uint64_t xfull;          // cluster exchange: the contributors' partial sums have landed (first block of a cluster)
-  uint64_t xfree;          // cluster exchange: the first block has consumed this block's previous partial sums
   float inv[kMegaMaxRows];
   int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
   int row_qoff[kMegaMaxRows];         // element offset of row r's queries in the query buffer, without the head part
@@ -169,20 +158,21 @@ __device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
   return c;
 }
 
-// How a site's units are dealt.  A "group" is a cluster for the sites whose tiles are split inside a cluster
-// (QKV, O, down when clusters are on) and a single block otherwise.  Groups take [g*U/n, (g+1)*U/n); every
-// maximal run of units of one tile inside a group's range is a segment, and block `rank` of the group takes
-// the K blocks [kb0 + rank*len/CS, kb0 + (rank+1)*len/CS) of it.
+// How a site's units are dealt.  A "group" is CS consecutive blocks that share segments (CS = 1 everywhere
+// at present: a B200 holds only 33 clusters of four of these blocks, and streaming with 132 of its 148 SMs
+// cost more than an exchange through distributed shared memory saved).  Groups take [g*U/n, (g+1)*U/n);
+// every maximal run of units of one tile inside a group's range is a segment, and block `rank` of the group
+// takes the K blocks [kb0 + rank*len/CS, kb0 + (rank+1)*len/CS) of it.
 struct SiteSplit {
   int n_tiles, KB, CS, rank, grp, ngrp;
   long long U, g_lo, g_hi;
 };
-__device__ __forceinline__ SiteSplit site_split(int site, const Dims& dm, int c, int G, int cluster) {
+__device__ __forceinline__ SiteSplit site_split(int site, const Dims& dm, int c, int G) {
   SiteSplit s;
   const SiteInfo t = site_info(site, dm, 0, 1);
   s.n_tiles = t.n_tiles;
   s.KB = t.KB;
-  s.CS = (cluster > 1 && (site == SITE_QKV || site == SITE_O || site == SITE_DOWN)) ? cluster : 1;
+  s.CS = 1;
   s.ngrp = G / s.CS;
   s.grp = c / s.CS;
   s.rank = c % s.CS;
@@ -213,33 +203,6 @@ __device__ __forceinline__ int site_units(const SiteSplit& s) {
   int n = 0;
   while (seg_next(s, u, g)) n += g.b - g.a;
   return n;
-}
-
-// cluster plumbing
-__device__ __forceinline__ uint32_t mapa_u32(uint32_t local_addr, int rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void st_cluster_f32(uint32_t remote_addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote_addr), "f"(v) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // The step as a list of phases: per layer QKV, attention (+ combine, which streams nothing), O, gate/up,
@@ -392,45 +355,21 @@ __device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int l
 // ---------------------------------------------------------------------------------------------
 // fused epilogues (the four epilogue warps: 128 threads, named barrier 2)
 // ---------------------------------------------------------------------------------------------
-// Bounded wait on a cluster-scope barrier in this block's shared memory (one thread).
-__device__ __forceinline__ bool mega_wait_cluster(uint32_t bar, uint32_t parity, MegaCtl* ctl, const MegaParams& p, int* status,
-                                                  int where, int extra) {
-  volatile int* af = &ctl->abort_flag;
-  volatile int* ag = p.abort_g;
-  for (uint32_t i = 0; i < kMegaSpin; ++i) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if (i > 64) {
-      if (*af) return false;
-      if ((i & 255) == 0 && *ag) { *af = 1; return false; }
-      __nanosleep(i > 4096 ? 128 : 20);
-    }
-  }
-  *af = 1;
-  att_note_timeout(ag, where, extra);
-  *ag = 1;
-  atomicCAS(status, DEV_OK, DEV_TIMEOUT);
-  return false;
-}
-
-// xbuf: the first block's landing area for its cluster's partial sums, [CS-1][16][128] fp32 (clusters only;
-// one chunk of 16 columns, i.e. at most 16 block rows).  xseq counts this cluster's exchanges so far.
 template <int HD>
-__device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, int& xseq, MegaCtl* ctl, float* xbuf,
-                                              const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
+__device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
                                               const Work& w, const Dims& dm, int et) {
   const int sidx = gseq - 1;
   const int R = p.R, Rp = p.Rp, rows = p.rows;
   const int quarter = et >> 5, lane = et & 31;
-  const SiteSplit ss = site_split(site, dm, blockIdx.x, gridDim.x, p.cluster);
-  if (ss.g_hi <= ss.g_lo) return;   // the whole group (cluster) is idle in this phase
+  const SiteSplit ss = site_split(site, dm, blockIdx.x, gridDim.x);
+  if (ss.g_hi <= ss.g_lo) return;   // nothing to do in this phase
   const int c = ss.grp, G = ss.ngrp;   // split-K partners across groups are addressed by group
   const long long U = ss.U;
   const int nt128 = dm.d / kTileN;
   const MegaLayerPtrs lp = p.lp[l];
-  const bool contributor = ss.CS > 1 && ss.rank > 0;
   // 1/rms of this phase's input rows (the planes hold x * gain; the scalar is applied here).  One warp
   // per row, lanes over the column tiles, fixed shuffle tree: all loads of a row are in flight together.
-  if (!contributor && (site == SITE_QKV || site == SITE_GU || site == SITE_LM)) {
+  if (site == SITE_QKV || site == SITE_GU || site == SITE_LM) {
     const int buf = (site == SITE_GU) ? 1 : 0;
     for (int r0 = quarter; r0 < R; r0 += 16) {
       float part[4];
@@ -458,49 +397,11 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 
   long long u = ss.g_lo;
   Seg sg;
-  int segno = 0;
   while (seg_next(ss, u, sg)) {
     const int tile = sg.tile, kb0 = sg.kb0;
-    ++segno;
     const bool mine = sg.b > sg.a;   // this block computed a share of the segment
     const int acc = seg & 1, use = seg >> 1;
     const uint32_t taddr = ctl->tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 2 * Rp);
-
-    if (contributor) {
-      // ---- a cluster's second..fourth block: push the partial sums into the first block's shared memory
-      float v[16];
-#pragma unroll
-      for (int i = 0; i < 16; ++i) v[i] = 0.f;
-      if (et == 0) {
-        int ok = 1;
-        if (mine) ok = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
-        // the landing area is free once the first block has consumed the previous exchange
-        if (ok && xseq > 0) ok = mega_wait_cluster(smem_u32(&ctl->xfree), (uint32_t)(xseq - 1) & 1u, ctl, p, w.status, 11, xseq) ? 1 : 0;
-        ctl->bcast[seg & 1] = ok;
-      }
-      bar_sync(2, 128);
-      if (!ctl->bcast[seg & 1]) return;
-      if (et == 0) MEGA_EV2(1, sidx, segno == 1 ? 0 : 2);
-      if (mine) {
-        tc_fence_after();
-        float lo[16];
-        tc_ld16(taddr, v);
-        tc_ld16(taddr + Rp, lo);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] += lo[i];
-        tc_fence_before();
-        mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
-        const uint32_t dst = mapa_u32(smem_u32(xbuf + ((size_t)(ss.rank - 1) * 16) * kTileN + fl), 0);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) st_cluster_f32(dst + (uint32_t)(i * kTileN * 4), v[i]);
-        ++seg;
-      }
-      bar_sync(2, 128);   // every thread's remote stores precede the (cumulative) release below
-      if (et == 0) mbar_arrive_remote(mapa_u32(smem_u32(&ctl->xfull), 0));
-      if (et == 0) MEGA_EV2(1, sidx, segno == 1 ? 1 : 3);
-      ++xseq;
-      continue;
-    }
 
     // per-tile constants of the fused epilogues; their global loads are issued before any wait
     int kind = 0, head = 0, dim = 0;
@@ -522,7 +423,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 
     const bool owner = (kb0 == 0), complete = owner && (sg.len == ss.KB);
     int c_last = c;
-    // An owner first makes sure the other groups that share the tile have published (with clusters they did
+    // An owner first makes sure the other groups that share the tile have published (often they did
     // long ago: their share of this tile was the first thing they computed), then waits for its own sums.
     if (owner && !complete) {
       c_last = unit_owner((long long)(tile + 1) * ss.KB - 1, U, G);
@@ -545,14 +446,12 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     if (et == 0) {
       int ok = 1;
       if (mine) ok = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
-      if (ok && ss.CS > 1) ok = mega_wait_cluster(smem_u32(&ctl->xfull), (uint32_t)xseq & 1u, ctl, p, w.status, 12, xseq) ? 1 : 0;
       ctl->bcast[seg & 1] = ok;
     }
     bar_sync(2, 128);
     if (!ctl->bcast[seg & 1]) return;
     tc_fence_after();
     if (et == 0) MEGA_EV(sidx, 4);
-    if (et == 0 && segno == 1) MEGA_EV2(4, sidx, 4);
 
     for (int c0 = 0; c0 < Rp; c0 += 16) {
       float v[16], xs[16];
@@ -578,18 +477,6 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       } else {
 #pragma unroll
         for (int i = 0; i < 16; ++i) v[i] = 0.f;
-      }
-      if (ss.CS > 1) {   // the cluster's other shares, in block order (single chunk: Rp == 16)
-        for (int r = 1; r < ss.CS; ++r) {
-          const int ar = kb0 + r * sg.len / ss.CS, br = kb0 + (r + 1) * sg.len / ss.CS;
-          if (br > ar) {
-            const float* src = xbuf + ((size_t)(r - 1) * 16) * kTileN + fl;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] += src[(size_t)i * kTileN];
-          }
-        }
-        bar_sync(2, 128);   // the landing area has been read by everyone
-        if (et >= 1 && et < ss.CS) mbar_arrive_remote(mapa_u32(smem_u32(&ctl->xfree), et));
       }
       if (!owner) {
         float* dst = p.pbuf + ((size_t)c * Rp + c0) * kTileN + fl;
@@ -743,13 +630,11 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
       ++seg;
     }
-    if (ss.CS > 1) ++xseq;
     if (!owner) {   // publish the partial: block barrier, then one cumulative fence and the flag
       bar_sync(2, 128);
       if (et == 0) {
         __threadfence();
         st_relaxed_s32(p.flags + c, gseq);
-        MEGA_EV2(4, sidx, 5);
       }
     }
   }
@@ -887,7 +772,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   extern __shared__ uint8_t mega_smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(mega_smem_raw) + 1023) & ~(uintptr_t)1023);
   MegaCtl* ctl = reinterpret_cast<MegaCtl*>(ring + (size_t)p.stages * p.stage_bytes);
-  float* xbuf = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(ctl) + ((sizeof(MegaCtl) + 127) & ~(size_t)127));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x, NS = p.stages, B = p.B, R = p.R, Rp = p.Rp, rows = p.rows;
   const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
@@ -904,8 +788,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     }
     ctl->abort_flag = 0;
     ctl->bars_passed = 0;
-    mbar_init(smem_u32(&ctl->xfull), (uint32_t)max(p.cluster - 1, 1));
-    mbar_init(smem_u32(&ctl->xfree), 1);
     int acc = 0;
     for (int b = 0; b < B; ++b) {
       const int L = kv.kv_len[args->seq_ids[b]];
@@ -926,7 +808,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (p.cluster > 1) cluster_sync_all();   // every block's barriers exist before any block arrives on them
   if (threadIdx.x < R) {
     const int r = threadIdx.x, b = r / rows, j = r % rows, gamma = rows - 1;
     const int pos = ctl->plan.L[b] + j;
@@ -965,7 +846,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       };
       auto fsite = [&](int site, int l) {
         if (!alive) return;
-        const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
+        const SiteSplit ss = site_split(site, dm, c, G);
         const int li = l - p.l0;
         const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
         long long u = ss.g_lo;
@@ -1021,7 +902,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
-        const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
+        const SiteSplit ss = site_split(site, dm, c, G);
         bool first = true;
         long long u = ss.g_lo;
         // Do not look at this phase's stages before the phase has begun: the attention phase in between
@@ -1070,7 +951,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
-        const SiteSplit ss = site_split(site, dm, c, G, p.cluster);
+        const SiteSplit ss = site_split(site, dm, c, G);
         if (ss.g_hi > ss.g_lo) {
           // inputs of this phase are complete once `nb` device-wide barriers have been passed
           if (!mega_wait_bars(nb, ctl, p, w.status, 3)) { alive = false; return; }
@@ -1105,16 +986,16 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kMegaRegsHeavy));
     // ------------------------------ workers ------------------------------
     const int wt = threadIdx.x - 128, ww = wt >> 5;
-    int nbar = 0, gseq = 0, seg = 0, it = 0, xseq = 0;
+    int nbar = 0, gseq = 0, seg = 0, it = 0;
     bool alive = true;
     if (p.do_embed) {
       mega_embed(ctl, p, args, kv, w, dm, wt);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     }
-    auto units = [&](int site) -> int { return site_units(site_split(site, dm, c, G, p.cluster)); };
+    auto units = [&](int site) -> int { return site_units(site_split(site, dm, c, G)); };
     auto gemm_phase = [&](int site, int l) {
       ++gseq;
-      if (alive && ww < 4) mega_epilogue<HD>(site, l, gseq, seg, xseq, ctl, xbuf, p, args, kv, w, dm, wt);
+      if (alive && ww < 4) mega_epilogue<HD>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
       it += units(site);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     };
@@ -1154,7 +1035,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   }
   tc_fence_before();
   __syncthreads();
-  if (p.cluster > 1) cluster_sync_all();   // no block leaves while another may still write into its shared memory
   if (warp == 1) {
     if (*reinterpret_cast<volatile int*>(&ctl->abort_flag)) __nanosleep(20000);   // let copies in flight land
     tc_fence_after();
