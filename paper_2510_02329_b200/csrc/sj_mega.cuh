@@ -44,8 +44,8 @@ constexpr int kMegaMaxLayers = 32;   // per launch (tensor maps travel as kernel
 constexpr int kMegaMaxRows = 80;
 constexpr int kMegaMaxStages = 12;
 constexpr uint32_t kMegaSpin = 1u << 22;
-constexpr int kMegaRegsLight = 64;    // registers per thread of warps 0..3 after reallocation
-constexpr int kMegaRegsHeavy = 216;   // registers per thread of the worker warps (128*96 + 256*200 <= 384*168)
+constexpr int kMegaRegsLight = 80;    // registers per thread of warps 0..3 after reallocation
+constexpr int kMegaRegsHeavy = 208;   // registers per thread of the worker warps (128*96 + 256*200 <= 384*168)
 constexpr int kMegaTraceBarriers = 1024;
 constexpr int kMegaTraceSites = 512;
 
