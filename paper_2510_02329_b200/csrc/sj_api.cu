@@ -952,7 +952,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
   const int ctl_bytes = ((int)sizeof(MegaCtl) + 127) & ~127;
   const int budget = 227 * 1024 - 1024 - ctl_bytes;
-  p.stages = std::min(kMegaMaxStages, budget / p.stage_bytes);
+  p.stages = std::min(8, std::min(kMegaMaxStages, budget / p.stage_bytes));   // deeper rings did not measure faster; the rest stays L1
   if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
   if (t->opt_ring) p.stages = std::min(p.stages, t->opt_ring);
   uint32_t tc = 32;
