@@ -152,10 +152,14 @@ __host__ __device__ __forceinline__ SiteInfo site_info(int site, const Dims& dm,
   return s;
 }
 // Block that owns unit u of a stream-K site.
-__device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
-  int c = (int)(u * G / U);
-  while ((long long)(c + 1) * U / G <= u) ++c;
-  return c;
+__device__ __forceinline__ int unit_owner(unsigned u, unsigned U, int G) {
+  unsigned c = u * (unsigned)G / U;
+  while ((c + 1) * U / (unsigned)G <= u) ++c;
+  return (int)c;
+}
+// Whether block c owns at least one unit when U units are dealt to G blocks.
+__device__ __forceinline__ bool has_units(int c, unsigned U, int G) {
+  return (unsigned)(c + 1) * U / (unsigned)G > (unsigned)c * U / (unsigned)G;
 }
 
 // How a site's units are dealt.  A "group" is CS consecutive blocks that share segments (CS = 1 everywhere
@@ -163,9 +167,11 @@ __device__ __forceinline__ int unit_owner(long long u, long long U, int G) {
 // cost more than an exchange through distributed shared memory saved).  Groups take [g*U/n, (g+1)*U/n);
 // every maximal run of units of one tile inside a group's range is a segment, and block `rank` of the group
 // takes the K blocks [kb0 + rank*len/CS, kb0 + (rank+1)*len/CS) of it.
+// Unit counts stay far below 2^24 (at most a few hundred tiles of a few hundred K blocks), so all of this
+// is 32-bit arithmetic: 64-bit division is a long inlined routine and these helpers sit in every role.
 struct SiteSplit {
   int n_tiles, KB, CS, rank, grp, ngrp;
-  long long U, g_lo, g_hi;
+  unsigned U, g_lo, g_hi;
 };
 __device__ __forceinline__ SiteSplit site_split(int site, const Dims& dm, int c, int G) {
   SiteSplit s;
@@ -176,29 +182,29 @@ __device__ __forceinline__ SiteSplit site_split(int site, const Dims& dm, int c,
   s.ngrp = G / s.CS;
   s.grp = c / s.CS;
   s.rank = c % s.CS;
-  s.U = (long long)s.n_tiles * s.KB;
+  s.U = (unsigned)s.n_tiles * (unsigned)s.KB;
   if (site == SITE_LM) {
-    s.g_lo = ((long long)s.grp * s.n_tiles / s.ngrp) * s.KB;
-    s.g_hi = ((long long)(s.grp + 1) * s.n_tiles / s.ngrp) * s.KB;
+    s.g_lo = ((unsigned)s.grp * (unsigned)s.n_tiles / (unsigned)s.ngrp) * (unsigned)s.KB;
+    s.g_hi = ((unsigned)(s.grp + 1) * (unsigned)s.n_tiles / (unsigned)s.ngrp) * (unsigned)s.KB;
   } else {
-    s.g_lo = (long long)s.grp * s.U / s.ngrp;
-    s.g_hi = (long long)(s.grp + 1) * s.U / s.ngrp;
+    s.g_lo = (unsigned)s.grp * s.U / (unsigned)s.ngrp;
+    s.g_hi = (unsigned)(s.grp + 1) * s.U / (unsigned)s.ngrp;
   }
   return s;
 }
 struct Seg { int tile, kb0, len, a, b; };
-__device__ __forceinline__ bool seg_next(const SiteSplit& s, long long& u, Seg& g) {
+__device__ __forceinline__ bool seg_next(const SiteSplit& s, unsigned& u, Seg& g) {
   if (u >= s.g_hi) return false;
-  g.tile = (int)(u / s.KB);
-  g.kb0 = (int)(u % s.KB);
-  g.len = (int)min((long long)(s.KB - g.kb0), s.g_hi - u);
+  g.tile = (int)(u / (unsigned)s.KB);
+  g.kb0 = (int)(u % (unsigned)s.KB);
+  g.len = (int)min((unsigned)(s.KB - g.kb0), s.g_hi - u);
   g.a = g.kb0 + s.rank * g.len / s.CS;
   g.b = g.kb0 + (s.rank + 1) * g.len / s.CS;
   u += g.len;
   return true;
 }
 __device__ __forceinline__ int site_units(const SiteSplit& s) {
-  long long u = s.g_lo;
+  unsigned u = s.g_lo;
   Seg g;
   int n = 0;
   while (seg_next(s, u, g)) n += g.b - g.a;
@@ -216,19 +222,6 @@ __device__ __forceinline__ void mega_phase(const MegaParams& p, int ph, int& sit
   l = p.l0 + ph / 5;
   const int k = ph % 5;
   site = k == 0 ? SITE_QKV : k == 1 ? -1 : k == 2 ? SITE_O : k == 3 ? SITE_GU : SITE_DOWN;
-}
-// The same walk with one call site per site kind: the single-thread loops (producers, MMA issuer) are small
-// and their per-unit instruction count bounds the streaming rate, so they get a copy specialised per site.
-template <typename FSite, typename FAtt>
-__device__ __forceinline__ void mega_walk_spec(const MegaParams& p, FSite fsite, FAtt fatt) {
-  for (int l = p.l0; l < p.l1; ++l) {
-    fsite(SITE_QKV, l);
-    fatt(l);
-    fsite(SITE_O, l);
-    fsite(SITE_GU, l);
-    fsite(SITE_DOWN, l);
-  }
-  if (p.do_lm) fsite(SITE_LM, p.l1 - 1);
 }
 // Position in the ring: stage index and how many times the ring has wrapped, advanced without divisions.
 struct RingPos {
@@ -364,7 +357,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
   const SiteSplit ss = site_split(site, dm, blockIdx.x, gridDim.x);
   if (ss.g_hi <= ss.g_lo) return;   // nothing to do in this phase
   const int c = ss.grp, G = ss.ngrp;   // split-K partners across groups are addressed by group
-  const long long U = ss.U;
+  const unsigned U = ss.U;
   const int nt128 = dm.d / kTileN;
   const MegaLayerPtrs lp = p.lp[l];
   // 1/rms of this phase's input rows (the planes hold x * gain; the scalar is applied here).  One warp
@@ -395,7 +388,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
   const float qscale = 1.4426950408889634f / sqrtf((float)HD);
   const int fl = et;   // feature inside the tile == TMEM lane
 
-  long long u = ss.g_lo;
+  unsigned u = ss.g_lo;
   Seg sg;
   while (seg_next(ss, u, sg)) {
     const int tile = sg.tile, kb0 = sg.kb0;
@@ -426,13 +419,13 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     // An owner first makes sure the other groups that share the tile have published (often they did
     // long ago: their share of this tile was the first thing they computed), then waits for its own sums.
     if (owner && !complete) {
-      c_last = unit_owner((long long)(tile + 1) * ss.KB - 1, U, G);
+      c_last = unit_owner((unsigned)(tile + 1) * (unsigned)ss.KB - 1u, U, G);
       if (et < 32) {   // one lane per contributing group
         int ok = 1;
         for (int base = c + 1; base <= c_last; base += 32) {
           const int c2 = base + lane;
           int okl = 1;
-          if (c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G)   // groups without units add nothing
+          if (c2 <= c_last && has_units(c2, U, G))   // groups without units add nothing
             okl = mega_spin_ge(reinterpret_cast<const unsigned*>(p.flags + c2), (unsigned)gseq, ctl, p, w.status, 7, gseq) ? 1 : 0;
           ok &= __all_sync(0xffffffffu, okl);
         }
@@ -490,7 +483,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int c2 = cb + k;
-          const bool live = c2 <= c_last && (long long)(c2 + 1) * U / G > (long long)c2 * U / G;
+          const bool live = c2 <= c_last && has_units(c2, U, G);
           const float* src = p.pbuf + ((size_t)(live ? c2 : c) * Rp + c0) * kTileN + fl;
 #pragma unroll
           for (int i = 0; i < 16; ++i) pv[k][i] = (live && c0 + i < R) ? __ldcg(src + (size_t)i * kTileN) : 0.f;
@@ -849,7 +842,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         const SiteSplit ss = site_split(site, dm, c, G);
         const int li = l - p.l0;
         const int tq = dm.Hq * dm.hd / kTileN, tk = dm.Hkv * dm.hd / kTileN;
-        long long u = ss.g_lo;
+        unsigned u = ss.g_lo;
         Seg sg;
         while (seg_next(ss, u, sg)) {
           // the tensor map(s) and row of this segment's tile; only the K coordinate changes per unit
@@ -890,7 +883,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           rp.next();
         }
       };
-      mega_walk_spec(p, fsite, fatt);
+      mega_walk(p, fsite, fatt);
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -904,7 +897,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         if (!alive) return;
         const SiteSplit ss = site_split(site, dm, c, G);
         bool first = true;
-        long long u = ss.g_lo;
+        unsigned u = ss.g_lo;
         // Do not look at this phase's stages before the phase has begun: the attention phase in between
         // may reuse a stage several times, and a parity wait started two uses early would be satisfied by
         // the wrong one.
@@ -939,7 +932,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         ++sidx;
       };
       auto fatt = [&](int l) { rp.advance(n_att); };
-      mega_walk_spec(p, fsite, fatt);
+      mega_walk(p, fsite, fatt);
     }
   } else if (warp == 2) {
     // ------------------------------ activation producer ------------------------------
@@ -959,7 +952,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           fence_proxy_async();
           MEGA_EV(sidx, 0);
           const CUtensorMap* tm = (site == SITE_O) ? &mp.a_q : (site == SITE_DOWN ? &mp.a_f : &mp.a_d);
-          long long u = ss.g_lo;
+          unsigned u = ss.g_lo;
           Seg sg;
           while (seg_next(ss, u, sg)) {
             for (int kb = sg.a; kb < sg.b; ++kb) {
@@ -979,7 +972,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         nb += (site == SITE_QKV) ? 3 : 1;
       };
       auto fatt = [&](int l) { rp.advance(n_att); };
-      mega_walk_spec(p, fsite, fatt);
+      mega_walk(p, fsite, fatt);
     }
   }
   } else {
