@@ -351,7 +351,8 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   const size_t act_rows = t->bf ? (size_t)2 * pad16(R) : (size_t)R;  // bf16: hi and lo planes
   ALLOC(tmp, uint8_t, act_rows * c.d_model * esz); W.A = tmp;
   ALLOC(W.Q, float, (size_t)R * qd);
-  if (t->bf) ALLOC(W.Qb, bf16, (size_t)R * qd);
+  if (t->bf) ALLOC(W.Qb, __half, (size_t)R * qd);
+  if (t->bf) ALLOC(W.KVn, __half, (size_t)R * 2 * kd);
   ALLOC(tmp, uint8_t, act_rows * qd * esz); W.ATT = tmp;
   ALLOC(tmp, uint8_t, act_rows * c.d_ffn * esz); W.H = tmp;
   ALLOC(W.Hf, float, (size_t)R * c.d_model);
@@ -835,7 +836,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   const StepArgs* args = t->d_args;
   Work W = t->work;
   if (!use_scratch) W.logits = nullptr;
-  if (!attn_tc) W.Qb = nullptr;
+  if (!attn_tc) W.Qb = nullptr, W.KVn = nullptr;
   cudaStream_t s = t->stream;
   const size_t row_smem = sizeof(float) * dm.d;
   SplitPlan one{nullptr, 0};
@@ -867,7 +868,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
                   (size_t)R * (qd + 2 * kd), l, (const T*)L.bq, (const T*)L.bk, (const T*)L.bv));
     // attention
     if (attn_tc) {
-      AttArgs aa{W.Qb, AttPartials{W.tc_m, W.tc_l, W.tc_o}, t->sm_count + B * dm.Hkv, l};
+      AttArgs aa{W.Qb, W.KVn, AttPartials{W.tc_m, W.tc_l, W.tc_o}, t->sm_count + B * dm.Hkv, l};
       const size_t tc_smem = kAttStages * kAttStageBytes + sizeof(AttSmemCtl) + 1024;
       const AttPartials parts{W.tc_m, W.tc_l, W.tc_o};
       const int items = B * dm.Hkv * nq, cgrid = std::max(1, std::min(4 * t->sm_count, (items + 7) / 8));

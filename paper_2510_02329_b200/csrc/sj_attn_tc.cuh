@@ -20,6 +20,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include <type_traits>
 
@@ -46,13 +47,21 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
 }
 __device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+// The attention MMAs run in fp16 (fp32 accumulate): queries and probabilities are rounded to 11 significant
+// bits instead of bf16's 8 (with random values the relative error of an attention output equals the relative
+// rounding error of the probabilities, and bf16 probabilities cost 3e-3 of hidden-state accuracy per layer),
+// and the cache's bf16 K/V fragments are converted on the fly, exactly for magnitudes in [6e-5, 65504].
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  __half2 t = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
+}
+// two packed bf16 -> two packed fp16
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) {
+  return pack_f16(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
 }
 __device__ __forceinline__ uint32_t ldcg_u32(const void* p) { return __ldcg(reinterpret_cast<const unsigned int*>(p)); }
 __device__ __forceinline__ uint32_t ldcg_u16(const void* p) { return (uint32_t)__ldcg(reinterpret_cast<const unsigned short*>(p)); }
@@ -112,9 +121,9 @@ struct AttWarp {
     l0 = l1 = 0.f;
   }
 
-  // A fragments of this warp's 16 query rows.  Qb: [nq][HD] bf16 of one (sequence, KV head), already
+  // A fragments of this warp's 16 query rows.  Qb: [nq][HD] fp16 of one (sequence, KV head), already
   // scaled by log2(e)/sqrt(HD).  Rows >= nq read as zero.
-  __device__ __forceinline__ void load_q(const bf16* __restrict__ Qb, int row0, int nq, int lane) {
+  __device__ __forceinline__ void load_q(const __half* __restrict__ Qb, int row0, int nq, int lane) {
     const int r0 = row0 + (lane >> 2), r1 = r0 + 8, c = (lane & 3) * 2;
 #pragma unroll
     for (int k = 0; k < HD / 16; ++k) {
@@ -181,6 +190,8 @@ struct AttWarp {
         const int d = kp * 32 + mid * 8, half = d >> 6, c = (d & 63) >> 3;
         const uint32_t addr = stage + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
         ldsm_x4(addr, kf[kp][n][0], kf[kp][n][1], kf[kp][n][2], kf[kp][n][3]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) kf[kp][n][e] = bf16x2_to_f16x2(kf[kp][n][e]);
       }
     }
     uint32_t vf[NT / 2][HD / 16][4];
@@ -193,6 +204,8 @@ struct AttWarp {
         const uint32_t addr =
             stage + 8192u + (uint32_t)((page * HB + half) * 2048 + r * 128 + ((c ^ (r & 7)) << 4));
         ldsm_x4_t(addr, vf[kk2][dp][0], vf[kk2][dp][1], vf[kk2][dp][2], vf[kk2][dp][3]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) vf[kk2][dp][e] = bf16x2_to_f16x2(vf[kk2][dp][e]);
       }
     }
     float s[NT][4];
@@ -216,10 +229,10 @@ struct AttWarp {
 #pragma unroll
     for (int kk2 = 0; kk2 < NT / 2; ++kk2) {
       uint32_t pa[4];
-      pa[0] = pack_bf16(s[2 * kk2][0], s[2 * kk2][1]);
-      pa[1] = pack_bf16(s[2 * kk2][2], s[2 * kk2][3]);
-      pa[2] = pack_bf16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
-      pa[3] = pack_bf16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
+      pa[0] = pack_f16(s[2 * kk2][0], s[2 * kk2][1]);
+      pa[1] = pack_f16(s[2 * kk2][2], s[2 * kk2][3]);
+      pa[2] = pack_f16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
+      pa[3] = pack_f16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
 #pragma unroll
       for (int dp = 0; dp < HD / 16; ++dp) {
         mma_16816(o[2 * dp], pa, vf[kk2][dp][0], vf[kk2][dp][1]);
@@ -228,9 +241,10 @@ struct AttWarp {
     }
   }
 
-  // The block's own rows: keys kq = 0..rows-1 at positions L + kq, read from the pages with plain
-  // loads (they were written earlier in this step).  Query row q = g*rows + j sees kq <= j.
-  // krow(kq) / vrow(kq) return the bf16 row pointers [HD].
+  // The block's own rows: keys kq = 0..rows-1 at positions L + kq, read with plain loads from the fp16
+  // copy written earlier in this step (the pages hold the same rows rounded to bf16 for later steps;
+  // reading the copy keeps 11 significant bits of the rows that weigh most when the cache is short).
+  // Query row q = g*rows + j sees kq <= j.  krow(kq) / vrow(kq) return the fp16 row pointers [HD].
   template <typename KFn, typename VFn>
   __device__ __forceinline__ void tail(KFn krow, VFn vrow, int rows, int row0, int nq, int lane) {
     const int q0 = row0 + (lane >> 2), q1 = q0 + 8;
@@ -243,7 +257,7 @@ struct AttWarp {
       for (int n = 0; n < NT; ++n) {
         const int key = kbase + n * 8 + (lane >> 2);
         if (kbase + n * 8 < rows) {   // warp-uniform
-          const bf16* kr = key < rows ? krow(key) : nullptr;
+          const __half* kr = key < rows ? krow(key) : nullptr;
 #pragma unroll
           for (int k = 0; k < HD / 16; ++k) {
             uint32_t b0 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2) : 0u;
@@ -265,15 +279,15 @@ struct AttWarp {
       for (int kk2 = 0; kk2 < NT / 2; ++kk2) {
         if (kbase + kk2 * 16 >= rows) continue;   // warp-uniform
         uint32_t pa[4];
-        pa[0] = pack_bf16(s[2 * kk2][0], s[2 * kk2][1]);
-        pa[1] = pack_bf16(s[2 * kk2][2], s[2 * kk2][3]);
-        pa[2] = pack_bf16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
-        pa[3] = pack_bf16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
+        pa[0] = pack_f16(s[2 * kk2][0], s[2 * kk2][1]);
+        pa[1] = pack_f16(s[2 * kk2][2], s[2 * kk2][3]);
+        pa[2] = pack_f16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
+        pa[3] = pack_f16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
         const int ka = kbase + kk2 * 16 + (lane & 3) * 2;   // keys ka, ka+1 (b0) and ka+8, ka+9 (b1)
-        const bf16* v00 = ka < rows ? vrow(ka) : nullptr;
-        const bf16* v01 = ka + 1 < rows ? vrow(ka + 1) : nullptr;
-        const bf16* v10 = ka + 8 < rows ? vrow(ka + 8) : nullptr;
-        const bf16* v11 = ka + 9 < rows ? vrow(ka + 9) : nullptr;
+        const __half* v00 = ka < rows ? vrow(ka) : nullptr;
+        const __half* v01 = ka + 1 < rows ? vrow(ka + 1) : nullptr;
+        const __half* v10 = ka + 8 < rows ? vrow(ka + 8) : nullptr;
+        const __half* v11 = ka + 9 < rows ? vrow(ka + 9) : nullptr;
 #pragma unroll
         for (int dn = 0; dn < HD / 8; ++dn) {
           const int d = dn * 8 + (lane >> 2);
@@ -338,7 +352,8 @@ __device__ __forceinline__ int att_find_seq(const int* pre, int B, int t) {
 }
 
 struct AttArgs {
-  const bf16* Qb;          // [B][Hkv][nq][HD] scaled queries
+  const __half* Qb;        // [B][Hkv][nq][HD] scaled queries (fp16)
+  const __half* KVn;       // [B][Hkv][2][rows][HD] this step's own key / value rows (fp16)
   AttPartials P;
   int n_tail_base;         // slot of tail (b, h): n_tail_base + b*Hkv + h
   int layer;
@@ -471,7 +486,7 @@ template <int HD, int NT>
 __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const AttPlan& pl, const AttGeom& g,
                                             const StepArgs* __restrict__ args, const KvView& kv, const AttArgs& a, int Hkv,
                                             int c, int G, int cw, int lane) {
-  const int B = args->B, rows = g.rows, n_active = g.MT * g.KS;
+  const int B = args->B, n_active = g.MT * g.KS;
   const int mi = cw / g.KS, ks = cw % g.KS, row0 = mi * 16;
   const long long T = pl.T;
   const long long t_lo = (long long)c * T / G, t_hi = (long long)(c + 1) * T / G;
@@ -519,20 +534,11 @@ __device__ __forceinline__ void att_tails(AttWarp<HD, NT>& st, const AttPlan& pl
   const int B = args->B, rows = g.rows;
   {
     for (int x = G - 1 - c; x < B * Hkv; x += G) {
-      const int b = x / Hkv, h = x % Hkv;
-      const int L = pl.L[b], seq = args->seq_ids[b];
       st.reset();
-      st.load_q(a.Qb + ((size_t)b * Hkv + h) * g.nq * HD, row0, g.nq, lane);
-      auto krow = [&](int kq) -> const bf16* {
-        const int pos = L + kq;
-        const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
-        return kv_row<bf16>(kv, a.layer, page, 0, h, pos % 16);
-      };
-      auto vrow = [&](int kq) -> const bf16* {
-        const int pos = L + kq;
-        const int page = __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pos / 16);
-        return kv_row<bf16>(kv, a.layer, page, 1, h, pos % 16);
-      };
+      st.load_q(a.Qb + (size_t)x * g.nq * HD, row0, g.nq, lane);
+      const __half* kn = a.KVn + (size_t)x * 2 * rows * HD;
+      auto krow = [&](int kq) -> const __half* { return kn + (size_t)kq * HD; };
+      auto vrow = [&](int kq) -> const __half* { return kn + (size_t)(rows + kq) * HD; };
       st.tail(krow, vrow, rows, row0, g.nq, lane);
       st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
     }

@@ -15,8 +15,10 @@ struct Work {
   // in the fp32 accumulator's epilogue.
   void* A;           // normalised activations (input of QKV / gate-up / LM head), K = d
   float* Q;          // [R, Hq*hd]    fp32 rotated queries
-  bf16* Qb;          // [B, Hkv, group*(gamma+1), hd] bf16 rotated queries times log2(e)/sqrt(hd), query row
+  __half* Qb;        // [B, Hkv, group*(gamma+1), hd] fp16 rotated queries times log2(e)/sqrt(hd), query row
                      // g*(gamma+1)+j of a KV head's group (tensor-core attention), or null
+  __half* KVn;       // [B, Hkv, 2 (K|V), gamma+1, hd] fp16 copy of this step's own key / value rows (the rows the
+                     // pages receive in bf16): the tensor-core attention reads the block's own rows from here
   void* ATT;         // attention output (input of the O projection), K = Hq*hd
   void* H;           // silu(gate)*up (input of the down projection), K = F
   float* P;          // partial sums of the current GEMM: [slot][R][N]
@@ -185,14 +187,19 @@ __global__ void k_qkv_rope(const StepArgs* __restrict__ args, KvView kv, Work w,
       if (w.Qb) {
         const int group = dm.Hq / dm.Hkv, j = r % rows;
         const float qs = 1.4426950408889634f / sqrtf((float)dm.hd);
-        bf16* qb = w.Qb + ((((size_t)b * dm.Hkv + head / group) * group + head % group) * rows + j) * dm.hd;
-        qb[i] = __float2bfloat16_rn(y1 * qs);
-        qb[i + half] = __float2bfloat16_rn(y2 * qs);
+        __half* qb = w.Qb + ((((size_t)b * dm.Hkv + head / group) * group + head % group) * rows + j) * dm.hd;
+        qb[i] = __float2half_rn(y1 * qs);
+        qb[i + half] = __float2half_rn(y2 * qs);
       }
     } else {
       T* krow = kv_row<T>(kv, layer, page, 0, head - dm.Hq, slot);
       krow[i] = from_f<T>(y1);
       krow[i + half] = from_f<T>(y2);
+      if (w.KVn) {
+        __half* kn = w.KVn + ((((size_t)b * dm.Hkv + head - dm.Hq) * 2) * rows + r % rows) * dm.hd;
+        kn[i] = __float2half_rn(y1);
+        kn[i + half] = __float2half_rn(y2);
+      }
     }
   }
   for (int p = threadIdx.x; p < kd; p += blockDim.x) {
@@ -200,6 +207,7 @@ __global__ void k_qkv_rope(const StepArgs* __restrict__ args, KvView kv, Work w,
     if (bv) x += to_f(bv[p]);
     T* vrow = kv_row<T>(kv, layer, page, 1, p / dm.hd, slot);
     vrow[p % dm.hd] = from_f<T>(x);
+    if (w.KVn) w.KVn[((((size_t)b * dm.Hkv + p / dm.hd) * 2 + 1) * rows + r % rows) * dm.hd + p % dm.hd] = __float2half_rn(x);
   }
 }
 

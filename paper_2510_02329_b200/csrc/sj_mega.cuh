@@ -114,6 +114,7 @@ struct MegaCtl {
   float inv[kMegaMaxRows];
   int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
   int row_qoff[kMegaMaxRows];         // element offset of row r's queries in the query buffer, without the head part
+  int row_nkvoff[kMegaMaxRows];       // element offset of row r in the fp16 copy of the step's own K/V rows, without head / K|V part
   long long row_kvoff[kMegaMaxRows];  // element offset of row r's slot in its cache page, without layer / K|V / head part
   float red[4][16];
   RowStat wstat[4][16];
@@ -517,16 +518,20 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         // query row (b, kvh, g, j) sits at ((b*Hq + head)*rows + j)*HD; a cache row at
         // ((((layer*n_pages + page)*2 + K|V)*Hkv + head)*page_size + slot)*HD: the per-row parts are tabulated
         if (kind == 0) {
-          bf16* qb = w.Qb + (size_t)head * rows * HD + dim;
+          __half* qb = w.Qb + (size_t)head * rows * HD + dim;
 #pragma unroll
           for (int i = 0; i < 16; ++i)
-            if (c0 + i < R) qb[ctl->row_qoff[c0 + i]] = __float2bfloat16_rn(v[i] * qscale);
+            if (c0 + i < R) qb[ctl->row_qoff[c0 + i]] = __float2half_rn(v[i] * qscale);
         } else {
           bf16* kvb = reinterpret_cast<bf16*>(kv.pool) +
                       ((size_t)l * kv.n_pages * 2 * dm.Hkv + (size_t)(kind - 1) * dm.Hkv + head) * kv.page_size * HD + dim;
 #pragma unroll
           for (int i = 0; i < 16; ++i)
             if (c0 + i < R) kvb[ctl->row_kvoff[c0 + i]] = __float2bfloat16_rn(v[i]);
+          __half* kn = w.KVn + (size_t)(head * 2 + kind - 1) * rows * HD + dim;
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (c0 + i < R) kn[ctl->row_nkvoff[c0 + i]] = __float2half_rn(v[i]);
         }
       } else if (site == SITE_O || site == SITE_DOWN) {
         const int f = tile * kTileN + fl;
@@ -810,6 +815,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     ctl->row_slot[r] = pos % kv.page_size;
     ctl->tgt_tok[r] = (j < gamma) ? args->draft_ids[b * gamma + j] : -1;
     ctl->row_qoff[r] = (b * dm.Hq * rows + j) * dm.hd;
+    ctl->row_nkvoff[r] = (b * dm.Hkv * 2 * rows + j) * dm.hd;
     ctl->row_kvoff[r] = ((long long)ctl->row_page[r] * 2 * dm.Hkv * kv.page_size + ctl->row_slot[r]) * dm.hd;
   }
   __syncthreads();
@@ -1007,7 +1013,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
                                      ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8
                                      : nullptr;
         AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status, ev};
-        AttArgs aa{w.Qb, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
+        AttArgs aa{w.Qb, w.KVn, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
         int it2 = it;
         att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
       }

@@ -214,3 +214,28 @@ def test_bit_reproducible_across_runs():
             assert np.array_equal(a[k], c[k]), k
     finally:
         case.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# full-width cuts of the benchmark shapes (all widths, head counts and the vocabulary as configured;
+# fewer layers and a short synthetic cache so that the fp64 oracle finishes in seconds)
+# ------------------------------------------------------------------------------------------------
+WIDTH_CASES = [
+    ("llama-1b-cut2", synth.LLAMA_1B.cut(2), [300], 8),            # tied embeddings, head_dim 64, group 4
+    ("llama-8b-cut2", synth.LLAMA_8B.cut(2), [210], 8),            # config 3's widths
+    ("llama-8b-cut1-g16", synth.LLAMA_8B.cut(1), [77], 16),        # 17 rows: two 16-column accumulator chunks
+    ("qwen-32b-cut1-b8", synth.QWEN_32B.cut(1), [40, 97, 16, 130, 64, 33, 250, 5], 8),   # 72 rows, qkv bias, F 27648
+]
+
+
+@pytest.mark.parametrize("name,shape,kv_lens,gamma", WIDTH_CASES, ids=[c[0] for c in WIDTH_CASES])
+def test_full_width_cuts_of_the_benchmark_shapes(name, shape, kv_lens, gamma):
+    case = harness.Case(shape, torch.bfloat16, kv_lens, gamma, seed=5, cache="fill", gen_device="cuda").gpu_setup(
+        max_rows=len(kv_lens) * (gamma + 1))
+    try:
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 1.0)]:
+            rep, _ = _run(case, mode, T)
+            assert rep.exact + rep.margin == len(kv_lens)
+            print(name, "mode", mode, rep)
+    finally:
+        case.close()
