@@ -72,10 +72,13 @@ struct MegaParams {
   const bf16* embed;
   const bf16* gain0;          // first layer's attention-norm gain
   float* sumsq;               // [2][d/128][kMegaMaxRows]
-  float* pbuf;                // [blocks][Rp][128] split-K partial sums
+  // Split-K partial sums, [blocks][Rp][128] words of 64 bits: the fp32 value in the low half and, in the
+  // high half, the number of the GEMM phase that wrote it (1, 2, ... within a launch).  A word is stored and
+  // loaded as one 64-bit access, so a reader that sees the phase number it expects also sees the value:
+  // no flag, no fence, and the reader polls the data itself.
+  unsigned long long* pbuf;   //                               }
   unsigned* gbar;             // device-wide barrier counter   } zeroed before every launch
   int* abort_g;               // device-wide abort word        }
-  int* flags;                 // [blocks] split-K flags        }
   int n_tail_base;
   // optional timeline of block 0 (global-timer nanoseconds):
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
@@ -83,6 +86,7 @@ struct MegaParams {
   //   load issued, 2 first stage ready at the MMA issuer, 3 last MMA committed, 4 last accumulator seen by the
   //   epilogue, 5 split-K contributors' flags seen, 6 epilogue done, 7 weight producer issued the last load
   unsigned long long* trace;
+  unsigned trace_block;       // the block that writes the timeline
 };
 
 __device__ __forceinline__ unsigned long long global_timer_ns() {
@@ -90,9 +94,14 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
   return t;
 }
+#define MEGA_EVA(sidx, k)                                                                            \
+  do {                                                                                               \
+    if (p.trace && (sidx) < 16)                                                                      \
+      p.trace[2 * kMegaTraceBarriers + 16 * kMegaTraceSites + ((sidx) * 256 + blockIdx.x) * 4 + (k)] = global_timer_ns(); \
+  } while (0)
 #define MEGA_EV(sidx, k)                                                                             \
   do {                                                                                               \
-    if (p.trace && blockIdx.x == 0 && (sidx) < kMegaTraceSites)                                      \
+    if (p.trace && blockIdx.x == p.trace_block && (sidx) < kMegaTraceSites)                                      \
       p.trace[2 * kMegaTraceBarriers + (sidx) * 8 + (k)] = global_timer_ns();                        \
   } while (0)
 
@@ -100,7 +109,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // owner-side ones, at [2*kMegaTraceBarriers + 8*kMegaTraceSites + 8*s + e]
 #define MEGA_EV2(blk, sidx, k)                                                                       \
   do {                                                                                               \
-    if (p.trace && blockIdx.x == (blk) && (sidx) < kMegaTraceSites)                                  \
+    if (p.trace && blockIdx.x == p.trace_block + (blk) && (sidx) < kMegaTraceSites)                                  \
       p.trace[2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (sidx) * 8 + (k)] = global_timer_ns();  \
   } while (0)
 
@@ -110,20 +119,20 @@ struct MegaCtl {
   uint32_t tmem_base;
   int abort_flag;
   int bars_passed;
-  int bcast[4];
+  int bcast[6];   // [2 * group + accumulator]: the group's wait on that accumulator succeeded; [4], [5] spare
   float inv[kMegaMaxRows];
   int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
   int row_qoff[kMegaMaxRows];         // element offset of row r's queries in the query buffer, without the head part
   int row_nkvoff[kMegaMaxRows];       // element offset of row r in the fp16 copy of the step's own K/V rows, without head / K|V part
   long long row_kvoff[kMegaMaxRows];  // element offset of row r's slot in its cache page, without layer / K|V / head part
-  float red[4][16];
-  RowStat wstat[4][16];
+  float red[2][4][8];          // [group][warp][row of the chunk]
+  RowStat wstat[2][4][8];
   RowStat rs[kMaxGamma + 1];
   float score[kMaxGamma + 1];
   AttPlan plan;
   int att_pages[kAttPageCache];   // page ids of this block's first ring tiles (the same in every layer)
   union {
-    float exch[128][17];
+    float exch[2][128][9];      // [group][feature][row of the chunk]
     RowStat sred[kMegaWorkers];
   } u;
 };
@@ -256,8 +265,13 @@ __device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
 __device__ __forceinline__ void red_relaxed_add(unsigned* p, unsigned v) {
   asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void st_relaxed_s32(int* p, int v) {
-  asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
 }
 
 // Bounded wait on a shared-memory barrier that also watches the device-wide abort word.
@@ -294,7 +308,7 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
   bar_sync(1, kMegaWorkers);
   ++nbar;
   if (wt == 0) {
-    const bool tr = p.trace && blockIdx.x == 0 && nbar < kMegaTraceBarriers;
+    const bool tr = p.trace && blockIdx.x == p.trace_block && nbar < kMegaTraceBarriers;
     if (tr) p.trace[2 * nbar] = global_timer_ns();
     if (!ctl->abort_flag) {
       __threadfence();
@@ -303,6 +317,7 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
     }
     __threadfence();
     if (tr) p.trace[2 * nbar + 1] = global_timer_ns();
+    if (p.trace && nbar < 32) p.trace[2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + nbar * 256 + blockIdx.x] = global_timer_ns();
     *reinterpret_cast<volatile int*>(&ctl->bars_passed) = nbar;
   }
   bar_sync(1, kMegaWorkers);
@@ -347,11 +362,17 @@ __device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int l
 }
 
 // ---------------------------------------------------------------------------------------------
-// fused epilogues (the four epilogue warps: 128 threads, named barrier 2)
+// fused epilogues.  All eight worker warps take part, as two groups of four warps (a warp reads the
+// accumulator lanes 32 * (warp % 4) .. + 31, so either group covers the tile's 128 features): the block
+// rows are cut into chunks of eight accumulator columns, group 0 takes the even chunks and group 1 the odd
+// ones.  One warp per scheduler runs a long dependent instruction chain at a fraction of an instruction
+// per cycle, so halving the rows per thread nearly halves the time between the last MMA and the barrier.
+// Each group has its own named barrier (2 + group, 128 threads) and its own exchange buffers.
 // ---------------------------------------------------------------------------------------------
 template <int HD>
 __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
-                                              const Work& w, const Dims& dm, int et) {
+                                              const Work& w, const Dims& dm, int wt) {
+  const int et = wt & 127, grp = wt >> 7, bar_id = 2 + grp;
   const int sidx = gseq - 1;
   const int R = p.R, Rp = p.Rp, rows = p.rows;
   const int quarter = et >> 5, lane = et & 31;
@@ -371,17 +392,17 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       for (int k = 0; k < 4; ++k) {
         const int r = r0 + 4 * k;
         part[k] = 0.f;
-        if (r < R)
+        if (r < R && ((r >> 3) & 1) == grp)
           for (int t = lane; t < nt128; t += 32) part[k] += __ldcg(p.sumsq + ((size_t)buf * nt128 + t) * kMegaMaxRows + r);
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int r = r0 + 4 * k;
         const float s = warp_sum(part[k]);
-        if (lane == 0 && r < R) ctl->inv[r] = 1.0f / sqrtf(s / (float)dm.d + dm.eps);
+        if (lane == 0 && r < R && ((r >> 3) & 1) == grp) ctl->inv[r] = 1.0f / sqrtf(s / (float)dm.d + dm.eps);
       }
     }
-    bar_sync(2, 128);
+    bar_sync(bar_id, 128);
   }
   const int qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd, tq = qd / kTileN, tk = kd / kTileN;
   const float invT = (site == SITE_LM) ? args->inv_temperature : 1.f;
@@ -416,103 +437,121 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     }
 
     const bool owner = (kb0 == 0), complete = owner && (sg.len == ss.KB);
-    int c_last = c;
-    // An owner first makes sure the other groups that share the tile have published (often they did
-    // long ago: their share of this tile was the first thing they computed), then waits for its own sums.
-    if (owner && !complete) {
-      c_last = unit_owner((unsigned)(tile + 1) * (unsigned)ss.KB - 1u, U, G);
-      if (et < 32) {   // one lane per contributing group
-        int ok = 1;
-        for (int base = c + 1; base <= c_last; base += 32) {
-          const int c2 = base + lane;
-          int okl = 1;
-          if (c2 <= c_last && has_units(c2, U, G))   // groups without units add nothing
-            okl = mega_spin_ge(reinterpret_cast<const unsigned*>(p.flags + c2), (unsigned)gseq, ctl, p, w.status, 7, gseq) ? 1 : 0;
-          ok &= __all_sync(0xffffffffu, okl);
-        }
-        __threadfence();
-        if (et == 0) ctl->bcast[2] = ok;
-      }
-      bar_sync(2, 128);
-      if (!ctl->bcast[2]) return;
-      if (et == 0) MEGA_EV(sidx, 5);
-    }
+    int c_last = c;   // last of the groups that share this tile
+    if (owner && !complete) c_last = unit_owner((unsigned)(tile + 1) * (unsigned)ss.KB - 1u, U, G);
     if (et == 0) {
       int ok = 1;
       if (mine) ok = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
-      ctl->bcast[seg & 1] = ok;
+      ctl->bcast[2 * grp + (seg & 1)] = ok;
     }
-    bar_sync(2, 128);
-    if (!ctl->bcast[seg & 1]) return;
+    bar_sync(bar_id, 128);
+    if (!ctl->bcast[2 * grp + (seg & 1)]) return;
     tc_fence_after();
     if (et == 0) MEGA_EV(sidx, 4);
 
-    for (int c0 = 0; c0 < Rp; c0 += 16) {
-      float v[16], xs[16];
-      float2 cs[16];
+    for (int c0 = 8 * grp; c0 < Rp; c0 += 16) {
+      float v[8], xs[8];
+      float2 cs[8];
       // every global load of this chunk is issued before anything waits on one of them
       if (owner && (site == SITE_O || site == SITE_DOWN)) {   // residual rows
         const int f = tile * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) xs[i] = (c0 + i < R) ? __ldcg(w.X + (size_t)(c0 + i) * dm.d + f) : 0.f;
+        for (int i = 0; i < 8; ++i) xs[i] = __ldcg(w.X + (size_t)min(c0 + i, R - 1) * dm.d + f);   // unpredicated: rows past R repeat the last row
       }
       if (owner && site == SITE_QKV && kind < 2) {            // rotary table rows
         const int ii = dim & (HD / 2 - 1);
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-          cs[i] = (c0 + i < R) ? __ldcg(w.rope + (size_t)(c0 + i) * (HD / 2) + ii) : make_float2(1.f, 0.f);
+        for (int i = 0; i < 8; ++i)
+          cs[i] = __ldcg(w.rope + (size_t)min(c0 + i, R - 1) * (HD / 2) + ii);
       }
       if (mine) {
-        float lo[16];
-        tc_ld16(taddr + c0, v);
-        tc_ld16(taddr + Rp + c0, lo);
+        float lo[8];
+        tc_ld8(taddr + c0, v);
+        tc_ld8(taddr + Rp + c0, lo);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] += lo[i];
+        for (int i = 0; i < 8; ++i) v[i] += lo[i];
       } else {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
       }
-      if (!owner) {
-        float* dst = p.pbuf + ((size_t)c * Rp + c0) * kTileN + fl;
+      const unsigned long long tag = (unsigned long long)(unsigned)gseq << 32;
+      if (et == 0 && owner) MEGA_EV2(0, sidx, 0);
+      if (!owner) {   // publish the partial sums, each with this phase's number
+        unsigned long long* dst = p.pbuf + ((size_t)c * Rp + c0) * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-          if (c0 + i < R) dst[(size_t)i * kTileN] = v[i];
+        for (int i = 0; i < 8; ++i)
+          if (c0 + i < R) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
         continue;
       }
-      for (int cb = c + 1; cb <= c_last; cb += 4) {   // four contributing groups' loads in flight at a time, added in group order
-        float pv[4][16];
+      // The other blocks' shares of this tile: two blocks' words in flight at a time, all of them reloaded
+      // until every one carries this phase's number, then added in group order (so the sum does not depend
+      // on arrival order).  Often they were published long ago: a group's share of somebody else's tile is
+      // the first thing it computes.  A wait that runs out raises the abort word and goes on with whatever
+      // it read (the block leaves together at its next block-wide check).
+      for (int cb = c + 1; cb <= c_last; cb += 2) {
+        unsigned long long pw[2][8];
+        const unsigned long long* src[2];
+        bool live[2];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < 2; ++k) {
           const int c2 = cb + k;
-          const bool live = c2 <= c_last && has_units(c2, U, G);
-          const float* src = p.pbuf + ((size_t)(live ? c2 : c) * Rp + c0) * kTileN + fl;
+          live[k] = c2 <= c_last && has_units(c2, U, G);   // groups without units add nothing
+          src[k] = p.pbuf + ((size_t)(live[k] ? c2 : c) * Rp + c0) * kTileN + fl;
+        }
+        volatile int* af = &ctl->abort_flag;
+        const int nr = min(8, R - c0);
+        for (uint32_t spin = 0;; ++spin) {
+          bool ok = true;
+          // every load is issued before any result is looked at: rows past R read row 0 again (in
+          // bounds, ignored below) instead of being predicated off, which would put a select after each load
 #pragma unroll
-          for (int i = 0; i < 16; ++i) pv[k][i] = (live && c0 + i < R) ? __ldcg(src + (size_t)i * kTileN) : 0.f;
+          for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) pw[k][i] = ld_relaxed_u64(src[k] + (size_t)(i < nr ? i : 0) * kTileN);
+#pragma unroll
+          for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ok = ok && (!live[k] || i >= nr || (pw[k][i] >> 32) == (tag >> 32));
+          if (ok) break;
+          if (spin > 16) {
+            if (*af) break;
+            if ((spin & 63) == 0 && *reinterpret_cast<volatile int*>(p.abort_g)) { *af = 1; break; }
+            if (spin > 4096) __nanosleep(64);
+            if (spin >= kMegaSpin) {
+              *af = 1;
+              att_note_timeout(p.abort_g, 7, gseq);
+              *reinterpret_cast<volatile int*>(p.abort_g) = 1;
+              atomicCAS(w.status, DEV_OK, DEV_TIMEOUT);
+              break;
+            }
+          }
         }
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < 2; ++k)
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] += pv[k][i];
+          for (int i = 0; i < 8; ++i) v[i] += (live[k] && i < nr) ? __uint_as_float((unsigned)pw[k][i]) : 0.f;
       }
-      if (et == 0) MEGA_EV2(0, sidx, 5);
+      if (et == 0) MEGA_EV(sidx, 5);
+      if (et == 0) MEGA_EV2(0, sidx, 1);
+      if (et == 0 && owner && c_last > c) MEGA_EVA(sidx, 2);
       if (site == SITE_QKV) {
         const int half = HD / 2;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
           v[i] = v[i] * (r < R ? ctl->inv[r] : 0.f) + bias;
         }
         if (kind < 2) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) ctl->u.exch[fl][i] = v[i];
-          bar_sync(2, 128);
+          for (int i = 0; i < 8; ++i) ctl->u.exch[grp][fl][i] = v[i];
+          bar_sync(bar_id, 128);
           const bool first = dim < half;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float xp = ctl->u.exch[fl ^ half][i];
+          for (int i = 0; i < 8; ++i) {
+            const float xp = ctl->u.exch[grp][fl ^ half][i];
             v[i] = first ? v[i] * cs[i].x - xp * cs[i].y : v[i] * cs[i].x + xp * cs[i].y;
           }
-          bar_sync(2, 128);
+          bar_sync(bar_id, 128);
         }
         if (et == 0) MEGA_EV2(0, sidx, 6);
         // query row (b, kvh, g, j) sits at ((b*Hq + head)*rows + j)*HD; a cache row at
@@ -520,25 +559,25 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         if (kind == 0) {
           __half* qb = w.Qb + (size_t)head * rows * HD + dim;
 #pragma unroll
-          for (int i = 0; i < 16; ++i)
+          for (int i = 0; i < 8; ++i)
             if (c0 + i < R) qb[ctl->row_qoff[c0 + i]] = __float2half_rn(v[i] * qscale);
         } else {
           bf16* kvb = reinterpret_cast<bf16*>(kv.pool) +
                       ((size_t)l * kv.n_pages * 2 * dm.Hkv + (size_t)(kind - 1) * dm.Hkv + head) * kv.page_size * HD + dim;
 #pragma unroll
-          for (int i = 0; i < 16; ++i)
+          for (int i = 0; i < 8; ++i)
             if (c0 + i < R) kvb[ctl->row_kvoff[c0 + i]] = __float2bfloat16_rn(v[i]);
           __half* kn = w.KVn + (size_t)(head * 2 + kind - 1) * rows * HD + dim;
 #pragma unroll
-          for (int i = 0; i < 16; ++i)
+          for (int i = 0; i < 8; ++i)
             if (c0 + i < R) kn[ctl->row_nkvoff[c0 + i]] = __float2half_rn(v[i]);
         }
       } else if (site == SITE_O || site == SITE_DOWN) {
         const int f = tile * kTileN + fl;
         const int buf = (site == SITE_O) ? 1 : 0;
-        float ss[16];
+        float ss[8];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
           ss[i] = 0.f;
           if (r < R) {
@@ -548,45 +587,47 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
             ss[i] = x * x;
           }
         }
+        if (et == 0) MEGA_EV2(0, sidx, 2);
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 8; ++i)
           if (c0 + i < R) ss[i] = warp_sum(ss[i]);   // block-uniform
         if (lane == 0) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) ctl->red[quarter][i] = ss[i];
+          for (int i = 0; i < 8; ++i) ctl->red[grp][quarter][i] = ss[i];
         }
-        bar_sync(2, 128);
-        if (et < 16 && c0 + et < R)
+        bar_sync(bar_id, 128);
+        if (et < 8 && c0 + et < R)
           p.sumsq[((size_t)buf * nt128 + tile) * kMegaMaxRows + c0 + et] =
-              ctl->red[0][et] + ctl->red[1][et] + ctl->red[2][et] + ctl->red[3][et];
-        bar_sync(2, 128);
+              ctl->red[grp][0][et] + ctl->red[grp][1][et] + ctl->red[grp][2][et] + ctl->red[grp][3][et];
+        bar_sync(bar_id, 128);
+        if (et == 0) MEGA_EV2(0, sidx, 3);
       } else if (site == SITE_GU) {
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
           v[i] *= (r < R ? ctl->inv[r] : 0.f);
         }
         if (fl >= 64) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) ctl->u.exch[fl - 64][i] = v[i];
+          for (int i = 0; i < 8; ++i) ctl->u.exch[grp][fl - 64][i] = v[i];
         }
-        bar_sync(2, 128);
+        bar_sync(bar_id, 128);
         if (fl < 64) {
           const int f = tile * 64 + fl;
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
+          for (int i = 0; i < 8; ++i) {
             const int r = c0 + i;
             if (r < R) {
-              const float g = v[i], up = ctl->u.exch[fl][i];
+              const float g = v[i], up = ctl->u.exch[grp][fl][i];
               store_act<bf16>(w.H, R, dm.F, r, f, g / (1.0f + expf(-g)) * up);
             }
           }
         }
-        bar_sync(2, 128);
+        bar_sync(bar_id, 128);
       } else {   // LM head
         const int n = tile * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
+        for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
           float z = -INFINITY;
           if (r < R && n < dm.V) {
@@ -608,18 +649,18 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           e = warp_sum(e);
           if (lane == 0) {
             RowStat st; st.m = m; st.s = e; st.arg = arg; st.pad = 0;
-            ctl->wstat[quarter][i] = st;
+            ctl->wstat[grp][quarter][i] = st;
           }
         }
-        bar_sync(2, 128);
-        if (et < 16 && c0 + et < R) {
-          RowStat a = ctl->wstat[0][et];
-          a = stat_merge(a, ctl->wstat[1][et]);
-          a = stat_merge(a, ctl->wstat[2][et]);
-          a = stat_merge(a, ctl->wstat[3][et]);
+        bar_sync(bar_id, 128);
+        if (et < 8 && c0 + et < R) {
+          RowStat a = ctl->wstat[grp][0][et];
+          a = stat_merge(a, ctl->wstat[grp][1][et]);
+          a = stat_merge(a, ctl->wstat[grp][2][et]);
+          a = stat_merge(a, ctl->wstat[grp][3][et]);
           w.stats[(size_t)tile * R + c0 + et] = a;
         }
-        bar_sync(2, 128);
+        bar_sync(bar_id, 128);
       }
     }
     if (et == 0) MEGA_EV2(0, sidx, 7);
@@ -628,15 +669,9 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
       ++seg;
     }
-    if (!owner) {   // publish the partial: block barrier, then one cumulative fence and the flag
-      bar_sync(2, 128);
-      if (et == 0) {
-        __threadfence();
-        st_relaxed_s32(p.flags + c, gseq);
-      }
-    }
   }
   if (et == 0) MEGA_EV(sidx, 6);
+  if (et == 0) MEGA_EVA(sidx, 3);
 }
 
 // a1 + first a2: embedding gather, fp32 residual stream, first GEMM input planes, sums of squares, and
@@ -782,7 +817,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
-      mbar_init(smem_u32(&ctl->tmem_empty[i]), 128);
+      mbar_init(smem_u32(&ctl->tmem_empty[i]), kMegaWorkers);
     }
     ctl->abort_flag = 0;
     ctl->bars_passed = 0;
@@ -935,6 +970,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           ++seg;
         }
         MEGA_EV(sidx, 3);
+        MEGA_EVA(sidx, 0);
         ++sidx;
       };
       auto fatt = [&](int l) { rp.advance(n_att); };
@@ -994,7 +1030,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     auto units = [&](int site) -> int { return site_units(site_split(site, dm, c, G)); };
     auto gemm_phase = [&](int site, int l) {
       ++gseq;
-      if (alive && ww < 4) mega_epilogue<HD>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
+      if (alive) mega_epilogue<HD>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
       it += units(site);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     };
