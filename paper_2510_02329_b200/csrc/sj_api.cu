@@ -419,7 +419,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     const int Rm = std::min(R, kMegaMaxRows);
     ALLOC(t->d_layer_ptrs, MegaLayerPtrs, c.n_layers);
     ALLOC(t->d_sumsq, float, (size_t)2 * (c.d_model / kTileN) * kMegaMaxRows);
-    ALLOC(t->d_sync, unsigned, 64 + (size_t)2 * t->sm_count * pad16(Rm) * kTileN);
+    ALLOC(t->d_sync, unsigned, 64 + (size_t)4 * t->sm_count * pad16(Rm) * kTileN);
     std::vector<MegaLayerPtrs> lp(c.n_layers);
     for (int l = 0; l < c.n_layers; ++l) {
       const LayerW& L = t->layers[l];
@@ -429,7 +429,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     }
     cudaError_t e = cudaMemcpy(t->d_layer_ptrs, lp.data(), lp.size() * sizeof(MegaLayerPtrs), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(t->d_sumsq, 0, sizeof(float) * 2 * (c.d_model / kTileN) * kMegaMaxRows);
-    if (e == cudaSuccess) e = cudaMemset(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)2 * t->sm_count * pad16(Rm) * kTileN));
+    if (e == cudaSuccess) e = cudaMemset(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)4 * t->sm_count * pad16(Rm) * kTileN));
     if (e == cudaSuccess)
       e = c.head_dim == 128
               ? cudaFuncSetAttribute(k_verify_mega<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
@@ -511,7 +511,7 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
   } else if (n == "trace") {
-    const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192;
+    const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192 + 8192;
     if (value && !t->d_trace) {
       sj_status st = dev_alloc(t, &t->d_trace, n_tr);
       if (st != SJ_OK) return st;
@@ -979,7 +979,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
     MegaMaps mm = t->mega_maps[ci];
     mm.pool = kv->tm_pool;
     mm.a_d = *mA_d; mm.a_q = *mA_q; mm.a_f = *mA_f;
-    CU_TRY(cudaMemsetAsync(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)2 * t->sm_count * Rp * kTileN), s));
+    CU_TRY(cudaMemsetAsync(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)4 * t->sm_count * Rp * kTileN), s));
     cudaEvent_t ea = nullptr, eb = nullptr;
     if (timing) {
       CU_TRY(cudaEventCreate(&ea));
@@ -1013,7 +1013,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
 extern "C" sj_status sj_step_trace(sj_target* t, unsigned long long* out_ns, int max_entries, int* n_entries) {
   if (!t || !out_ns || !n_entries || max_entries <= 0) return fail(SJ_ERR_INVALID_ARG, "null argument");
   if (!t->d_trace) return fail(SJ_ERR_STATE, "tracing was never enabled (sj_set_option \"trace\")");
-  const int n = std::min(max_entries, 2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192);
+  const int n = std::min(max_entries, 2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192 + 8192);
   CU_TRY(cudaStreamSynchronize(t->stream));
   CU_TRY(cudaMemcpy(out_ns, t->d_trace, sizeof(unsigned long long) * n, cudaMemcpyDeviceToHost));
   *n_entries = n;

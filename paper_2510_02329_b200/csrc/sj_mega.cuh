@@ -76,6 +76,7 @@ struct MegaParams {
   // high half, the number of the GEMM phase that wrote it (1, 2, ... within a launch).  A word is stored and
   // loaded as one 64-bit access, so a reader that sees the phase number it expects also sees the value:
   // no flag, no fence, and the reader polls the data itself.
+  // Two slots per block ([block][2][Rp][128]): slot 1 for the tile whose first K block it holds, slot 0 otherwise.
   unsigned long long* pbuf;   //                               }
   unsigned* gbar;             // device-wide barrier counter   } zeroed before every launch
   int* abort_g;               // device-wide abort word        }
@@ -310,6 +311,7 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
   if (wt == 0) {
     const bool tr = p.trace && blockIdx.x == p.trace_block && nbar < kMegaTraceBarriers;
     if (tr) p.trace[2 * nbar] = global_timer_ns();
+    if (p.trace && nbar < 32) p.trace[2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192 + nbar * 256 + blockIdx.x] = global_timer_ns();
     if (!ctl->abort_flag) {
       __threadfence();
       red_relaxed_add(p.gbar, 1u);
@@ -410,6 +412,8 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
   const float qscale = 1.4426950408889634f / sqrtf((float)HD);
   const int fl = et;   // feature inside the tile == TMEM lane
 
+  int n_rs = 0, rs_tile0 = 0, rs_first0 = 0, rs_last0 = 0, rs_tile1 = 0, rs_first1 = 0, rs_last1 = 0;
+  float rs_gn0 = 1.f, rs_gn1 = 1.f;
   unsigned u = ss.g_lo;
   Seg sg;
   while (seg_next(ss, u, sg)) {
@@ -436,9 +440,16 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       gn = __bfloat162float(lp.gain_next[tile * kTileN + fl]);
     }
 
-    const bool owner = (kb0 == 0), complete = owner && (sg.len == ss.KB);
-    int c_last = c;   // last of the groups that share this tile
-    if (owner && !complete) c_last = unit_owner((unsigned)(tile + 1) * (unsigned)ss.KB - 1u, U, G);
+    const bool complete = (kb0 == 0) && (sg.len == ss.KB);
+    // The O and down projections split a shared tile's epilogue by ROWS: the n blocks that hold K ranges of
+    // the tile each finish R / n of its rows (all 128 features of them) and publish their sums of the other
+    // rows, instead of one block finishing the whole tile while the others idle at the barrier.  (Needs every
+    // block to hold units, so that the sharing blocks are consecutive.)
+    const bool rowsplit = (site == SITE_O || site == SITE_DOWN) && !complete && U >= (unsigned)G;
+    const bool owner = (kb0 == 0) && !rowsplit;
+    int c_first = c, c_last = c;   // first and last of the blocks that share this tile
+    if ((owner && !complete) || rowsplit) c_last = unit_owner((unsigned)(tile + 1) * (unsigned)ss.KB - 1u, U, G);
+    if (rowsplit) c_first = unit_owner((unsigned)tile * (unsigned)ss.KB, U, G);
     if (et == 0) {
       int ok = 1;
       if (mine) ok = mega_wait(smem_u32(&ctl->tmem_full[acc]), use & 1, ctl, p, w.status, 6, gseq) ? 1 : 0;
@@ -476,8 +487,15 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       }
       const unsigned long long tag = (unsigned long long)(unsigned)gseq << 32;
       if (et == 0 && owner) MEGA_EV2(0, sidx, 0);
+      if (rowsplit) {   // publish every row; the rows are finished after the loop over the segments
+        unsigned long long* dst = p.pbuf + ((size_t)(2 * c + (c == c_first ? 1 : 0)) * Rp + c0) * kTileN + fl;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (c0 + i < R) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
+        continue;
+      }
       if (!owner) {   // publish the partial sums, each with this phase's number
-        unsigned long long* dst = p.pbuf + ((size_t)c * Rp + c0) * kTileN + fl;
+        unsigned long long* dst = p.pbuf + ((size_t)(2 * c) * Rp + c0) * kTileN + fl;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
           if (c0 + i < R) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
@@ -496,7 +514,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         for (int k = 0; k < 2; ++k) {
           const int c2 = cb + k;
           live[k] = c2 <= c_last && has_units(c2, U, G);   // groups without units add nothing
-          src[k] = p.pbuf + ((size_t)(live[k] ? c2 : c) * Rp + c0) * kTileN + fl;
+          src[k] = p.pbuf + ((size_t)(2 * (live[k] ? c2 : c)) * Rp + c0) * kTileN + fl;
         }
         volatile int* af = &ctl->abort_flag;
         const int nr = min(8, R - c0);
@@ -668,6 +686,94 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
       ++seg;
+    }
+    if (rowsplit) {   // at most two per phase: the block's first and last segment
+      if (n_rs == 0) { rs_tile0 = tile; rs_first0 = c_first; rs_last0 = c_last; rs_gn0 = gn; }
+      else { rs_tile1 = tile; rs_first1 = c_first; rs_last1 = c_last; rs_gn1 = gn; }
+      ++n_rs;
+    }
+  }
+  // Row-split tiles (O and down projections): this block's rows of each shared tile.  Every sharing block
+  // has published all its rows by now or will without waiting for anybody (publishing comes first in every
+  // block), so the waits below cannot form a chain.  A row's sums are added in block order.
+#pragma unroll 1
+  for (int q = 0; q < n_rs; ++q) {
+    const int tile = q ? rs_tile1 : rs_tile0, c_first = q ? rs_first1 : rs_first0, c_last = q ? rs_last1 : rs_last0;
+    const float gn = q ? rs_gn1 : rs_gn0;
+    const int n = c_last - c_first + 1, j = c - c_first;
+    const int f = tile * kTileN + fl;
+    const int buf = (site == SITE_O) ? 1 : 0;
+    const unsigned long long tag = (unsigned long long)(unsigned)gseq << 32;
+    volatile int* af = &ctl->abort_flag;
+#pragma unroll 1
+    for (int c0 = 8 * grp; c0 < Rp; c0 += 16) {
+      // Rows are dealt with weight 1 to the first and the last sharing block and weight 2 to the others:
+      // the first block of one tile is as a rule the last block of the tile before, and finishes rows of both.
+      const int wsum = 2 * n - 2, w_lo = j == 0 ? 0 : 2 * j - 1, w_hi = j == n - 1 ? wsum : 2 * j + 1;
+      const int a = max(w_lo * R / wsum - c0, 0), b = min(w_hi * R / wsum - c0, min(8, R - c0));   // this block's rows of the chunk: [a, b)
+#pragma unroll 1
+      for (int i = a; i < b; i += 2) {   // two rows at a time: their loads share one round trip
+        const int i1 = min(i + 1, b - 1);   // == i when the second row is absent: it repeats the first
+        const int r0 = c0 + i, r1 = c0 + i1;
+        const float x0 = __ldcg(w.X + (size_t)r0 * dm.d + f), x1 = __ldcg(w.X + (size_t)r1 * dm.d + f);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll 1
+        for (int k0 = 0; k0 < n; k0 += 6) {   // the sharing blocks (this one included), six at a time
+          unsigned long long pw[2][6];
+          const unsigned long long* src[6];
+#pragma unroll
+          for (int k = 0; k < 6; ++k) {
+            const int c2 = c_first + min(k0 + k, n - 1);   // past the last one: it is read again and ignored
+            src[k] = p.pbuf + ((size_t)(2 * c2 + (c2 == c_first ? 1 : 0)) * Rp + c0) * kTileN + fl;
+          }
+          for (uint32_t spin = 0;; ++spin) {
+            bool ok = true;
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+              pw[0][k] = ld_relaxed_u64(src[k] + (size_t)i * kTileN);
+              pw[1][k] = ld_relaxed_u64(src[k] + (size_t)i1 * kTileN);
+            }
+#pragma unroll
+            for (int k = 0; k < 6; ++k) ok = ok && (pw[0][k] >> 32) == (tag >> 32) && (pw[1][k] >> 32) == (tag >> 32);
+            if (ok) break;
+            if (spin > 16) {
+              if (*af) break;
+              if ((spin & 63) == 0 && *reinterpret_cast<volatile int*>(p.abort_g)) { *af = 1; break; }
+              if (spin > 4096) __nanosleep(64);
+              if (spin >= kMegaSpin) {
+                *af = 1;
+                att_note_timeout(p.abort_g, 7, gseq);
+                *reinterpret_cast<volatile int*>(p.abort_g) = 1;
+                atomicCAS(w.status, DEV_OK, DEV_TIMEOUT);
+                break;
+              }
+            }
+          }
+#pragma unroll
+          for (int k = 0; k < 6; ++k) {
+            const bool use = k0 + k < n;
+            s0 += use ? __uint_as_float((unsigned)pw[0][k]) : 0.f;
+            s1 += use ? __uint_as_float((unsigned)pw[1][k]) : 0.f;
+          }
+        }
+        const float y0 = x0 + s0, y1 = x1 + s1;
+        w.X[(size_t)r0 * dm.d + f] = y0;
+        store_act<bf16>(w.A, R, dm.d, r0, f, y0 * gn);
+        if (i1 != i) {
+          w.X[(size_t)r1 * dm.d + f] = y1;
+          store_act<bf16>(w.A, R, dm.d, r1, f, y1 * gn);
+        }
+        const float q0 = warp_sum(y0 * y0), q1 = warp_sum(y1 * y1);
+        if (lane == 0) {
+          ctl->red[grp][quarter][i] = q0;
+          ctl->red[grp][quarter][i1] = q1;
+        }
+      }
+      bar_sync(bar_id, 128);
+      if (et >= a && et < b)
+        p.sumsq[((size_t)buf * nt128 + tile) * kMegaMaxRows + c0 + et] =
+            ctl->red[grp][0][et] + ctl->red[grp][1][et] + ctl->red[grp][2][et] + ctl->red[grp][3][et];
+      bar_sync(bar_id, 128);
     }
   }
   if (et == 0) MEGA_EV(sidx, 6);
