@@ -476,21 +476,38 @@ __device__ __forceinline__ unsigned long long att_timer_ns() {
   return t;
 }
 
+// One m-tile (query rows row0 .. row0+15) of tail segment x = b * Hkv + h: the block's own rows as keys.
 template <int HD, int NT>
-__device__ __forceinline__ void att_tails(AttWarp<HD, NT>& st, const AttPlan& pl, const AttGeom& g, const StepArgs* __restrict__ args,
-                                       const KvView& kv, const AttArgs& a, int Hkv, int c, int G, int row0, int lane);
+__device__ __forceinline__ void att_tail_task(AttWarp<HD, NT>& st, const AttGeom& g, const AttArgs& a, int x, int row0, int lane) {
+  const int rows = g.rows;
+  st.reset();
+  st.load_q(a.Qb + (size_t)x * g.nq * HD, row0, g.nq, lane);
+  const __half* kn = a.KVn + (size_t)x * 2 * rows * HD;
+  auto krow = [&](int kq) -> const __half* { return kn + (size_t)kq * HD; };
+  auto vrow = [&](int kq) -> const __half* { return kn + (size_t)(rows + kq) * HD; };
+  st.tail(krow, vrow, rows, row0, g.nq, lane);
+  st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
+}
 
-// One consumer warp (cw of n_active = MT*KS) of block c of G: all ring segments of the block's tile
-// range [t_lo, t_hi) starting at ring position `it`, then the block's tail segments.
+// One consumer warp (cw of kAttMaxWarps) of block c of G.  The first n_active = MT*KS warps take all ring
+// segments of the block's tile range [t_lo, t_hi) starting at ring position `it`; the others take tail tasks.
 template <int HD, int NT>
 __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const AttPlan& pl, const AttGeom& g,
                                             const StepArgs* __restrict__ args, const KvView& kv, const AttArgs& a, int Hkv,
                                             int c, int G, int cw, int lane) {
-  const int B = args->B, n_active = g.MT * g.KS;
+  const int B = args->B, n_active = g.MT * g.KS, n_spare = kAttMaxWarps - n_active;
+  AttWarp<HD, NT> st;
+  if (cw >= n_active) {
+    // A consumer warp without a share of the ring tiles takes tail tasks (one m-tile of one tail segment
+    // each), dealt over the spare warps of all blocks from the last block down: the tails then run beside
+    // the tiles instead of after them.
+    for (int q = (G - 1 - c) * n_spare + (cw - n_active); q < B * Hkv * g.MT; q += G * n_spare)
+      att_tail_task<HD, NT>(st, g, a, q / g.MT, (q % g.MT) * 16, lane);
+    return true;
+  }
   const int mi = cw / g.KS, ks = cw % g.KS, row0 = mi * 16;
   const long long T = pl.T;
   const long long t_lo = (long long)c * T / G, t_hi = (long long)(c + 1) * T / G;
-  AttWarp<HD, NT> st;
   long long t = t_lo;
   while (t < t_hi) {
     const AttTile x = att_locate(pl, B, g.KPS, (int)t);
@@ -523,26 +540,10 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
     if (rg.ev && cw == 0 && lane == 0) rg.ev[2] = att_timer_ns();
     t += n;
   }
-  // tail segments: (b, h) number x goes to block G-1-(x mod G), key share 0 only
-  if (ks == 0 && G - 1 - c < B * Hkv) att_tails<HD, NT>(st, pl, g, args, kv, a, Hkv, c, G, row0, lane);
+  // without spare warps: tail segment (b, h) number x goes to block G-1-(x mod G), key share 0 only
+  if (n_spare == 0 && ks == 0)
+    for (int x = G - 1 - c; x < B * Hkv; x += G) att_tail_task<HD, NT>(st, g, a, x, row0, lane);
   return true;
-}
-
-template <int HD, int NT>
-__device__ __forceinline__ void att_tails(AttWarp<HD, NT>& st, const AttPlan& pl, const AttGeom& g, const StepArgs* __restrict__ args,
-                                       const KvView& kv, const AttArgs& a, int Hkv, int c, int G, int row0, int lane) {
-  const int B = args->B, rows = g.rows;
-  {
-    for (int x = G - 1 - c; x < B * Hkv; x += G) {
-      st.reset();
-      st.load_q(a.Qb + (size_t)x * g.nq * HD, row0, g.nq, lane);
-      const __half* kn = a.KVn + (size_t)x * 2 * rows * HD;
-      auto krow = [&](int kq) -> const __half* { return kn + (size_t)kq * HD; };
-      auto vrow = [&](int kq) -> const __half* { return kn + (size_t)(rows + kq) * HD; };
-      st.tail(krow, vrow, rows, row0, g.nq, lane);
-      st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
-    }
-  }
 }
 
 template <int HD>
@@ -630,7 +631,7 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
                        (it + 1) * npg <= kAttPageCache ? ctl->pages + it * npg : nullptr);
       }
     }
-  } else if (warp - 1 < g.MT * g.KS) {
+  } else {
     AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, kAttStageBytes, kAttStages, abort_flag, nullptr, w.status, nullptr};
     int it = 0;
     att_consume_dispatch<HD>(rg, it, pl, g, args, kv, a, Hkv, c, G, warp - 1, lane);

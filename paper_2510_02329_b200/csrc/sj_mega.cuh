@@ -1149,7 +1149,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         continue;
       }
       // attention over the cache tiles of the ring, then the combine
-      if (alive && ww < g.MT * g.KS) {
+      if (alive) {
         // attention events of block 0 go to the second event set of the layer's QKV phase
         unsigned long long* ev = (p.trace && c == 0 && (l - p.l0) * 4 < kMegaTraceSites)
                                      ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8
