@@ -103,8 +103,9 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *   "step_impl"  1 = the whole step as one persistent cooperative kernel (bf16, tcgen05 GEMMs, at most 80
  *                block rows; default when the shape allows), 0 = one kernel per stage
  *   "ring_stages" persistent kernel: cap on the shared-memory ring depth (0 = as many as fit, the default)
- *   "trace"      1 = the persistent kernel's block 0 stamps its arrival at and release from every device-wide
- *                barrier, and eight events per GEMM phase, with the nanosecond global timer (sj_step_trace())
+ *   "trace"      k > 0 = the persistent kernel records a timeline with the nanosecond global timer
+ *                (sj_step_trace()): block k - 1 stamps its arrival at and release from every device-wide
+ *                barrier and eight events per GEMM phase; every block stamps the first 32 barriers
  *   "graph"      1 = replay the step as a CUDA graph (default unless the stream is NULL, which
  *                cannot be captured), 0 = plain launches
  *   "pdl"        1 = programmatic dependent launch between the step's kernels (default)
@@ -118,14 +119,17 @@ sj_status sj_set_option(sj_target *t, const char *name, int value);
  * count.  Synchronises the stream. */
 sj_status sj_kernel_time(sj_target *t, const char *name, double *total_ms, long *launches);
 
-/* Timeline of the last persistent-kernel step run under "trace" (block 0, global-timer nanoseconds):
- * out_ns[2k] is the time the block reached device-wide barrier k (k = 1, 2, ... in program order: after the
- * embedding phase, then per layer after QKV, attention, combine, O, gate/up and down, then after the LM
- * head), out_ns[2k+1] the time it was released (k < 1024); out_ns[2048 + 8s + e] is event e of GEMM phase s
- * (s counts QKV, O, gate/up, down per layer, then the LM head): 0 activation loads released, 1 last
- * activation load issued, 2 first stage ready, 3 last MMA issued, 4 last accumulator seen by the epilogue,
- * 5 split-K contributors seen, 6 epilogue done, 7 last weight load issued.  Unused entries are 0.  Copies
- * at most max_entries values into the host array; synchronises the stream. */
+/* Timeline of the last persistent-kernel step run under "trace" (global-timer nanoseconds; unused entries 0).
+ * For the traced block: out_ns[2k] is the time it reached device-wide barrier k (k = 1, 2, ... in program
+ * order: after the embedding phase, then per layer after QKV, attention, combine, O, gate/up and down, then
+ * after the LM head), out_ns[2k+1] the time it was released (k < 1024); out_ns[2048 + 8s + e] is event e of
+ * GEMM phase s (s counts QKV, O, gate/up, down per layer, then the LM head): 0 activation loads released,
+ * 1 last activation load issued, 2 first stage ready, 3 last MMA issued, 4 last accumulator seen by the
+ * epilogue, 5 split-K partial sums gathered, 6 epilogue done, 7 last weight load issued;
+ * out_ns[2048 + 4096 + 8s + e] is a second, finer set of epilogue and attention events whose meaning is
+ * private to the kernel source.  For every block c < 256 and barrier k < 32: out_ns[10240 + 256k + c] is
+ * the block's release time and out_ns[18432 + 256k + c] its arrival time.  Copies at most max_entries
+ * (26624 for everything) values into the host array; synchronises the stream. */
 sj_status sj_step_trace(sj_target *t, unsigned long long *out_ns, int max_entries, int *n_entries);
 
 /* Wait for the target's stream and return the device status word (SJ_OK, SJ_ERR_TIMEOUT,

@@ -165,7 +165,7 @@ class Target:
         check(self._lib.sj_kernel_time(self.handle, name.encode(), C.byref(ms), C.byref(n)))
         return ms.value, n.value
 
-    def step_trace(self, max_entries: int = 2048 + 16 * 512):
+    def step_trace(self, max_entries: int = 2048 + 16 * 512 + 2 * 32 * 256):
         """Timeline (ns) of the last persistent-kernel step run with option ``trace`` = 1."""
         buf = (C.c_ulonglong * max_entries)()
         n = C.c_int()

@@ -511,7 +511,7 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
   } else if (n == "trace") {
-    const size_t n_tr = (size_t)2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192 + 8192;
+    const size_t n_tr = kMegaTraceEntries;
     if (value && !t->d_trace) {
       sj_status st = dev_alloc(t, &t->d_trace, n_tr);
       if (st != SJ_OK) return st;
@@ -1013,7 +1013,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
 extern "C" sj_status sj_step_trace(sj_target* t, unsigned long long* out_ns, int max_entries, int* n_entries) {
   if (!t || !out_ns || !n_entries || max_entries <= 0) return fail(SJ_ERR_INVALID_ARG, "null argument");
   if (!t->d_trace) return fail(SJ_ERR_STATE, "tracing was never enabled (sj_set_option \"trace\")");
-  const int n = std::min(max_entries, 2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192 + 8192);
+  const int n = std::min(max_entries, kMegaTraceEntries);
   CU_TRY(cudaStreamSynchronize(t->stream));
   CU_TRY(cudaMemcpy(out_ns, t->d_trace, sizeof(unsigned long long) * n, cudaMemcpyDeviceToHost));
   *n_entries = n;

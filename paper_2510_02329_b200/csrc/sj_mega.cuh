@@ -48,6 +48,10 @@ constexpr int kMegaRegsLight = 80;    // registers per thread of warps 0..3 afte
 constexpr int kMegaRegsHeavy = 208;   // registers per thread of the worker warps (128*96 + 256*200 <= 384*168)
 constexpr int kMegaTraceBarriers = 1024;
 constexpr int kMegaTraceSites = 512;
+constexpr int kMegaTraceAllBarriers = 32;   // barriers whose arrival / release time every block records
+constexpr int kMegaTraceRelease = 2 * kMegaTraceBarriers + 16 * kMegaTraceSites;   // [barrier][256 blocks]
+constexpr int kMegaTraceArrive = kMegaTraceRelease + kMegaTraceAllBarriers * 256;
+constexpr int kMegaTraceEntries = kMegaTraceArrive + kMegaTraceAllBarriers * 256;
 
 enum MegaSite { SITE_QKV = 0, SITE_O = 1, SITE_GU = 2, SITE_DOWN = 3, SITE_LM = 4 };
 
@@ -81,11 +85,12 @@ struct MegaParams {
   unsigned* gbar;             // device-wide barrier counter   } zeroed before every launch
   int* abort_g;               // device-wide abort word        }
   int n_tail_base;
-  // optional timeline of block 0 (global-timer nanoseconds):
+  // optional timeline (global-timer nanoseconds), block `trace_block`:
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
   //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
   //   load issued, 2 first stage ready at the MMA issuer, 3 last MMA committed, 4 last accumulator seen by the
-  //   epilogue, 5 split-K contributors' flags seen, 6 epilogue done, 7 weight producer issued the last load
+  //   epilogue, 5 split-K partial sums gathered, 6 epilogue done, 7 weight producer issued the last load
+  // and of every block: [kMegaTraceRelease + 256*k + block], [kMegaTraceArrive + 256*k + block] for k < 32
   unsigned long long* trace;
   unsigned trace_block;       // the block that writes the timeline
 };
@@ -95,11 +100,6 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
   return t;
 }
-#define MEGA_EVA(sidx, k)                                                                            \
-  do {                                                                                               \
-    if (p.trace && (sidx) < 16)                                                                      \
-      p.trace[2 * kMegaTraceBarriers + 16 * kMegaTraceSites + ((sidx) * 256 + blockIdx.x) * 4 + (k)] = global_timer_ns(); \
-  } while (0)
 #define MEGA_EV(sidx, k)                                                                             \
   do {                                                                                               \
     if (p.trace && blockIdx.x == p.trace_block && (sidx) < kMegaTraceSites)                                      \
@@ -311,7 +311,7 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
   if (wt == 0) {
     const bool tr = p.trace && blockIdx.x == p.trace_block && nbar < kMegaTraceBarriers;
     if (tr) p.trace[2 * nbar] = global_timer_ns();
-    if (p.trace && nbar < 32) p.trace[2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + 8192 + nbar * 256 + blockIdx.x] = global_timer_ns();
+    if (p.trace && nbar < kMegaTraceAllBarriers) p.trace[kMegaTraceArrive + nbar * 256 + blockIdx.x] = global_timer_ns();
     if (!ctl->abort_flag) {
       __threadfence();
       red_relaxed_add(p.gbar, 1u);
@@ -319,7 +319,7 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
     }
     __threadfence();
     if (tr) p.trace[2 * nbar + 1] = global_timer_ns();
-    if (p.trace && nbar < 32) p.trace[2 * kMegaTraceBarriers + 16 * kMegaTraceSites + 16384 + nbar * 256 + blockIdx.x] = global_timer_ns();
+    if (p.trace && nbar < kMegaTraceAllBarriers) p.trace[kMegaTraceRelease + nbar * 256 + blockIdx.x] = global_timer_ns();
     *reinterpret_cast<volatile int*>(&ctl->bars_passed) = nbar;
   }
   bar_sync(1, kMegaWorkers);
@@ -551,7 +551,6 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       }
       if (et == 0) MEGA_EV(sidx, 5);
       if (et == 0) MEGA_EV2(0, sidx, 1);
-      if (et == 0 && owner && c_last > c) MEGA_EVA(sidx, 2);
       if (site == SITE_QKV) {
         const int half = HD / 2;
 #pragma unroll
@@ -777,7 +776,6 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     }
   }
   if (et == 0) MEGA_EV(sidx, 6);
-  if (et == 0) MEGA_EVA(sidx, 3);
 }
 
 // a1 + first a2: embedding gather, fp32 residual stream, first GEMM input planes, sums of squares, and
@@ -1076,7 +1074,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           ++seg;
         }
         MEGA_EV(sidx, 3);
-        MEGA_EVA(sidx, 0);
         ++sidx;
       };
       auto fatt = [&](int l) { rp.advance(n_att); };
