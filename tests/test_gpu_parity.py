@@ -239,3 +239,26 @@ def test_full_width_cuts_of_the_benchmark_shapes(name, shape, kv_lens, gamma):
             print(name, "mode", mode, rep)
     finally:
         case.close()
+
+
+# ------------------------------------------------------------------------------------------------
+# the benchmark's own sizes: every layer, the full vocabulary, the cache length and gamma of the
+# workload, in the launch configuration bench.py times (default options, one persistent-kernel launch
+# per step).  The fp64 oracle computes the whole step: one layer's weights at a time are copied from
+# the device and widened, so the host holds a few GB; about a minute for the 8B shape.
+# ------------------------------------------------------------------------------------------------
+FULL_CASES = [("cfg2", synth.WORKLOADS["cfg2"]), ("cfg3", synth.WORKLOADS["cfg3"])]
+
+
+@pytest.mark.parametrize("name,wl", FULL_CASES, ids=[c[0] for c in FULL_CASES])
+def test_full_size_benchmark_workloads(name, wl):
+    kv_lens = [int(x) for x in synth.kv_lengths(wl, 0)]
+    case = harness.Case(wl.shape, torch.bfloat16, kv_lens, wl.gamma, seed=0, cache="fill", gen_device="cuda").gpu_setup(
+        max_rows=len(kv_lens) * (wl.gamma + 1))
+    try:
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 1.0)]:
+            rep, _ = _run(case, mode, T)
+            assert rep.exact + rep.margin == len(kv_lens)
+            print(name, "mode", mode, rep)
+    finally:
+        case.close()
