@@ -657,10 +657,16 @@ template <> struct AttVec<2> {
   static __device__ __forceinline__ void fma(float* acc, const float2& v, float w) { acc[0] += v.x * w; acc[1] += v.y * w; }
 };
 
+// kAttCombineSplit warps share one item (each a contiguous part of the head dimension): with two, the 2 x 32
+// dims a lane holds per sub-partial are one 8-byte load and all sub-partials of a config-3 item (39) are in
+// flight at once; with one warp per item they need two dependent batches.
+template <int HD> struct AttCombineSplit { static constexpr int value = HD >= 128 ? 2 : 1; };
 template <typename T, int HD>
 __device__ __forceinline__ void att_combine_item(const AttPartials& P, const AttPlan& pl, const AttGeom& g, int G_att,
-                                                 int n_tail_base, int Hkv, int item, void* ATT, int R, int Hq, int lane,
+                                                 int n_tail_base, int Hkv, int item_part, void* ATT, int R, int Hq, int lane,
                                                  unsigned long long* ev = nullptr) {
+  constexpr int SPLIT = AttCombineSplit<HD>::value;
+  const int item = item_part / SPLIT, part = item_part % SPLIT;
   const int q = item % g.nq, bh = item / g.nq, b = bh / Hkv, h = bh % Hkv;
   const int L = pl.L[b];
   const int nt_b = (L + g.KPS - 1) / g.KPS;
@@ -685,10 +691,11 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     const int cc = c_first + (k >> ks_shift);
     return (long long)(cc + 1) * pl.T / G_att > (long long)cc * pl.T / G_att;
   };
-  constexpr int DPL = HD / 32;   // dims per lane
-  constexpr int OB = 24;         // output rows whose loads one lane keeps in flight
+  constexpr int DPL = HD / 32 / SPLIT;   // dims per lane
+  constexpr int OB = DPL <= 2 ? 40 : 24;   // output rows whose loads one lane keeps in flight
+  constexpr int RS = HD / DPL;             // row stride of the outputs in units of V
   typedef typename AttVec<DPL>::type V;
-  const V* Po = reinterpret_cast<const V*>(P.o) + lane;   // row r of the outputs starts at Po + r * 32
+  const V* Po = reinterpret_cast<const V*>(P.o) + part * 32 + lane;   // row r of the outputs starts at Po + r * RS
   float lsum = 0.f, Mrun = -INFINITY, acc[DPL];
 #pragma unroll
   for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
@@ -706,7 +713,7 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     const int kn = min(96, n_sub - k0);
     V ob[OB];
 #pragma unroll
-    for (int k = 0; k < OB; ++k) ob[k] = __ldcg(Po + (size_t)sub_index(k0 + min(k, kn - 1)) * 32);
+    for (int k = 0; k < OB; ++k) ob[k] = __ldcg(Po + (size_t)sub_index(k0 + min(k, kn - 1)) * RS);
     float Mb = fmaxf(fmaxf(mk[0], mk[1]), mk[2]);
     if (ev && lane == 0) ev[0] = att_timer_ns();
     Mb = warp_max(Mb);
@@ -727,12 +734,12 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     if (ev && lane == 0) ev[1] = att_timer_ns();
 #pragma unroll
     for (int k = 0; k < OB; ++k) {
-      const float wgt = k < kn ? __shfl_sync(0xffffffffu, wk[0], k) : 0.f;   // OB <= 32: the first weight register
+      const float wgt = k < kn ? __shfl_sync(0xffffffffu, k < 32 ? wk[0] : wk[1], k & 31) : 0.f;
       AttVec<DPL>::fma(acc, ob[k], wgt);
     }
     for (int kb = OB; kb < kn; kb += OB) {   // further output rows, OB at a time, added in order
 #pragma unroll
-      for (int k = 0; k < OB; ++k) ob[k] = __ldcg(Po + (size_t)sub_index(k0 + min(kb + k, kn - 1)) * 32);
+      for (int k = 0; k < OB; ++k) ob[k] = __ldcg(Po + (size_t)sub_index(k0 + min(kb + k, kn - 1)) * RS);
 #pragma unroll
       for (int k = 0; k < OB; ++k) {
         const int kk = kb + k;
@@ -746,7 +753,7 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
   const int gq = q / g.rows, j = q % g.rows, r = b * g.rows + j, head = h * g.group + gq;
   const float inv = 1.0f / lsum;
 #pragma unroll
-  for (int i = 0; i < DPL; ++i) store_act<T>(ATT, R, Hq * HD, r, head * HD + lane * DPL + i, acc[i] * inv);
+  for (int i = 0; i < DPL; ++i) store_act<T>(ATT, R, Hq * HD, r, head * HD + (part * 32 + lane) * DPL + i, acc[i] * inv);
 }
 
 template <int HD>
@@ -760,7 +767,7 @@ __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dim
   if (threadIdx.x == 0) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS);
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
-  const int items = B * dm.Hkv * g.nq;
+  const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;
   for (int item = warp * gridDim.x + blockIdx.x; item < items; item += gridDim.x * wpb)   // spread over blocks first
     att_combine_item<bf16, HD>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, w.ATT, B * rows, dm.Hq, lane);
 }

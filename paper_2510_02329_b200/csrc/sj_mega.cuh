@@ -1148,7 +1148,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
       if (alive) {
         const AttPartials P{w.tc_m, w.tc_l, w.tc_o};
-        const int items = B * dm.Hkv * g.nq;
+        const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;
         for (int item = ww * G + c; item < items; item += G * 8)   // spread over blocks first
           att_combine_item<bf16, HD>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane,
                                      (p.trace && c == 0 && ww == 0 && (l - p.l0) * 4 < kMegaTraceSites)
