@@ -353,12 +353,17 @@ __device__ __forceinline__ void mega_issue_w(const MegaMaps& mp, int site, int l
 
 // ---------------------------------------------------------------------------------------------
 // fused epilogues.  All eight worker warps take part, as two groups of four warps (a warp reads the
-// accumulator lanes 32 * (warp % 4) .. + 31, so either group covers the tile's 128 features): the block
-// rows are cut into chunks of eight accumulator columns, group 0 takes the even chunks and group 1 the odd
-// ones.  One warp per scheduler runs a long dependent instruction chain at a fraction of an instruction
+// accumulator lanes 32 * (warp % 4) .. + 31, so either group covers the tile's 128 features): of every 16
+// block rows group 0 takes the first half of those that exist and group 1 the rest (5 + 4 at 9 rows).  One warp per scheduler runs a long dependent instruction chain at a fraction of an instruction
 // per cycle, so halving the rows per thread nearly halves the time between the last MMA and the barrier.
 // Each group has its own named barrier (2 + group, 128 threads) and its own exchange buffers.
 // ---------------------------------------------------------------------------------------------
+// Which of the two epilogue groups handles block row r: the rows of every 16-row chunk are halved.
+__device__ __forceinline__ int mega_row_group(int r, int R) {
+  const int c16 = r & ~15, n16 = min(16, R - c16);
+  return (r - c16) >= ((n16 + 1) >> 1) ? 1 : 0;
+}
+
 template <int HD>
 __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
                                               const Work& w, const Dims& dm, int wt) {
@@ -382,14 +387,14 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       for (int k = 0; k < 4; ++k) {
         const int r = r0 + 4 * k;
         part[k] = 0.f;
-        if (r < R && ((r >> 3) & 1) == grp)
+        if (r < R && mega_row_group(r, R) == grp)
           for (int t = lane; t < nt128; t += 32) part[k] += __ldcg(p.sumsq + ((size_t)buf * nt128 + t) * kMegaMaxRows + r);
       }
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int r = r0 + 4 * k;
         const float s = warp_sum(part[k]);
-        if (lane == 0 && r < R && ((r >> 3) & 1) == grp) ctl->inv[r] = 1.0f / sqrtf(s / (float)dm.d + dm.eps);
+        if (lane == 0 && r < R && mega_row_group(r, R) == grp) ctl->inv[r] = 1.0f / sqrtf(s / (float)dm.d + dm.eps);
       }
     }
     bar_sync(bar_id, 128);
@@ -448,20 +453,23 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     tc_fence_after();
     if (et == 0) MEGA_EV(sidx, 4);
 
-    for (int c0 = 8 * grp; c0 < Rp; c0 += 16) {
+    for (int c16 = 0; c16 < Rp; c16 += 16) {
+      // this group's rows of the 16-row chunk: the first or the second half of the rows that exist
+      const int n16 = max(min(16, R - c16), 0), h16 = (n16 + 1) >> 1;
+      const int c0 = c16 + (grp ? h16 : 0), nr = grp ? n16 - h16 : h16, rend = c0 + nr;
       float v[8], xs[8];
       float2 cs[8];
       // every global load of this chunk is issued before anything waits on one of them
       if (owner && (site == SITE_O || site == SITE_DOWN)) {   // residual rows
         const int f = tile * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) xs[i] = __ldcg(w.X + (size_t)min(c0 + i, R - 1) * dm.d + f);   // unpredicated: rows past R repeat the last row
+        for (int i = 0; i < 8; ++i) xs[i] = __ldcg(w.X + (size_t)max(min(c0 + i, rend - 1), 0) * dm.d + f);   // unpredicated: rows past R repeat the last row
       }
       if (owner && site == SITE_QKV && kind < 2) {            // rotary table rows
         const int ii = dim & (HD / 2 - 1);
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          cs[i] = __ldcg(w.rope + (size_t)min(c0 + i, R - 1) * (HD / 2) + ii);
+          cs[i] = __ldcg(w.rope + (size_t)max(min(c0 + i, rend - 1), 0) * (HD / 2) + ii);
       }
       if (mine) {
         float lo[8];
@@ -479,14 +487,14 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         unsigned long long* dst = p.pbuf + ((size_t)(2 * c + (c == c_first ? 1 : 0)) * Rp + c0) * kTileN + fl;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          if (c0 + i < R) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
+          if (i < nr) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
         continue;
       }
       if (!owner) {   // publish the partial sums, each with this phase's number
         unsigned long long* dst = p.pbuf + ((size_t)(2 * c) * Rp + c0) * kTileN + fl;
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          if (c0 + i < R) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
+          if (i < nr) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
         continue;
       }
       // The other blocks' shares of this tile: two blocks' words in flight at a time, all of them reloaded
@@ -505,7 +513,6 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           src[k] = p.pbuf + ((size_t)(2 * (live[k] ? c2 : c)) * Rp + c0) * kTileN + fl;
         }
         volatile int* af = &ctl->abort_flag;
-        const int nr = min(8, R - c0);
         for (uint32_t spin = 0;; ++spin) {
           bool ok = true;
           // every load is issued before any result is looked at: rows past R read row 0 again (in
@@ -544,7 +551,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
-          v[i] = v[i] * (r < R ? ctl->inv[r] : 0.f) + bias;
+          v[i] = v[i] * (r < rend ? ctl->inv[r] : 0.f) + bias;
         }
         if (kind < 2) {
 #pragma unroll
@@ -565,17 +572,17 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           __half* qb = w.Qb + (size_t)head * rows * HD + dim;
 #pragma unroll
           for (int i = 0; i < 8; ++i)
-            if (c0 + i < R) qb[ctl->row_qoff[c0 + i]] = __float2half_rn(v[i] * qscale);
+            if (i < nr) qb[ctl->row_qoff[c0 + i]] = __float2half_rn(v[i] * qscale);
         } else {
           bf16* kvb = reinterpret_cast<bf16*>(kv.pool) +
                       ((size_t)l * kv.n_pages * 2 * dm.Hkv + (size_t)(kind - 1) * dm.Hkv + head) * kv.page_size * HD + dim;
 #pragma unroll
           for (int i = 0; i < 8; ++i)
-            if (c0 + i < R) kvb[ctl->row_kvoff[c0 + i]] = __float2bfloat16_rn(v[i]);
+            if (i < nr) kvb[ctl->row_kvoff[c0 + i]] = __float2bfloat16_rn(v[i]);
           __half* kn = w.KVn + (size_t)(head * 2 + kind - 1) * rows * HD + dim;
 #pragma unroll
           for (int i = 0; i < 8; ++i)
-            if (c0 + i < R) kn[ctl->row_nkvoff[c0 + i]] = __float2half_rn(v[i]);
+            if (i < nr) kn[ctl->row_nkvoff[c0 + i]] = __float2half_rn(v[i]);
         }
       } else if (site == SITE_O || site == SITE_DOWN) {
         const int f = tile * kTileN + fl;
@@ -585,7 +592,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
           ss[i] = 0.f;
-          if (r < R) {
+          if (r < rend) {
             const float x = xs[i] + v[i];
             w.X[(size_t)r * dm.d + f] = x;
             store_act<bf16>(w.A, R, dm.d, r, f, x * gn);
@@ -595,13 +602,13 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         if (et == 0) MEGA_EV2(0, sidx, 2);
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-          if (c0 + i < R) ss[i] = warp_sum(ss[i]);   // block-uniform
+          if (i < nr) ss[i] = warp_sum(ss[i]);   // block-uniform
         if (lane == 0) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) ctl->red[grp][quarter][i] = ss[i];
         }
         bar_sync(bar_id, 128);
-        if (et < 8 && c0 + et < R)
+        if (et < nr)
           p.sumsq[((size_t)buf * nt128 + tile) * kMegaMaxRows + c0 + et] =
               ctl->red[grp][0][et] + ctl->red[grp][1][et] + ctl->red[grp][2][et] + ctl->red[grp][3][et];
         bar_sync(bar_id, 128);
@@ -610,7 +617,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
-          v[i] *= (r < R ? ctl->inv[r] : 0.f);
+          v[i] *= (r < rend ? ctl->inv[r] : 0.f);
         }
         if (fl >= 64) {
 #pragma unroll
@@ -622,7 +629,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const int r = c0 + i;
-            if (r < R) {
+            if (r < rend) {
               const float g = v[i], up = ctl->u.exch[grp][fl][i];
               store_act<bf16>(w.H, R, dm.F, r, f, g / (1.0f + expf(-g)) * up);
             }
@@ -635,7 +642,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         for (int i = 0; i < 8; ++i) {
           const int r = c0 + i;
           float z = -INFINITY;
-          if (r < R && n < dm.V) {
+          if (r < rend && n < dm.V) {
             const float raw = v[i] * ctl->inv[r];
             if (w.logits) w.logits[(size_t)r * dm.V + n] = raw;
             if (dbg_logits) dbg_logits[(size_t)r * dm.V + n] = raw;
@@ -658,7 +665,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           }
         }
         bar_sync(bar_id, 128);
-        if (et < 8 && c0 + et < R) {
+        if (et < nr) {
           RowStat a = ctl->wstat[grp][0][et];
           a = stat_merge(a, ctl->wstat[grp][1][et]);
           a = stat_merge(a, ctl->wstat[grp][2][et]);
@@ -693,11 +700,13 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     const unsigned long long tag = (unsigned long long)(unsigned)gseq << 32;
     volatile int* af = &ctl->abort_flag;
 #pragma unroll 1
-    for (int c0 = 8 * grp; c0 < Rp; c0 += 16) {
+    for (int c16 = 0; c16 < Rp; c16 += 16) {
+      const int n16 = max(min(16, R - c16), 0), h16 = (n16 + 1) >> 1;
+      const int c0 = c16 + (grp ? h16 : 0), nr = grp ? n16 - h16 : h16;
       // Rows are dealt with weight 1 to the first and the last sharing block and weight 2 to the others:
       // the first block of one tile is as a rule the last block of the tile before, and finishes rows of both.
       const int wsum = 2 * n - 2, w_lo = j == 0 ? 0 : 2 * j - 1, w_hi = j == n - 1 ? wsum : 2 * j + 1;
-      const int a = max(w_lo * R / wsum - c0, 0), b = min(w_hi * R / wsum - c0, min(8, R - c0));   // this block's rows of the chunk: [a, b)
+      const int a = max(w_lo * R / wsum - c0, 0), b = min(w_hi * R / wsum - c0, nr);   // this block's rows of the chunk: [a, b)
 #pragma unroll 1
       for (int i = a; i < b; i += 2) {   // two rows at a time: their loads share one round trip
         const int i1 = min(i + 1, b - 1);   // == i when the second row is absent: it repeats the first
