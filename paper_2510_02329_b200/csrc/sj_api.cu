@@ -278,6 +278,13 @@ static bool tc_shapes_ok(const sj_model_config& c) {
          (c.n_q_heads * c.head_dim) % kBK == 0;
 }
 
+typedef void (*MegaKernel)(const MegaMaps, const MegaParams, const StepArgs*, const KvView, const Work, const Dims);
+// The persistent kernel for a head dimension (64 or 128) and a number of row slots (4, 6 or 8).
+static MegaKernel mega_kernel(int hd, int ns) {
+  if (hd == 128) return ns == 4 ? k_verify_mega<128, 4> : (ns == 6 ? k_verify_mega<128, 6> : k_verify_mega<128, 8>);
+  return ns == 4 ? k_verify_mega<64, 4> : (ns == 6 ? k_verify_mega<64, 6> : k_verify_mega<64, 8>);
+}
+
 extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weights* w, void* cuda_stream,
                                       sj_target** out) {
   if (!cfg || !w || !out) return fail(SJ_ERR_INVALID_ARG, "null argument");
@@ -430,10 +437,8 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     cudaError_t e = cudaMemcpy(t->d_layer_ptrs, lp.data(), lp.size() * sizeof(MegaLayerPtrs), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(t->d_sumsq, 0, sizeof(float) * 2 * (c.d_model / kTileN) * kMegaMaxRows);
     if (e == cudaSuccess) e = cudaMemset(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)4 * t->sm_count * pad16(Rm) * kTileN));
-    if (e == cudaSuccess)
-      e = c.head_dim == 128
-              ? cudaFuncSetAttribute(k_verify_mega<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
-              : cudaFuncSetAttribute(k_verify_mega<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    for (int ns = 4; ns <= 8 && e == cudaSuccess; ns += 2)
+      e = cudaFuncSetAttribute(mega_kernel(c.head_dim, ns), cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "whole-step kernel set-up: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
     for (int l0 = 0; l0 < c.n_layers; l0 += kMegaMaxLayers) {
       t->mega_maps.emplace_back();
@@ -998,8 +1003,9 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
     cfg.attrs = at;
     cfg.numAttrs = 1;
     const StepArgs* args = t->d_args;
-    if (dm.hd == 128) CU_TRY(cudaLaunchKernelEx(&cfg, k_verify_mega<128>, mm, p, args, kv->view, W, dm));
-    else CU_TRY(cudaLaunchKernelEx(&cfg, k_verify_mega<64>, mm, p, args, kv->view, W, dm));
+    // row slots per epilogue thread: a group gets at most (min(R, 16) + 1) / 2 rows of a 16-row chunk
+    const int ns = R <= 8 ? 4 : (R <= 12 ? 6 : 8);
+    CU_TRY(cudaLaunchKernelEx(&cfg, mega_kernel(dm.hd, ns), mm, p, args, kv->view, W, dm));
     if (timing) {
       CU_TRY(cudaEventRecord(eb, s));
       t->timed.push_back({"verify_step", ea, eb});

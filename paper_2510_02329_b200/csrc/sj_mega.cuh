@@ -364,7 +364,10 @@ __device__ __forceinline__ int mega_row_group(int r, int R) {
   return (r - c16) >= ((n16 + 1) >> 1) ? 1 : 0;
 }
 
-template <int HD>
+// NS: row slots a thread unrolls per chunk (4, 6 or 8): at least the rows a group gets of a 16-row chunk.
+// Every slot's instructions issue whether its row exists or not, so the kernel is instantiated for the
+// slot counts 4 (up to 8 block rows), 6 (up to 12) and 8.
+template <int HD, int NS>
 __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
                                               const Work& w, const Dims& dm, int wt) {
   const int et = wt & 127, grp = wt >> 7, bar_id = 2 + grp;
@@ -457,43 +460,43 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       // this group's rows of the 16-row chunk: the first or the second half of the rows that exist
       const int n16 = max(min(16, R - c16), 0), h16 = (n16 + 1) >> 1;
       const int c0 = c16 + (grp ? h16 : 0), nr = grp ? n16 - h16 : h16, rend = c0 + nr;
-      float v[8], xs[8];
-      float2 cs[8];
+      float v[NS], xs[NS];
+      float2 cs[NS];
       // every global load of this chunk is issued before anything waits on one of them
       if (owner && (site == SITE_O || site == SITE_DOWN)) {   // residual rows
         const int f = tile * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) xs[i] = __ldcg(w.X + (size_t)max(min(c0 + i, rend - 1), 0) * dm.d + f);   // unpredicated: rows past R repeat the last row
+        for (int i = 0; i < NS; ++i) xs[i] = __ldcg(w.X + (size_t)max(min(c0 + i, rend - 1), 0) * dm.d + f);   // unpredicated: rows past R repeat the last row
       }
       if (owner && site == SITE_QKV && kind < 2) {            // rotary table rows
         const int ii = dim & (HD / 2 - 1);
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < NS; ++i)
           cs[i] = __ldcg(w.rope + (size_t)max(min(c0 + i, rend - 1), 0) * (HD / 2) + ii);
       }
       if (mine) {
-        float lo[8];
-        tc_ld8(taddr + c0, v);
-        tc_ld8(taddr + Rp + c0, lo);
+        float hi8[8], lo8[8];
+        tc_ld8(taddr + c0, hi8);
+        tc_ld8(taddr + Rp + c0, lo8);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] += lo[i];
+        for (int i = 0; i < NS; ++i) v[i] = hi8[i] + lo8[i];
       } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        for (int i = 0; i < NS; ++i) v[i] = 0.f;
       }
       const unsigned long long tag = (unsigned long long)(unsigned)gseq << 32;
       if (et == 0 && owner) MEGA_EV2(0, sidx, 0);
       if (rowsplit) {   // publish every row; the rows are finished after the loop over the segments
         unsigned long long* dst = p.pbuf + ((size_t)(2 * c + (c == c_first ? 1 : 0)) * Rp + c0) * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < NS; ++i)
           if (i < nr) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
         continue;
       }
       if (!owner) {   // publish the partial sums, each with this phase's number
         unsigned long long* dst = p.pbuf + ((size_t)(2 * c) * Rp + c0) * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < NS; ++i)
           if (i < nr) st_relaxed_u64(dst + (size_t)i * kTileN, tag | __float_as_uint(v[i]));
         continue;
       }
@@ -503,7 +506,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       // the first thing it computes.  A wait that runs out raises the abort word and goes on with whatever
       // it read (the block leaves together at its next block-wide check).
       for (int cb = c + 1; cb <= c_last; cb += 2) {
-        unsigned long long pw[2][8];
+        unsigned long long pw[2][NS];
         const unsigned long long* src[2];
         bool live[2];
 #pragma unroll
@@ -520,11 +523,11 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
           for (int k = 0; k < 2; ++k)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) pw[k][i] = ld_relaxed_u64(src[k] + (size_t)(i < nr ? i : 0) * kTileN);
+            for (int i = 0; i < NS; ++i) pw[k][i] = ld_relaxed_u64(src[k] + (size_t)(i < nr ? i : 0) * kTileN);
 #pragma unroll
           for (int k = 0; k < 2; ++k)
 #pragma unroll
-            for (int i = 0; i < 8; ++i) ok = ok && (!live[k] || i >= nr || (pw[k][i] >> 32) == (tag >> 32));
+            for (int i = 0; i < NS; ++i) ok = ok && (!live[k] || i >= nr || (pw[k][i] >> 32) == (tag >> 32));
           if (ok) break;
           if (spin > 16) {
             if (*af) break;
@@ -542,24 +545,24 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
 #pragma unroll
         for (int k = 0; k < 2; ++k)
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] += (live[k] && i < nr) ? __uint_as_float((unsigned)pw[k][i]) : 0.f;
+          for (int i = 0; i < NS; ++i) v[i] += (live[k] && i < nr) ? __uint_as_float((unsigned)pw[k][i]) : 0.f;
       }
       if (et == 0) MEGA_EV(sidx, 5);
       if (et == 0) MEGA_EV2(0, sidx, 1);
       if (site == SITE_QKV) {
         const int half = HD / 2;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < NS; ++i) {
           const int r = c0 + i;
           v[i] = v[i] * (r < rend ? ctl->inv[r] : 0.f) + bias;
         }
         if (kind < 2) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) ctl->u.exch[grp][fl][i] = v[i];
+          for (int i = 0; i < NS; ++i) ctl->u.exch[grp][fl][i] = v[i];
           bar_sync(bar_id, 128);
           const bool first = dim < half;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < NS; ++i) {
             const float xp = ctl->u.exch[grp][fl ^ half][i];
             v[i] = first ? v[i] * cs[i].x - xp * cs[i].y : v[i] * cs[i].x + xp * cs[i].y;
           }
@@ -571,25 +574,25 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         if (kind == 0) {
           __half* qb = w.Qb + (size_t)head * rows * HD + dim;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < NS; ++i)
             if (i < nr) qb[ctl->row_qoff[c0 + i]] = __float2half_rn(v[i] * qscale);
         } else {
           bf16* kvb = reinterpret_cast<bf16*>(kv.pool) +
                       ((size_t)l * kv.n_pages * 2 * dm.Hkv + (size_t)(kind - 1) * dm.Hkv + head) * kv.page_size * HD + dim;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < NS; ++i)
             if (i < nr) kvb[ctl->row_kvoff[c0 + i]] = __float2bfloat16_rn(v[i]);
           __half* kn = w.KVn + (size_t)(head * 2 + kind - 1) * rows * HD + dim;
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
+          for (int i = 0; i < NS; ++i)
             if (i < nr) kn[ctl->row_nkvoff[c0 + i]] = __float2half_rn(v[i]);
         }
       } else if (site == SITE_O || site == SITE_DOWN) {
         const int f = tile * kTileN + fl;
         const int buf = (site == SITE_O) ? 1 : 0;
-        float ss[8];
+        float ss[NS];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < NS; ++i) {
           const int r = c0 + i;
           ss[i] = 0.f;
           if (r < rend) {
@@ -601,11 +604,11 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         }
         if (et == 0) MEGA_EV2(0, sidx, 2);
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < NS; ++i)
           if (i < nr) ss[i] = warp_sum(ss[i]);   // block-uniform
         if (lane == 0) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) ctl->red[grp][quarter][i] = ss[i];
+          for (int i = 0; i < NS; ++i) ctl->red[grp][quarter][i] = ss[i];
         }
         bar_sync(bar_id, 128);
         if (et < nr)
@@ -615,19 +618,19 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         if (et == 0) MEGA_EV2(0, sidx, 3);
       } else if (site == SITE_GU) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < NS; ++i) {
           const int r = c0 + i;
           v[i] *= (r < rend ? ctl->inv[r] : 0.f);
         }
         if (fl >= 64) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) ctl->u.exch[grp][fl - 64][i] = v[i];
+          for (int i = 0; i < NS; ++i) ctl->u.exch[grp][fl - 64][i] = v[i];
         }
         bar_sync(bar_id, 128);
         if (fl < 64) {
           const int f = tile * 64 + fl;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
+          for (int i = 0; i < NS; ++i) {
             const int r = c0 + i;
             if (r < rend) {
               const float g = v[i], up = ctl->u.exch[grp][fl][i];
@@ -639,7 +642,7 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
       } else {   // LM head
         const int n = tile * kTileN + fl;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
+        for (int i = 0; i < NS; ++i) {
           const int r = c0 + i;
           float z = -INFINITY;
           if (r < rend && n < dm.V) {
@@ -899,7 +902,7 @@ __device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p,
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int HD>
+template <int HD, int SLOTS>
 __global__ void __launch_bounds__(kMegaThreads, 1)
 k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const StepArgs* __restrict__ args, const KvView kv,
               const Work w, const Dims dm) {
@@ -1130,7 +1133,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     auto units = [&](int site) -> int { return site_units(site_split(site, dm, c, G)); };
     auto gemm_phase = [&](int site, int l) {
       ++gseq;
-      if (alive) mega_epilogue<HD>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
+      if (alive) mega_epilogue<HD, SLOTS>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
       it += units(site);
       alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
     };
