@@ -122,15 +122,16 @@ struct AttWarp {
   }
 
   // A fragments of this warp's 16 query rows.  Qb: [nq][HD] fp16 of one (sequence, KV head), already
-  // scaled by log2(e)/sqrt(HD).  Rows >= nq read as zero.
+  // scaled by log2(e)/sqrt(HD).  Rows >= nq repeat row nq-1 (their results are never stored): the loads are
+  // unpredicated, so that all of them are in flight together.
   __device__ __forceinline__ void load_q(const __half* __restrict__ Qb, int row0, int nq, int lane) {
-    const int r0 = row0 + (lane >> 2), r1 = r0 + 8, c = (lane & 3) * 2;
+    const int r0 = min(row0 + (lane >> 2), nq - 1), r1 = min(row0 + (lane >> 2) + 8, nq - 1), c = (lane & 3) * 2;
 #pragma unroll
     for (int k = 0; k < HD / 16; ++k) {
-      qa[k][0] = r0 < nq ? ldcg_u32(Qb + (size_t)r0 * HD + k * 16 + c) : 0u;
-      qa[k][1] = r1 < nq ? ldcg_u32(Qb + (size_t)r1 * HD + k * 16 + c) : 0u;
-      qa[k][2] = r0 < nq ? ldcg_u32(Qb + (size_t)r0 * HD + k * 16 + c + 8) : 0u;
-      qa[k][3] = r1 < nq ? ldcg_u32(Qb + (size_t)r1 * HD + k * 16 + c + 8) : 0u;
+      qa[k][0] = ldcg_u32(Qb + (size_t)r0 * HD + k * 16 + c);
+      qa[k][1] = ldcg_u32(Qb + (size_t)r1 * HD + k * 16 + c);
+      qa[k][2] = ldcg_u32(Qb + (size_t)r0 * HD + k * 16 + c + 8);
+      qa[k][3] = ldcg_u32(Qb + (size_t)r1 * HD + k * 16 + c + 8);
     }
   }
 
