@@ -262,3 +262,18 @@ def test_full_size_benchmark_workloads(name, wl):
             print(name, "mode", mode, rep)
     finally:
         case.close()
+
+
+def test_more_layers_than_one_launch_holds():
+    """35 layers of the tiny widths: the persistent kernel runs them as two launches (32 + 3); the second
+    one starts from the residual stream and sums of squares the first one left."""
+    shape = synth.TINY.cut(35)
+    case = harness.Case(shape, torch.bfloat16, [70, 19], 4, seed=3).gpu_setup()
+    try:
+        for mode in (orc.GREEDY, orc.SAMPLING):
+            rep, g = _run(case, mode, options={"gemm_impl": 1, "step_impl": 1})
+            assert rep.exact + rep.margin == 2
+            rep0, g0 = _run(case, mode, options={"gemm_impl": 1, "step_impl": 0})
+            assert np.abs(g["hidden"] - g0["hidden"]).max() < 2e-2
+    finally:
+        case.close()
