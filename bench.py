@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 # helpers
 # ----------------------------------------------------------------------------------------------
 # DRAM bytes the persistent kernel moved per algorithmic byte in the ncu capture of a 4-layer cut
-# (2.8875 GB moved for 2.8626 GB of weights and cache; profiles/k_verify_mega_cfg3_4layers_full.md).
+# (2.8875 GB moved for 2.8626 GB of weights and cache; the ncu summary of that cut is under profiles/).
 # Traffic grows in proportion to the streamed bytes (nothing is re-read), so the full step's traffic
 # is the same ratio times its algorithmic bytes.  Set to None whenever the kernel changes until recaptured.
 MEGA_DRAM_TRAFFIC_RATIO = 1.0087
