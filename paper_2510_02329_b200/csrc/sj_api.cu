@@ -279,11 +279,14 @@ static bool tc_shapes_ok(const sj_model_config& c) {
 }
 
 typedef void (*MegaKernel)(const MegaMaps, const MegaParams, const StepArgs*, const KvView, const Work, const Dims);
-// The persistent kernel for a head dimension (64 or 128) and a number of row slots (4, 6 or 8).
-static MegaKernel mega_kernel(int hd, int ns) {
-  if (hd == 128) return ns == 4 ? k_verify_mega<128, 4> : (ns == 6 ? k_verify_mega<128, 6> : k_verify_mega<128, 8>);
-  return ns == 4 ? k_verify_mega<64, 4> : (ns == 6 ? k_verify_mega<64, 6> : k_verify_mega<64, 8>);
+// The persistent kernel for a head dimension (64 or 128), a number of row slots (4, 6 or 8), with or without
+// the timeline code.
+template <bool TR>
+static MegaKernel mega_kernel_t(int hd, int ns) {
+  if (hd == 128) return ns == 4 ? k_verify_mega<128, 4, TR> : (ns == 6 ? k_verify_mega<128, 6, TR> : k_verify_mega<128, 8, TR>);
+  return ns == 4 ? k_verify_mega<64, 4, TR> : (ns == 6 ? k_verify_mega<64, 6, TR> : k_verify_mega<64, 8, TR>);
 }
+static MegaKernel mega_kernel(int hd, int ns, bool trace) { return trace ? mega_kernel_t<true>(hd, ns) : mega_kernel_t<false>(hd, ns); }
 
 extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weights* w, void* cuda_stream,
                                       sj_target** out) {
@@ -438,7 +441,8 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     if (e == cudaSuccess) e = cudaMemset(t->d_sumsq, 0, sizeof(float) * 2 * (c.d_model / kTileN) * kMegaMaxRows);
     if (e == cudaSuccess) e = cudaMemset(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)4 * t->sm_count * pad16(Rm) * kTileN));
     for (int ns = 4; ns <= 8 && e == cudaSuccess; ns += 2)
-      e = cudaFuncSetAttribute(mega_kernel(c.head_dim, ns), cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      for (int tr = 0; tr < 2 && e == cudaSuccess; ++tr)
+        e = cudaFuncSetAttribute(mega_kernel(c.head_dim, ns, tr != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "whole-step kernel set-up: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
     for (int l0 = 0; l0 < c.n_layers; l0 += kMegaMaxLayers) {
       t->mega_maps.emplace_back();
@@ -1005,7 +1009,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
     const StepArgs* args = t->d_args;
     // row slots per epilogue thread: a group gets at most (min(R, 16) + 1) / 2 rows of a 16-row chunk
     const int ns = R <= 8 ? 4 : (R <= 12 ? 6 : 8);
-    CU_TRY(cudaLaunchKernelEx(&cfg, mega_kernel(dm.hd, ns), mm, p, args, kv->view, W, dm));
+    CU_TRY(cudaLaunchKernelEx(&cfg, mega_kernel(dm.hd, ns, t->opt_trace != 0), mm, p, args, kv->view, W, dm));
     if (timing) {
       CU_TRY(cudaEventRecord(eb, s));
       t->timed.push_back({"verify_step", ea, eb});

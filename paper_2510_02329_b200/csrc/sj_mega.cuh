@@ -100,8 +100,11 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)::"memory");
   return t;
 }
+// The timeline is compiled in only in the kernel's tracing instantiation (`kTr` in scope): the timer reads
+// are volatile and hold back the compiler's scheduling even when no trace is taken (1.7 % of a step).
 #define MEGA_EV(sidx, k)                                                                             \
   do {                                                                                               \
+    if constexpr (kTr)                                                                               \
     if (p.trace && blockIdx.x == p.trace_block && (sidx) < kMegaTraceSites)                                      \
       p.trace[2 * kMegaTraceBarriers + (sidx) * 8 + (k)] = global_timer_ns();                        \
   } while (0)
@@ -110,6 +113,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // owner-side ones, at [2*kMegaTraceBarriers + 8*kMegaTraceSites + 8*s + e]
 #define MEGA_EV2(blk, sidx, k)                                                                       \
   do {                                                                                               \
+    if constexpr (kTr)                                                                               \
     if (p.trace && blockIdx.x == p.trace_block + (blk) && (sidx) < kMegaTraceSites)                                  \
       p.trace[2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (sidx) * 8 + (k)] = global_timer_ns();  \
   } while (0)
@@ -292,14 +296,15 @@ __device__ __forceinline__ bool mega_spin_ge(const unsigned* word, unsigned targ
 // Device-wide barrier for the 256 workers of every block.  Returns false once the step is aborting.
 // Block-level barrier, then one thread publishes (fence, arrive) and waits (poll, fence): the fences are
 // cumulative over what the block barrier ordered before them.
+template <bool kTr>
 __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p, int* status, int& nbar, int wt) {
   fence_proxy_async();   // this phase's generic-proxy stores are read by other blocks' TMA loads
   bar_sync(1, kMegaWorkers);
   ++nbar;
   if (wt == 0) {
-    const bool tr = p.trace && blockIdx.x == p.trace_block && nbar < kMegaTraceBarriers;
+    const bool tr = kTr && p.trace && blockIdx.x == p.trace_block && nbar < kMegaTraceBarriers;
     if (tr) p.trace[2 * nbar] = global_timer_ns();
-    if (p.trace && nbar < kMegaTraceAllBarriers) p.trace[kMegaTraceArrive + nbar * 256 + blockIdx.x] = global_timer_ns();
+    if (kTr && p.trace && nbar < kMegaTraceAllBarriers) p.trace[kMegaTraceArrive + nbar * 256 + blockIdx.x] = global_timer_ns();
     if (!ctl->abort_flag) {
       __threadfence();
       red_relaxed_add(p.gbar, 1u);
@@ -307,7 +312,7 @@ __device__ __forceinline__ bool mega_grid_sync(MegaCtl* ctl, const MegaParams& p
     }
     __threadfence();
     if (tr) p.trace[2 * nbar + 1] = global_timer_ns();
-    if (p.trace && nbar < kMegaTraceAllBarriers) p.trace[kMegaTraceRelease + nbar * 256 + blockIdx.x] = global_timer_ns();
+    if (kTr && p.trace && nbar < kMegaTraceAllBarriers) p.trace[kMegaTraceRelease + nbar * 256 + blockIdx.x] = global_timer_ns();
     *reinterpret_cast<volatile int*>(&ctl->bars_passed) = nbar;
   }
   bar_sync(1, kMegaWorkers);
@@ -367,7 +372,7 @@ __device__ __forceinline__ int mega_row_group(int r, int R) {
 // NS: row slots a thread unrolls per chunk (4, 6 or 8): at least the rows a group gets of a 16-row chunk.
 // Every slot's instructions issue whether its row exists or not, so the kernel is instantiated for the
 // slot counts 4 (up to 8 block rows), 6 (up to 12) and 8.
-template <int HD, int NS>
+template <int HD, int NS, bool kTr>
 __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& seg, MegaCtl* ctl, const MegaParams& p, const StepArgs* __restrict__ args, const KvView& kv,
                                               const Work& w, const Dims& dm, int wt) {
   const int et = wt & 127, grp = wt >> 7, bar_id = 2 + grp;
@@ -902,7 +907,7 @@ __device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p,
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int HD, int SLOTS>
+template <int HD, int SLOTS, bool kTr>
 __global__ void __launch_bounds__(kMegaThreads, 1)
 k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const StepArgs* __restrict__ args, const KvView kv,
               const Work w, const Dims dm) {
@@ -1128,14 +1133,14 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     bool alive = true;
     if (p.do_embed) {
       mega_embed(ctl, p, args, kv, w, dm, wt);
-      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+      alive = mega_grid_sync<kTr>(ctl, p, w.status, nbar, wt);
     }
     auto units = [&](int site) -> int { return site_units(site_split(site, dm, c, G)); };
     auto gemm_phase = [&](int site, int l) {
       ++gseq;
-      if (alive) mega_epilogue<HD, SLOTS>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
+      if (alive) mega_epilogue<HD, SLOTS, kTr>(site, l, gseq, seg, ctl, p, args, kv, w, dm, wt);
       it += units(site);
-      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+      alive = mega_grid_sync<kTr>(ctl, p, w.status, nbar, wt);
     };
     const int n_ph = mega_n_phases(p);
     for (int ph = 0; ph < n_ph; ++ph) {
@@ -1148,7 +1153,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       // attention over the cache tiles of the ring, then the combine
       if (alive) {
         // attention events of block 0 go to the second event set of the layer's QKV phase
-        unsigned long long* ev = (p.trace && c == 0 && (l - p.l0) * 4 < kMegaTraceSites)
+        unsigned long long* ev = (kTr && p.trace && c == 0 && (l - p.l0) * 4 < kMegaTraceSites)
                                      ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8
                                      : nullptr;
         AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status, ev};
@@ -1157,17 +1162,17 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
       }
       it += n_att;
-      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+      alive = mega_grid_sync<kTr>(ctl, p, w.status, nbar, wt);
       if (alive) {
         const AttPartials P{w.tc_m, w.tc_l, w.tc_o};
         const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;
         for (int item = ww * G + c; item < items; item += G * 8)   // spread over blocks first
           att_combine_item<bf16, HD>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane,
-                                     (p.trace && c == 0 && ww == 0 && (l - p.l0) * 4 < kMegaTraceSites)
+                                     (kTr && p.trace && c == 0 && ww == 0 && (l - p.l0) * 4 < kMegaTraceSites)
                                          ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8 + 4
                                          : nullptr);
       }
-      alive = mega_grid_sync(ctl, p, w.status, nbar, wt);
+      alive = mega_grid_sync<kTr>(ctl, p, w.status, nbar, wt);
     }
     if (p.do_lm && alive && c < B) mega_finalize(ctl, p, args, kv, w, dm, wt);
   }
