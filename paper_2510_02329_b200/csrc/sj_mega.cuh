@@ -45,7 +45,10 @@ constexpr int kMegaMaxRows = 80;
 constexpr int kMegaMaxStages = 12;
 constexpr uint32_t kMegaSpin = 1u << 22;
 constexpr int kMegaRegsLight = 80;    // registers per thread of warps 0..3 after reallocation
-constexpr int kMegaRegsHeavy = 208;   // registers per thread of the worker warps (128*96 + 256*200 <= 384*168)
+constexpr int kMegaRegsHeavy = 208;   // registers per thread of the worker warps
+// The block is launched with 168 registers per thread (384 threads); the workers' increase can only be granted
+// out of what the four light warps gave back, otherwise `setmaxnreg.inc` waits for ever.
+static_assert(128 * kMegaRegsLight + 256 * kMegaRegsHeavy <= kMegaThreads * 168, "register reallocation exceeds the block's registers");
 constexpr int kMegaTraceBarriers = 1024;
 constexpr int kMegaTraceSites = 512;
 constexpr int kMegaTraceAllBarriers = 32;   // barriers whose arrival / release time every block records
