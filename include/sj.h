@@ -103,6 +103,7 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *   "step_impl"  1 = the whole step as one persistent cooperative kernel (bf16, tcgen05 GEMMs, at most 80
  *                block rows; default when the shape allows), 0 = one kernel per stage
  *   "ring_stages" persistent kernel: cap on the shared-memory ring depth (0 = as many as fit, the default)
+ *   "tmem_slots"  persistent kernel: cap on the weight tiles parked in tensor memory, 2..14 (0 = as many as fit)
  *   "trace"      k > 0 = the persistent kernel records a timeline with the nanosecond global timer
  *                (sj_step_trace()): block k - 1 stamps its arrival at and release from every device-wide
  *                barrier and eight events per GEMM phase; every block stamps the first 32 barriers
@@ -188,9 +189,11 @@ typedef struct {
  * Errors before launch: INVALID_ARG, SHAPE (B*(gamma+1) > max_rows), OOM (page pool), STATE. */
 sj_status sj_verify(sj_target *t, sj_kv *kv, const sj_verify_args *args, const sj_verify_out *out);
 
-/* Truncate sequences to new_len <= current length (host arrays [B]).  Asynchronous; if new_len
- * exceeds the true length the device leaves the sequence unchanged and sj_sync() returns
- * SJ_ERR_STATE.  new_len above what the host knows could be live fails at once with STATE. */
+/* Truncate sequences to new_len <= current length (host arrays [B]) and return the whole pages
+ * past new_len to the pool (the KV-length rollback that follows the first-rejection scan, Sec. 3.1).
+ * Asynchronous; if new_len exceeds the true length the device leaves the sequence unchanged and
+ * sj_sync() returns SJ_ERR_STATE.  new_len above what the host knows could be live fails at once
+ * with STATE. */
 sj_status sj_rollback_kv(sj_kv *kv, const int *seq_ids, const int *new_len, int B);
 
 /* Skinny GEMM used by every projection of the step, exposed for kernel-level tests and
@@ -231,6 +234,21 @@ sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, const void *a
  * Errors: INVALID_ARG (null), SHAPE (sizes, scratch limit), UNSUPPORTED (not sm_100), CUDA, TIMEOUT. */
 enum { SJ_NOALLOC_SCRATCH_BYTES = 8 * 1024 * 1024 };
 sj_status sj_gemm_skinny_noalloc(int R, int N, int K, const void *a, const void *w, float *y, void *cuda_stream);
+
+/* Fault drill without a fault (the paper has no counterpart).  Every device-side wait of the library is
+ * bounded: when one runs out, the kernel records the fact, returns normally, and the next sj_sync() reports
+ * SJ_ERR_TIMEOUT; the context stays usable.  This call queues, on the target's stream, a one-block kernel
+ * that runs that same wait code on a barrier (kind 0: the stand-alone GEMM kernels' wait; kind 1: the ring /
+ * accumulator wait of the attention and whole-step kernels) or a device-memory word (kind 2: the whole-step
+ * kernel's device-wide barrier poll) that nothing will ever signal, with a limit of max_polls (1 .. 2^20)
+ * polls.  Use it to exercise an application's handling of SJ_ERR_TIMEOUT.  Nothing traps, faults or hangs.
+ * Errors: INVALID_ARG, UNSUPPORTED (the target was created without the whole-step kernel's workspace). */
+sj_status sj_debug_expire_wait(sj_target *t, int kind, unsigned max_polls);
+
+/* How many device-memory allocation and release calls (cudaMalloc / cudaFree) the library has made in this
+ * process so far.  Diagnostic (the paper has no counterpart): lets a caller check that a call it relies on
+ * to be allocation-free, such as sj_gemm_skinny_noalloc() or a steady-state sj_verify(), really made none. */
+long sj_device_memory_calls(void);
 
 const char *sj_last_error(void);
 

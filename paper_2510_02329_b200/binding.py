@@ -24,7 +24,7 @@ MODE_GREEDY, MODE_SAMPLING = 0, 1
 EXPORTS = ["sj_create_target", "sj_destroy_target", "sj_load_judge_head", "sj_set_option", "sj_sync",
            "sj_kv_create", "sj_kv_destroy", "sj_kv_fill", "sj_kv_read", "sj_kv_set_len", "sj_kv_set_pending",
            "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_gemm_skinny_noalloc", "sj_last_error",
-           "sj_kernel_time", "sj_step_trace"]
+           "sj_kernel_time", "sj_step_trace", "sj_device_memory_calls", "sj_debug_expire_wait"]
 
 
 class SjError(RuntimeError):
@@ -80,6 +80,9 @@ def load(build_if_needed: bool = True) -> C.CDLL:
     for name in EXPORTS:
         if name != "sj_last_error":
             getattr(lib, name).restype = C.c_int
+    lib.sj_debug_expire_wait.argtypes = [C.c_void_p, C.c_int, C.c_uint]
+    lib.sj_device_memory_calls.restype = C.c_long
+    lib.sj_device_memory_calls.argtypes = []
     lib.sj_create_target.argtypes = [C.POINTER(ModelConfig), C.POINTER(Weights), C.c_void_p, C.POINTER(C.c_void_p)]
     lib.sj_destroy_target.argtypes = [C.c_void_p]
     lib.sj_load_judge_head.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_float, C.c_float]
@@ -158,6 +161,10 @@ class Target:
 
     def sync(self) -> None:
         check(self._lib.sj_sync(self.handle))
+
+    def expire_wait(self, kind: int, max_polls: int = 2000) -> None:
+        """``sj_debug_expire_wait``: queue a one-block kernel whose bounded wait runs out (a drill for SJ_ERR_TIMEOUT)."""
+        check(self._lib.sj_debug_expire_wait(self.handle, int(kind), int(max_polls)))
 
     def kernel_time(self, name: str):
         """(total ms, launches) of the event-bracketed launches whose name starts with ``name``."""
@@ -287,3 +294,8 @@ def gemm_skinny_noalloc(a: torch.Tensor, w: torch.Tensor, y: torch.Tensor) -> No
     assert a.dtype == torch.bfloat16 and w.dtype == torch.bfloat16 and y.dtype == torch.float32 and y.shape == (R, N)
     check(load().sj_gemm_skinny_noalloc(R, N, K, _ptr(a), _ptr(w), _ptr(y),
                                         C.c_void_p(torch.cuda.current_stream().cuda_stream)))
+
+
+def device_memory_calls() -> int:
+    """``sj_device_memory_calls``: cudaMalloc / cudaFree calls the library has made so far in this process."""
+    return int(load().sj_device_memory_calls())

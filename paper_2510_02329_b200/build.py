@@ -1,6 +1,7 @@
 """Compile the CUDA library in-tree for sm_100a (no JIT cache: the .so sits beside this file)."""
 from __future__ import annotations
 
+import glob
 import os
 import subprocess
 import sys
@@ -8,9 +9,13 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(HERE, "csrc", "sj_api.cu")
 LIB = os.path.join(HERE, "libsjverify.so")
-DEPS = [os.path.join(HERE, "csrc", f) for f in ("sj_api.cu", "sj_common.cuh", "sj_kernels.cuh", "sj_gemm_tc.cuh",
-                                                 "sj_attn_tc.cuh")]
-DEPS.append(os.path.join(os.path.dirname(HERE), "include", "sj.h"))
+
+
+def deps():
+    """Every file the library is compiled from: all of csrc/ plus the public header."""
+    src = sorted(glob.glob(os.path.join(HERE, "csrc", "*.cu")) + glob.glob(os.path.join(HERE, "csrc", "*.cuh")))
+    return src + [os.path.join(os.path.dirname(HERE), "include", "sj.h")]
+
 
 
 def lib_path() -> str:
@@ -21,7 +26,7 @@ def needs_build() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.exists(d) and os.path.getmtime(d) > t for d in DEPS)
+    return any(os.path.getmtime(d) > t for d in deps())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

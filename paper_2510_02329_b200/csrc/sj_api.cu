@@ -1,6 +1,7 @@
 // Host runtime and C ABI of the verification step: handles, paged-KV bookkeeping, argument checks,
 // launch sequence (optionally replayed as a CUDA graph with programmatic dependent launches).
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -42,6 +43,19 @@ static sj_status fail(sj_status st, const char* fmt, ...) {
   } while (0)
 
 extern "C" const char* sj_last_error(void) { return g_err; }
+
+// Every device allocation and release of the library goes through these two, so that a caller (or a test)
+// can check that a call it believes allocation-free really is (sj_device_memory_calls()).
+static std::atomic<long> g_mem_calls{0};
+static cudaError_t counted_malloc(void** p, size_t bytes) {
+  g_mem_calls.fetch_add(1, std::memory_order_relaxed);
+  return cudaMalloc(p, bytes);
+}
+static cudaError_t counted_free(void* p) {
+  g_mem_calls.fetch_add(1, std::memory_order_relaxed);
+  return cudaFree(p);
+}
+extern "C" long sj_device_memory_calls(void) { return g_mem_calls.load(std::memory_order_relaxed); }
 
 // ---------------------------------------------------------------------------------------------
 // launch helper (programmatic dependent launch attribute on request)
@@ -134,12 +148,14 @@ static void build_tile_slots(int n_tiles, int KB, int G, std::vector<int2>& out,
 }
 
 struct RowGeom {  // how R activation rows are fed to the MMA
-  int NB, nblk, acc_stride, acc_bufs, stages, a_stage_bytes;
+  int NB, nblk, a_blocks, plane_rows, acc_stride, acc_bufs, stages, a_stage_bytes;
   uint32_t tmem_cols;
   size_t smem_bytes;
 };
 
-static RowGeom row_geom(int R) {
+// `merged`: R counts the rows of ONE plane; the stage holds both planes and the lo plane's products are
+// accumulated into the hi plane's columns.
+static RowGeom row_geom(int R, bool merged = false) {
   RowGeom g;
   int rp = round_up(std::max(R, 1), 16);
   g.NB = rp > 256 ? 2 : 1;
@@ -150,7 +166,9 @@ static RowGeom row_geom(int R) {
   uint32_t need = (uint32_t)(cols * g.acc_bufs), tc = 32;
   while (tc < need) tc <<= 1;
   g.tmem_cols = tc;
-  g.a_stage_bytes = round_up(cols * 128, 1024);
+  g.a_blocks = merged ? 2 * g.NB : g.NB;
+  g.plane_rows = merged ? rp : 0;
+  g.a_stage_bytes = round_up((merged ? 2 : 1) * cols * 128, 1024);
   int stage = kWTileBytes + g.a_stage_bytes;
   const int budget = 200 * 1024;
   g.stages = std::max(2, std::min(12, budget / stage));
@@ -190,7 +208,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_slots = 0;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -234,7 +252,7 @@ static void clear_graphs(sj_target* t) {
 template <typename T>
 static sj_status dev_alloc(sj_target* t, T** p, size_t n) {
   void* q = nullptr;
-  cudaError_t e = cudaMalloc(&q, std::max<size_t>(n, 1) * sizeof(T));
+  cudaError_t e = counted_malloc(&q, std::max<size_t>(n, 1) * sizeof(T));
   if (e != cudaSuccess) {
     cudaGetLastError();
     return fail(e == cudaErrorMemoryAllocation ? SJ_ERR_OOM : SJ_ERR_CUDA, "cudaMalloc(%zu bytes): %s", n * sizeof(T),
@@ -484,7 +502,7 @@ extern "C" sj_status sj_destroy_target(sj_target* t) {
   cudaStreamSynchronize(t->stream);
   clear_graphs(t);
   for (auto& e : t->timed) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
-  for (void* p : t->owned) cudaFree(p);
+  for (void* p : t->owned) counted_free(p);
   delete t;
   cudaGetLastError();
   return SJ_OK;
@@ -519,6 +537,9 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
   } else if (n == "ring_stages") {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
+  } else if (n == "tmem_slots") {
+    if (value != 0 && (value < 2 || value > kMegaMaxSlots)) return fail(SJ_ERR_INVALID_ARG, "tmem_slots must be 0 (auto) or 2..%d", kMegaMaxSlots);
+    t->opt_slots = value;
   } else if (n == "trace") {
     const size_t n_tr = kMegaTraceEntries;
     if (value && !t->d_trace) {
@@ -562,6 +583,39 @@ extern "C" sj_status sj_sync(sj_target* t) {
   return SJ_OK;
 }
 
+// One block whose first thread runs one of the library's bounded waits on something that nothing will ever
+// signal, with a small poll limit: the wait gives up, records DEV_TIMEOUT, and the kernel returns normally.
+__global__ void k_expire_wait(int kind, uint32_t limit, unsigned* word, int* abort_g, int* status) {
+  __shared__ uint64_t bar;
+  __shared__ MegaCtl ctl;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    ctl.abort_flag = 0;
+    if (kind == 0) {
+      mbar_wait(smem_u32(&bar), 0, &ctl.abort_flag, status, limit);                      // stand-alone GEMM kernels
+    } else if (kind == 1) {
+      att_mbar_wait(smem_u32(&bar), 0, &ctl.abort_flag, status, abort_g, 15, 0, limit);  // ring / accumulator waits
+    } else {
+      MegaParams p;
+      p.abort_g = abort_g;
+      mega_spin_ge(word, 1u, &ctl, p, status, 15, 0, limit);                             // device-wide barrier poll
+    }
+  }
+}
+
+extern "C" sj_status sj_debug_expire_wait(sj_target* t, int kind, unsigned max_polls) {
+  if (!t) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (kind < 0 || kind > 2) return fail(SJ_ERR_INVALID_ARG, "kind must be 0, 1 or 2");
+  if (max_polls == 0 || max_polls > (1u << 20)) return fail(SJ_ERR_INVALID_ARG, "max_polls must be in [1, 2^20]");
+  if (!t->d_sync) return fail(SJ_ERR_UNSUPPORTED, "this target has no whole-step kernel workspace");
+  // [1] abort word, [2..3] timeout note (as in a step), [8] the word that stays zero
+  CU_TRY(cudaMemsetAsync(t->d_sync, 0, sizeof(unsigned) * 16, t->stream));
+  CU_TRY(launch(k_expire_wait, dim3(1), dim3(32), 0, t->stream, false, kind, (uint32_t)max_polls, t->d_sync + 8,
+                reinterpret_cast<int*>(t->d_sync + 1), t->work.status));
+  return SJ_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // KV cache
 // ---------------------------------------------------------------------------------------------
@@ -578,13 +632,13 @@ extern "C" sj_status sj_kv_create(sj_target* t, int max_seqs, long max_pages, in
   const size_t page_elems = (size_t)2 * t->dm.Hkv * page_size * t->dm.hd;
   const size_t bytes = (size_t)t->dm.n_layers * max_pages * page_elems * esz;
   void* pool = nullptr;
-  cudaError_t e = cudaMalloc(&pool, bytes);
+  cudaError_t e = counted_malloc(&pool, bytes);
   int* meta = nullptr;
   const int mpps = (int)std::min<long>(max_pages, 1 << 20);
-  if (e == cudaSuccess) e = cudaMalloc((void**)&meta, sizeof(int) * ((size_t)max_seqs * (mpps + 2) + 2 * SJ_MAX_BATCH));
+  if (e == cudaSuccess) e = counted_malloc((void**)&meta, sizeof(int) * ((size_t)max_seqs * (mpps + 2) + 2 * SJ_MAX_BATCH));
   if (e != cudaSuccess) {
     cudaGetLastError();
-    if (pool) cudaFree(pool);
+    if (pool) counted_free(pool);
     delete kv;
     return fail(e == cudaErrorMemoryAllocation ? SJ_ERR_OOM : SJ_ERR_CUDA, "KV pool of %zu bytes: %s", bytes,
                 cudaGetErrorString(e));
@@ -599,8 +653,8 @@ extern "C" sj_status sj_kv_create(sj_target* t, int max_seqs, long max_pages, in
   }
   if (e != cudaSuccess) {
     cudaGetLastError();
-    cudaFree(pool);
-    cudaFree(meta);
+    counted_free(pool);
+    counted_free(meta);
     delete kv;
     return fail(SJ_ERR_CUDA, "KV pool clear: %s", cudaGetErrorString(e));
   }
@@ -628,8 +682,8 @@ extern "C" sj_status sj_kv_destroy(sj_kv* kv) {
   if (!kv) return SJ_OK;
   cudaStreamSynchronize(kv->t->stream);
   clear_graphs(kv->t);  // captured steps hold this cache's pointers
-  cudaFree(kv->view.pool);
-  cudaFree(kv->d_block_table);
+  counted_free(kv->view.pool);
+  counted_free(kv->d_block_table);
   delete kv;
   cudaGetLastError();
   return SJ_OK;
@@ -766,26 +820,36 @@ extern "C" sj_status sj_rollback_kv(sj_kv* kv, const int* seq_ids, const int* ne
   CU_TRY(cudaMemcpyAsync(kv->d_tmp, stage, sizeof(int) * 2 * B, cudaMemcpyHostToDevice, kv->t->stream));
   CU_TRY(launch(k_rollback, dim3((B + 127) / 128), dim3(128), 0, kv->t->stream, false, kv->view, (const int*)kv->d_tmp,
                 (const int*)(kv->d_tmp + B), B, kv->t->work.status));
-  for (int i = 0; i < B; ++i) kv->len_hi[seq_ids[i]] = new_len[i];  // still an upper bound if the device refuses
+  // Whole pages past the new length go back to the pool.  Everything that still touches them (a verify in
+  // flight, this rollback) was enqueued on the target's stream before any later call can hand them out
+  // again, and that call's kernels run on the same stream.  If the device refuses the rollback (the live
+  // length turned out shorter than new_len) the pages kept for new_len still cover it.
+  for (int i = 0; i < B; ++i) {
+    kv->len_hi[seq_ids[i]] = new_len[i];
+    release_beyond(kv, seq_ids[i], new_len[i]);
+  }
   return SJ_OK;
 }
 
 // ---------------------------------------------------------------------------------------------
 // the step
 // ---------------------------------------------------------------------------------------------
-// Rows handed to the MMA for R activation rows: both bf16 planes (hi at row 0, lo at row pad16(R)) while
-// they fit the 512 TMEM columns, else the hi plane alone.
+// How R activation rows reach the MMA.  Two bf16 planes (hi at row 0, lo at row pad16(R)): as 2 * pad16(R)
+// accumulator columns that the epilogue adds, while those fit the 512 TMEM columns; beyond that (R > 256)
+// the lo plane's products are accumulated into the hi plane's columns by a second MMA per K step.
 static bool planes_fit(int R) { return 2 * pad16(R) <= 512; }
-static int fed_rows(int R, bool planes) { return planes && planes_fit(R) ? 2 * pad16(R) : R; }
+static RowGeom feed_geom(int R, bool planes) {
+  if (!planes) return row_geom(R);
+  return planes_fit(R) ? row_geom(2 * pad16(R)) : row_geom(pad16(R), true);
+}
 
 static sj_status activation_map(sj_target* t, std::map<int, CUtensorMap>& cache, const void* base, int R, int K,
                                 const CUtensorMap** out) {
   auto it = cache.find(R);
   if (it == cache.end()) {
     CUtensorMap m;
-    const int fed = fed_rows(R, true);
-    RowGeom g = row_geom(fed);
-    sj_status st = make_map(&m, base, fed, K, g.nblk);
+    RowGeom g = feed_geom(R, true);
+    sj_status st = make_map(&m, base, 2 * pad16(R), K, g.nblk);
     if (st != SJ_OK) return st;
     it = cache.emplace(R, m).first;
   }
@@ -795,10 +859,11 @@ static sj_status activation_map(sj_target* t, std::map<int, CUtensorMap>& cache,
 
 static cudaError_t launch_tc(sj_target* t, const TcSite& s, const CUtensorMap* mA, const CUtensorMap* w0,
                              const CUtensorMap* w1, const CUtensorMap* w2, int R, bool pdl, bool planes) {
-  RowGeom g = row_geom(fed_rows(R, planes));
+  RowGeom g = feed_geom(R, planes);
   TcGemmParams p;
   memset(&p, 0, sizeof(p));
   p.lo_off = (planes && planes_fit(R)) ? pad16(R) : 0;
+  p.a_blocks = g.a_blocks; p.plane_rows = g.plane_rows;
   p.n_tiles = s.n_tiles; p.KB = s.KB; p.G = s.G; p.U = (long long)s.n_tiles * s.KB; p.R = R;
   p.NB = g.NB; p.nblk = g.nblk; p.N_total = s.N;
   for (int i = 0; i < 3; ++i) p.seg_tile_end[i] = s.seg_tile_end[i];
@@ -957,15 +1022,20 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   MegaParams p;
   memset(&p, 0, sizeof(p));
   p.B = B; p.rows = rows; p.R = R; p.Rp = Rp;
-  p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
+  // shared memory: a ring of 16 KiB stages (weight tiles on their way to TMEM, cache tiles), then one
+  // activation slice per TMEM weight slot; tensor memory: 4 * Rp accumulator columns, 32 per weight slot
+  p.stage_bytes = kWTileBytes;
+  p.a_bytes = round_up(2 * Rp * 128, 1024);
   const int ctl_bytes = ((int)sizeof(MegaCtl) + 127) & ~127;
   const int budget = 227 * 1024 - 1024 - ctl_bytes;
-  p.stages = std::min(8, std::min(kMegaMaxStages, budget / p.stage_bytes));   // deeper rings did not measure faster; the rest stays L1
-  if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
+  int slots = std::min(kMegaMaxSlots, (512 - 4 * Rp) / 32);
+  while (slots > 2 && budget - slots * p.a_bytes < 4 * kWTileBytes) --slots;
+  p.slots = slots;
+  p.stages = std::min(8, std::min(kMegaMaxStages, (budget - slots * p.a_bytes) / kWTileBytes));   // deeper rings did not measure faster; the rest stays L1
+  if (p.stages < 3 || slots < 2) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
   if (t->opt_ring) p.stages = std::min(p.stages, t->opt_ring);
-  uint32_t tc = 32;
-  while (tc < (uint32_t)(4 * Rp)) tc <<= 1;
-  p.tmem_cols = tc;
+  if (t->opt_slots) p.slots = std::max(2, std::min(p.slots, t->opt_slots));
+  p.tmem_cols = 512;
   p.lp = t->d_layer_ptrs;
   p.embed = (const bf16*)t->embed;
   p.gain0 = (const bf16*)t->layers[0].na;
@@ -977,7 +1047,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.trace = t->opt_trace ? t->d_trace : nullptr;
   p.trace_block = t->opt_trace ? (unsigned)std::min(t->opt_trace - 1, t->sm_count - 1) : 0u;
   const int grid = t->sm_count;
-  const size_t smem = (size_t)p.stages * p.stage_bytes + ctl_bytes + 1024;
+  const size_t smem = (size_t)p.stages * p.stage_bytes + (size_t)p.slots * p.a_bytes + ctl_bytes + 1024;
   const bool timing = t->opt_timing != 0;
   const int NL = dm.n_layers;
   for (size_t ci = 0; ci < t->mega_maps.size(); ++ci) {
@@ -1113,7 +1183,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
     int rcap = std::max(rows, t->att_rows_cap);
     for (float** p : {&t->work.att_m, &t->work.att_l, &t->work.att_o}) {
       if (*p) {
-        cudaFree(*p);
+        counted_free(*p);
         t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)*p), t->owned.end());
         *p = nullptr;
       }
@@ -1133,7 +1203,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
       clear_graphs(t);
       for (float** p : {&t->work.tc_m, &t->work.tc_l, &t->work.tc_o}) {
         if (*p) {
-          cudaFree(*p);
+          counted_free(*p);
           t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)*p), t->owned.end());
           *p = nullptr;
         }
@@ -1153,7 +1223,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
     CU_TRY(cudaStreamSynchronize(t->stream));
     clear_graphs(t);
     if (t->work.logits) {
-      cudaFree(t->work.logits);
+      counted_free(t->work.logits);
       t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)t->work.logits), t->owned.end());
       t->work.logits = nullptr;
     }
@@ -1258,7 +1328,7 @@ extern "C" sj_status sj_gemm_skinny(int dtype, int impl, int R, int N, int K, co
   TcSite site;
   int seg[1] = {N};
   sj_status st = setup_site(&tmp, site, 1, seg, K, false);
-  auto cleanup = [&]() { for (void* p : tmp.owned) cudaFree(p); };
+  auto cleanup = [&]() { for (void* p : tmp.owned) counted_free(p); };
   if (st != SJ_OK) { cleanup(); return st; }
   float* P = nullptr;
   int* status = nullptr;

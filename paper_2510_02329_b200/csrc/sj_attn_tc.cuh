@@ -395,8 +395,8 @@ __device__ __forceinline__ void att_note_timeout(volatile int* abort_g, int wher
 // and with almost all of the SM's memory configured as shared memory a local-memory access costs an L2
 // round trip.)
 __device__ __forceinline__ bool att_mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                                volatile int* abort_g, int where, int extra) {
-  for (uint32_t i = 0; i < kAttSpin; ++i) {
+                                                volatile int* abort_g, int where, int extra, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (att_mbar_try(bar, parity)) return true;
     if (i > 64) {
       if (*abort_flag) return false;
@@ -411,9 +411,10 @@ __device__ __forceinline__ bool att_mbar_wait_slow(uint32_t bar, uint32_t parity
   return false;
 }
 __device__ __forceinline__ bool att_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                              volatile int* abort_g = nullptr, int where = 0, int extra = 0) {
+                                              volatile int* abort_g = nullptr, int where = 0, int extra = 0,
+                                              uint32_t limit = kAttSpin) {
   if (att_mbar_try(bar, parity)) return true;
-  return att_mbar_wait_slow(bar, parity, abort_flag, status, abort_g, where, extra);
+  return att_mbar_wait_slow(bar, parity, abort_flag, status, abort_g, where, extra, limit);
 }
 __device__ __forceinline__ void att_tma_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
   asm volatile(

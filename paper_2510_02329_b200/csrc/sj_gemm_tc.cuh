@@ -35,11 +35,14 @@ struct TcGemmParams {
   int R;                // valid rows
   int lo_off;           // > 0: activations come as hi/lo bf16 planes; the lo plane's accumulator
                         // columns start at lo_off and are added to the hi columns in the epilogue
-  int NB, nblk;         // activation rows are fed as NB blocks of nblk rows (nblk % 16 == 0, <= 256)
+  int NB, nblk;         // the accumulator holds NB blocks of nblk rows (nblk % 16 == 0, <= 256)
+  int a_blocks;         // activation blocks of nblk rows per stage: NB, or 2 * NB when the hi and the lo plane
+                        // are accumulated into the SAME columns (block i adds into accumulator block i % NB)
+  int plane_rows;       // row of the lo plane's first block in the activation matrix (used when a_blocks > NB)
   int N_total;          // output features (all segments)
   int seg_tile_end[3];  // exclusive prefix of tiles per weight segment
   int stages;
-  int a_stage_bytes;    // NB*nblk*128 rounded up to 1024
+  int a_stage_bytes;    // a_blocks*nblk*128 rounded up to 1024
   uint32_t tmem_cols;   // power of two >= 32
   int acc_bufs;         // 1 or 2
   int acc_stride;       // columns per accumulator buffer
@@ -72,9 +75,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls or when another thread of the block gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+// Non-blocking look at a barrier phase (try_wait may suspend the thread for a while before it answers: right
+// for a dedicated waiter, wrong for a thread that polls several barriers in turn).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after `limit` polls or when another thread of the block gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          uint32_t limit = kSpinLimit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 64) {
       if (*abort_flag) return false;
@@ -116,6 +133,21 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+// The same MMA with the A operand (128 rows x 16 bf16 = 8 columns of 32 bits per row) in tensor memory.
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Copy 128 rows x 32 bytes of a shared-memory tile (described like an MMA operand; one 16-element K step of a
+// 128-byte-swizzled bf16 tile) into tensor memory: row i to lane i, 8 columns from `taddr`.
+__device__ __forceinline__ void tc_cp_128x256b(uint32_t taddr, uint64_t s_desc) {
+  asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
 }
 __device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
   uint32_t r[8];
@@ -216,7 +248,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       const uint64_t pol_w = l2_policy_evict_first(), pol_a = l2_policy_evict_last();
-      const uint32_t tx_bytes = kWTileBytes + (uint32_t)p.NB * p.nblk * 128;
+      const uint32_t tx_bytes = kWTileBytes + (uint32_t)p.a_blocks * p.nblk * 128;
       auto w_load = [&](int it) {
         long long u = u_lo + it;
         int tile = (int)(u / p.KB), kb = (int)(u % p.KB);
@@ -234,9 +266,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         int kb = (int)(u % p.KB);
         int s = it % p.stages;
         uint32_t bar = smem_u32(&ctl->full[s]);
-        for (int nb = 0; nb < p.NB; ++nb)
+        for (int nb = 0; nb < p.a_blocks; ++nb)
           tma_load_2d(smem_u32(smem + (size_t)s * stage_bytes + kWTileBytes + (size_t)nb * p.nblk * 128), &tmA, bar,
-                      kb * kBK, nb * p.nblk, pol_a);
+                      kb * kBK, (nb / p.NB) * p.plane_rows + (nb % p.NB) * p.nblk, pol_a);
       };
       const int pre = min(p.stages, n_units);
       for (int it = 0; it < pre; ++it) w_load(it);   // weights never depend on the previous kernel
@@ -271,12 +303,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           tc_fence_after();
           uint32_t wa = smem_u32(smem + (size_t)s * stage_bytes);
           uint64_t dw = smem_desc_sw128(wa);
-          for (int nb = 0; nb < p.NB; ++nb) {
+          for (int nb = 0; nb < p.a_blocks; ++nb) {
             uint64_t da = smem_desc_sw128(wa + kWTileBytes + nb * p.nblk * 128);
-            uint32_t dcol = tmem_base + acc * p.acc_stride + nb * p.nblk;
+            uint32_t dcol = tmem_base + acc * p.acc_stride + (nb % p.NB) * p.nblk;
 #pragma unroll
             for (int k = 0; k < kBK / 16; ++k)
-              tc_mma_bf16(dcol, dw + 2 * k, da + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+              tc_mma_bf16(dcol, dw + 2 * k, da + 2 * k, idesc, (i > 0 || k > 0 || nb >= p.NB) ? 1u : 0u);
           }
           tc_commit(smem_u32(&ctl->empty[s]));  // frees the ring slot once these MMAs have read it
         }

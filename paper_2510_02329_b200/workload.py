@@ -10,6 +10,38 @@ import torch
 from . import binding, synth
 
 
+def target_following_drafts(target: "binding.Target", kv: "binding.KVCache", seq_ids, pending, vocab: int, gamma: int,
+                            match_prob: float, seed: int = 0) -> np.ndarray:
+    """Draft ids ``[B, gamma]`` that equal the target's greedy token, given the block so far, with probability
+    ``match_prob`` per position and are uniform over the vocabulary otherwise.
+
+    The greedy token after ``[x_t, d_1 .. d_j]`` is read off the library itself: a step over those j drafts
+    with the alignment test off and the judge threshold at 0 accepts every position (a sigmoid is positive),
+    so its next token is the arg max of the block's last row.  gamma such steps (uncommitted: the cache is left
+    as it was) give the chain position by position; the choices are seeded and the drafts are then fixed inputs.
+    """
+    B = len(seq_ids)
+    rng = np.random.Generator(np.random.Philox(key=[seed, 21]))
+    follow = rng.random((B, gamma)) < match_prob
+    other = rng.integers(0, vocab, size=(B, gamma), dtype=np.int64).astype(np.int32)
+    drafts = np.zeros((B, gamma), dtype=np.int32)
+    kv.set_pending(seq_ids, pending)
+    for j in range(gamma):
+        if j == 0:
+            # a one-draft block with both tests off rejects at once: the next token is row 0's arg max
+            blk, flags = torch.zeros((B, 1), dtype=torch.int32, device="cuda"), dict(use_align=False, use_judge=False)
+        else:
+            blk = torch.from_numpy(np.ascontiguousarray(drafts[:, :j])).cuda()
+            flags = dict(use_align=False, use_judge=True, theta=0.0)
+        out = binding.VerifyBuffers(B, blk.shape[1])
+        binding.verify(target, kv, seq_ids, blk, out, mode=binding.MODE_GREEDY, commit=False, **flags)
+        target.sync()
+        assert j == 0 or bool((out.accepted_len == j).all()), "a judge threshold of 0 must accept every position"
+        greedy = out.next_token.cpu().numpy()
+        drafts[:, j] = np.where(follow[:, j], greedy, other[:, j])
+    return drafts
+
+
 class DeviceWorkload:
     def __init__(self, wl: synth.Workload, dtype: torch.dtype = torch.bfloat16, seed: int = 0,
                  n_layers: Optional[int] = None, stream: Optional[torch.cuda.Stream] = None,
@@ -46,6 +78,10 @@ class DeviceWorkload:
                 self.kv.fill(b, l, 0, k, v)
         self.kv.set_len(self.seq_ids, self.kv_lens)
         self.inputs = synth.step_inputs(shape.vocab, self.B, self.gamma, seed, draft_ids=draft_ids)
+        if draft_ids is None and wl.draft_match_prob > 0.0:
+            d = target_following_drafts(self.target, self.kv, self.seq_ids, self.inputs.pending, shape.vocab, self.gamma,
+                                        wl.draft_match_prob, seed)
+            self.inputs = synth.step_inputs(shape.vocab, self.B, self.gamma, seed, draft_ids=d)
         self.upload_inputs()
         self.out = binding.VerifyBuffers(self.B, self.gamma)
         torch.cuda.synchronize()

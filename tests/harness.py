@@ -56,12 +56,44 @@ class Case:
         self.inputs = synth.step_inputs(shape.vocab, self.B, gamma, seed, draft_ids=draft_ids)
 
     # ---------------- oracle ----------------
-    def run_oracle(self, mode: int, temperature: float = 1.0, theta: float = 0.5, use_align=True, use_judge=True):
-        caches = [[(helpers.np64(k), helpers.np64(v)) for k, v in seq] for seq in self.cache_t]
+    def _oracle_caches(self):
+        """Per sequence, a sequence-like object whose item l is layer l's (K, V) widened to fp64 on demand: the
+        cache of a large workload does not fit host memory as fp64 all at once."""
+        cache_t = self.cache_t
+
+        class _Layers:
+            def __init__(self, seq):
+                self.seq = seq
+
+            def __len__(self):
+                return len(self.seq)
+
+            def __getitem__(self, l):
+                k, v = self.seq[l]
+                return helpers.np64(k), helpers.np64(v)
+
+        return [_Layers(seq) for seq in cache_t]
+
+    def oracle_forward(self):
+        """The target forward of the step (Eq. 2) for every sequence: independent of mode, temperature and theta."""
         si = self.inputs
-        return orc.verify(self.osh, self.top64, self.model.layer64, si.pending, si.draft_ids, caches, mode=mode,
-                          temperature=temperature, q_tok=si.draft_q_tok, q_full=si.draft_q_full, uniforms=si.uniforms,
-                          judge_w=self.judge_w64, judge_b=0.0, theta=theta, use_align=use_align, use_judge=use_judge)
+        tokens = [np.concatenate([[int(si.pending[b])], np.asarray(si.draft_ids[b], np.int64)]) for b in range(self.B)]
+        return orc.forward_blocks(self.osh, self.top64, self.model.layer64, tokens, self._oracle_caches())
+
+    def oracle_verdicts(self, fwd, mode: int, temperature: float = 1.0, theta: float = 0.5, use_align=True, use_judge=True):
+        """The acceptance decisions (Eq. 3, Eq. 5, Sec. 3.1-3.2) for a forward computed by oracle_forward()."""
+        si = self.inputs
+        return [orc.verdict(bf.logits, bf.hidden, np.asarray(si.draft_ids[b]), self.kv_lens[b], mode=mode,
+                            temperature=temperature, q_tok=si.draft_q_tok[b], q_full=si.draft_q_full[b],
+                            uniforms=si.uniforms[b], judge_w=self.judge_w64, judge_b=0.0, theta=theta,
+                            use_align=use_align, use_judge=use_judge) for b, bf in enumerate(fwd)]
+
+    def run_oracle(self, mode: int, temperature: float = 1.0, theta: float = 0.5, use_align=True, use_judge=True):
+        si = self.inputs
+        return orc.verify(self.osh, self.top64, self.model.layer64, si.pending, si.draft_ids, self._oracle_caches(),
+                          mode=mode, temperature=temperature, q_tok=si.draft_q_tok, q_full=si.draft_q_full,
+                          uniforms=si.uniforms, judge_w=self.judge_w64, judge_b=0.0, theta=theta, use_align=use_align,
+                          use_judge=use_judge)
 
     # ---------------- CUDA library ----------------
     def gpu_setup(self, max_rows: Optional[int] = None, page_slack: int = 8, shuffle_pages: bool = True):
@@ -100,6 +132,18 @@ class Case:
         self.d_qtok = torch.from_numpy(si.draft_q_tok).to(dev)
         self.d_qfull = torch.from_numpy(si.draft_q_full).to(dev)
         self.d_unif = torch.from_numpy(si.uniforms).to(dev)
+        return self
+
+    def follow_target(self, match_prob: float):
+        """Replace the drafts by ones that follow the target's greedy chain with probability ``match_prob`` per
+        position (the chain is read off the library; the drafts are then fixed inputs of both sides)."""
+        from paper_2510_02329_b200 import workload
+        d = workload.target_following_drafts(self.target, self.kv, self.seq_ids, self.inputs.pending, self.shape.vocab,
+                                             self.gamma, match_prob, self.seed)
+        self.inputs = synth.step_inputs(self.shape.vocab, self.B, self.gamma, self.seed, draft_ids=d)
+        si = self.inputs
+        self.d_draft = torch.from_numpy(si.draft_ids).cuda()
+        self.d_qtok = torch.from_numpy(si.draft_q_tok).cuda()
         return self
 
     def run_gpu(self, mode: int, temperature: float = 1.0, theta: float = -1.0, use_align=True, use_judge=True,

@@ -62,3 +62,22 @@ def test_compute_calls_fail_loudly_without_a_device():
     h = C.c_void_p()
     st = lib.sj_create_target(C.byref(cfg), C.byref(w), None, C.byref(h))
     assert st == 6 and not h.value, lib.sj_last_error()          # SJ_ERR_CUDA, never a silent CPU path
+
+
+def test_every_included_source_is_a_build_dependency():
+    """An edit of any file the library is compiled from must trigger a rebuild."""
+    from paper_2510_02329_b200 import build as b
+    deps = {os.path.basename(d) for d in b.deps()}
+    csrc = os.path.join(ROOT, "paper_2510_02329_b200", "csrc")
+    seen, todo = set(), ["sj_api.cu"]
+    while todo:
+        f = todo.pop()
+        if f in seen:
+            continue
+        seen.add(f)
+        for inc in re.findall(r'#include\s+"([^"]+)"', open(os.path.join(csrc, f)).read()):
+            name = os.path.basename(inc)
+            if os.path.exists(os.path.join(csrc, name)):
+                todo.append(name)
+            assert name in deps, f"{f} includes {inc}, which the build does not watch"
+    assert {"sj_api.cu", "sj_mega.cuh", "sj.h"} <= seen | deps

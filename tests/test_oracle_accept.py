@@ -165,3 +165,27 @@ def test_judge_score_closed_form():
     h = rng.standard_normal((5, 32)); w = rng.standard_normal(32); b = 0.37
     assert np.allclose(orc.judge_scores(h, w, b), scipy.special.expit(h @ w + b), rtol=1e-14, atol=0)
     assert orc.judge_scores(np.zeros((1, 32)), w, 0.0)[0] == 0.5
+
+
+def test_residual_with_zero_mass_falls_back_to_the_target_distribution():
+    """p == q at the rejected position (here both exactly uniform): max(0, p - q) has no mass, so the emitted
+    token is drawn from p itself.  With u = 0.6 over four equally likely tokens the inverse CDF gives token 2;
+    an all-zero weight vector would instead run off the end (token 3)."""
+    V = 4
+    logits = np.zeros((2, V))                       # softmax: exactly 0.25 each
+    hidden = np.zeros((2, 3))
+    q_full = np.full((1, V), 0.25)
+    # the scalar q handed over for the drafted token is larger than p, so u * q >= p rejects position 1
+    v = orc.verdict(logits, hidden, np.array([1]), 5, mode=orc.SAMPLING, temperature=1.0, q_tok=np.array([1.0]),
+                    q_full=q_full, uniforms=np.array([0.99, 0.6]), use_judge=False)
+    assert v.accepted_len == 0 and v.next_token == 2 and v.new_kv_len == 6
+    for u, tok in [(0.0, 0), (0.2499, 0), (0.25, 1), (0.74, 2), (0.76, 3)]:
+        v = orc.verdict(logits, hidden, np.array([1]), 5, mode=orc.SAMPLING, q_tok=np.array([1.0]), q_full=q_full,
+                        uniforms=np.array([0.99, u]), use_judge=False)
+        assert v.next_token == tok
+    # q above p everywhere it matters (q puts all its mass on one token the target gives 1/4): the residual is
+    # p on the other three tokens, renormalised; u = 0.5 lands on the middle one of them
+    q_full = np.array([[0.0, 1.0, 0.0, 0.0]])
+    v = orc.verdict(logits, hidden, np.array([1]), 5, mode=orc.SAMPLING, q_tok=np.array([1.0]), q_full=q_full,
+                    uniforms=np.array([0.99, 0.5]), use_judge=False)
+    assert v.accepted_len == 0 and v.next_token == 2
