@@ -103,7 +103,6 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *   "step_impl"  1 = the whole step as one persistent cooperative kernel (bf16, tcgen05 GEMMs, at most 80
  *                block rows; default when the shape allows), 0 = one kernel per stage
  *   "ring_stages" persistent kernel: cap on the shared-memory ring depth (0 = as many as fit, the default)
- *   "tmem_slots"  persistent kernel: cap on the weight tiles parked in tensor memory, 2..14 (0 = as many as fit)
  *   "trace"      k > 0 = the persistent kernel records a timeline with the nanosecond global timer
  *                (sj_step_trace()): block k - 1 stamps its arrival at and release from every device-wide
  *                barrier and eight events per GEMM phase; every block stamps the first 32 barriers

@@ -208,7 +208,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_slots = 0;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -537,9 +537,6 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
   } else if (n == "ring_stages") {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
-  } else if (n == "tmem_slots") {
-    if (value != 0 && (value < 2 || value > kMegaMaxSlots)) return fail(SJ_ERR_INVALID_ARG, "tmem_slots must be 0 (auto) or 2..%d", kMegaMaxSlots);
-    t->opt_slots = value;
   } else if (n == "trace") {
     const size_t n_tr = kMegaTraceEntries;
     if (value && !t->d_trace) {
@@ -1022,20 +1019,15 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   MegaParams p;
   memset(&p, 0, sizeof(p));
   p.B = B; p.rows = rows; p.R = R; p.Rp = Rp;
-  // shared memory: a ring of 16 KiB stages (weight tiles on their way to TMEM, cache tiles), then one
-  // activation slice per TMEM weight slot; tensor memory: 4 * Rp accumulator columns, 32 per weight slot
-  p.stage_bytes = kWTileBytes;
-  p.a_bytes = round_up(2 * Rp * 128, 1024);
+  p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
   const int ctl_bytes = ((int)sizeof(MegaCtl) + 127) & ~127;
   const int budget = 227 * 1024 - 1024 - ctl_bytes;
-  int slots = std::min(kMegaMaxSlots, (512 - 4 * Rp) / 32);
-  while (slots > 2 && budget - slots * p.a_bytes < 4 * kWTileBytes) --slots;
-  p.slots = slots;
-  p.stages = std::min(8, std::min(kMegaMaxStages, (budget - slots * p.a_bytes) / kWTileBytes));   // deeper rings did not measure faster; the rest stays L1
-  if (p.stages < 3 || slots < 2) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
+  p.stages = std::min(8, std::min(kMegaMaxStages, budget / p.stage_bytes));   // deeper rings did not measure faster; the rest stays L1
+  if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
   if (t->opt_ring) p.stages = std::min(p.stages, t->opt_ring);
-  if (t->opt_slots) p.slots = std::max(2, std::min(p.slots, t->opt_slots));
-  p.tmem_cols = 512;
+  uint32_t tc = 32;
+  while (tc < (uint32_t)(4 * Rp)) tc <<= 1;
+  p.tmem_cols = tc;
   p.lp = t->d_layer_ptrs;
   p.embed = (const bf16*)t->embed;
   p.gain0 = (const bf16*)t->layers[0].na;
@@ -1047,7 +1039,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.trace = t->opt_trace ? t->d_trace : nullptr;
   p.trace_block = t->opt_trace ? (unsigned)std::min(t->opt_trace - 1, t->sm_count - 1) : 0u;
   const int grid = t->sm_count;
-  const size_t smem = (size_t)p.stages * p.stage_bytes + (size_t)p.slots * p.a_bytes + ctl_bytes + 1024;
+  const size_t smem = (size_t)p.stages * p.stage_bytes + ctl_bytes + 1024;
   const bool timing = t->opt_timing != 0;
   const int NL = dm.n_layers;
   for (size_t ci = 0; ci < t->mega_maps.size(); ++ci) {

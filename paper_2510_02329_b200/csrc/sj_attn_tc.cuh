@@ -5,8 +5,8 @@
 // (one tile = 16 KiB: KPS keys of K and of V of one KV head; KPS = 32 for head_dim 128, 64 for head_dim
 // 64).  Tiles are ordered (sequence, KV head, tile) and block c owns tiles [c*T/G, (c+1)*T/G); every
 // maximal run of tiles of one (sequence, KV head) inside a block's range is a segment.  The block's own
-// gamma+1 new rows (positions L_b ..) are a separate "tail" segment per (sequence, KV head), read from
-// the pages with plain loads.  A segment's result is an unnormalised partial (running max m in the
+// gamma+1 new rows (positions L_b ..) are a separate "tail" segment per (sequence, KV head), read with
+// plain loads from the fp16 copy of those rows that the QKV epilogue writes beside the bf16 pages.  A segment's result is an unnormalised partial (running max m in the
 // log2 domain, sum l, output o) per query row; a combine pass merges the partials of a (sequence, KV
 // head) in a fixed order (deterministic).
 //

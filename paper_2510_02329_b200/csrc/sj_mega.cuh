@@ -11,18 +11,10 @@
 //
 // Roles per block (384 threads):
 //   warp 0      weight / cache-tile producer (TMA into the ring; never stops at a phase boundary)
-//   warp 1      tcgen05 issuer, owns the TMEM allocation: copies every weight tile from its ring stage into a
-//               TMEM slot as soon as it lands (tcgen05.cp; the stage is free again at once) and, in the same
-//               order but later, multiplies it (A operand in TMEM) with the activation slice of its slot
+//   warp 1      tcgen05.mma issuer, owns the TMEM allocation
 //   warp 2      activation producer: TMA of the activation K-slices, gated by the device-wide barrier
 //   warps 4..11 workers: all eight drain TMEM (fused epilogues, two groups of four warps) and run attention,
 //               the combine, the embedding and the final acceptance phase
-//
-// Weight buffering.  The loss of this kernel is the dependent chain at every phase boundary (last tile,
-// epilogue, split-K exchange, barrier, first activation slice), during which weights can only keep streaming
-// while there is room for them on the SM.  Besides the shared-memory ring, the part of tensor memory that
-// the accumulators leave free holds up to 14 more 16 KiB weight tiles (32 columns each): while a chain is in
-// flight the producer fills ring and TMEM with the next phase's first 20-odd tiles instead of 8.
 //
 // GEMM phases: work units are (128-feature tile, 64-wide K block) in tile-major order, dealt evenly to
 // the blocks (stream-K).  Partial sums of a tile that several blocks share travel as 64-bit words {fp32
@@ -50,7 +42,6 @@ constexpr int kMegaWorkers = 256;
 constexpr int kMegaMaxLayers = 32;   // per launch (tensor maps travel as kernel parameters)
 constexpr int kMegaMaxRows = 80;
 constexpr int kMegaMaxStages = 12;
-constexpr int kMegaMaxSlots = 14;    // TMEM weight slots (32 columns each) beside the accumulators
 constexpr uint32_t kMegaSpin = 1u << 22;
 constexpr int kMegaRegsLight = 80;    // registers per thread of warps 0..3 after reallocation
 constexpr int kMegaRegsHeavy = 208;   // registers per thread of the worker warps
@@ -81,9 +72,7 @@ struct MegaLayerPtrs {
 struct MegaParams {
   int l0, l1, do_embed, do_lm;
   int B, rows, R, Rp;
-  int stages, stage_bytes;    // ring of 16 KiB stages: weight tiles on their way to TMEM, and cache tiles
-  int slots, a_bytes;         // slot k: TMEM columns [4*Rp + 32k, +32) for a weight tile, and the activation
-                              // slice it is multiplied with, a_bytes of shared memory after the ring
+  int stages, stage_bytes;
   uint32_t tmem_cols;
   const MegaLayerPtrs* lp;    // [n_layers], device
   const bf16* embed;
@@ -133,10 +122,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 
 struct MegaCtl {
   uint64_t full[kMegaMaxStages], empty[kMegaMaxStages], tmem_full[2], tmem_empty[2];
-  uint64_t afull[kMegaMaxSlots];       // slot k's activation slice has landed
-  uint64_t slot_free[kMegaMaxSlots];   // the MMAs that read slot k (weights in TMEM, activations in shared memory) are done
   int cons_cnt[kMegaMaxStages];
-  int issued;                          // ring positions whose loads the weight producer has issued
   uint32_t tmem_base;
   int abort_flag;
   int bars_passed;
@@ -929,22 +915,17 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
               const Work w, const Dims dm) {
   extern __shared__ uint8_t mega_smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(mega_smem_raw) + 1023) & ~(uintptr_t)1023);
-  MegaCtl* ctl = reinterpret_cast<MegaCtl*>(ring + (size_t)p.stages * p.stage_bytes + (size_t)p.slots * p.a_bytes);
+  MegaCtl* ctl = reinterpret_cast<MegaCtl*>(ring + (size_t)p.stages * p.stage_bytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x, NS = p.stages, B = p.B, R = p.R, Rp = p.Rp, rows = p.rows;
   const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
-      mbar_init(smem_u32(&ctl->full[i]), 1);
+      mbar_init(smem_u32(&ctl->full[i]), 2);
       mbar_init(smem_u32(&ctl->empty[i]), 1);
       ctl->cons_cnt[i] = 0;
     }
-    for (int i = 0; i < p.slots; ++i) {
-      mbar_init(smem_u32(&ctl->afull[i]), 1);
-      mbar_init(smem_u32(&ctl->slot_free[i]), 1);
-    }
-    ctl->issued = 0;
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[i]), kMegaWorkers);
@@ -1003,8 +984,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     if (lane == 0) {
       const uint64_t pol_w = l2_policy_evict_first();
       RingPos rp{0, 0, NS};
-      int sidx = 0, n_issued = 0;
-      volatile int* issued = &ctl->issued;
+      int sidx = 0;
       bool alive = true;
       auto wait_slot = [&]() -> bool {
         return rp.r == 0 || mega_wait(smem_u32(&ctl->empty[rp.s]), (uint32_t)(rp.r - 1) & 1u, ctl, p, w.status, 1, rp.r);
@@ -1036,7 +1016,6 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
             tma_load_2d(dst, tm0, bar, kb * kBK, row, pol_w);
             if (site == SITE_GU) tma_load_2d(dst + 8192u, tm1, bar, kb * kBK, row, pol_w);
             rp.next();
-            *issued = ++n_issued;
           }
         }
         MEGA_EV(sidx, 7);
@@ -1048,175 +1027,72 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           if (!wait_slot()) { alive = false; return; }
           const uint32_t bar = smem_u32(&ctl->full[rp.s]);
           mbar_expect_tx(bar, kAttStageBytes);
+          mbar_arrive(bar);   // stands in for the activation producer, which skips cache tiles
           const AttTile x = att_locate(pl, B, g.KPS, (int)t);
           const int ai = (int)(t - t_lo) * (g.KPS / 16);
           att_issue_tile(&mp.pool, kv, l, args->seq_ids[x.b], x.h, x.ti, x.L, g.KPS, HD, stage_addr(rp.s), bar,
                          ai + g.KPS / 16 <= kAttPageCache ? ctl->att_pages + ai : nullptr);
           rp.next();
-          *issued = ++n_issued;
         }
       };
       mega_walk(p, fsite, fatt);
     }
   } else if (warp == 1) {
-    // ------------------------------ tcgen05 issuer ------------------------------
-    // Two cursors over this block's weight units, in unit order.  The MMA cursor multiplies a unit once its
-    // activation slice has landed (which needs the phase's device-wide barrier) and the accumulator is free:
-    // straight from the ring stage in the steady state of a phase.  While the NEXT phase cannot begin yet (its
-    // barrier has not been passed), the COPY cursor parks that phase's landed tiles in TMEM slot (unit % slots),
-    // up to `slots` units ahead, and frees their stages, so that the producer keeps streaming through the
-    // dependent chain at the phase boundary; the MMA cursor later takes those units from TMEM.  Units are
-    // always multiplied in unit order (the sums do not depend on timing); copies and MMAs issued by one thread
-    // execute in order.
-    // This one thread is the pace-maker of the steady state (a unit every 0.33 us): a dependent instruction
-    // costs it about five cycles, so every index below is kept incrementally (no division per unit) and in
-    // plain scalars (a struct handed to a helper by reference ends up in local memory, an L2 round trip).
+    // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(2 * Rp);
-      const uint32_t tmem_base = ctl->tmem_base, tmem_w = tmem_base + (uint32_t)(4 * Rp);
-      const int NT = p.slots, n_ph = mega_n_phases(p);
-      const uint32_t act0 = smem_u32(ring + (size_t)NS * p.stage_bytes), ring0 = smem_u32(ring);
-      const uint32_t a_bytes = (uint32_t)p.a_bytes, s_bytes = (uint32_t)p.stage_bytes;
-      const uint32_t bar_full = smem_u32(&ctl->full[0]), bar_empty = smem_u32(&ctl->empty[0]);
-      const uint32_t bar_afull = smem_u32(&ctl->afull[0]), bar_sfree = smem_u32(&ctl->slot_free[0]);
-      volatile int* issued = &ctl->issued;
-      volatile int* af = &ctl->abort_flag;
-      volatile int* bars_passed = &ctl->bars_passed;
-      // Per cursor: `ph` the next phase to open, `left` units left in the current phase, `pos` the unit's ring
-      // position with its stage `st` and the stage's phase parity `sp`, `nb` / `need` the device-wide barriers
-      // that must have been passed before the next / the current phase's activations exist.
-#define MEGA_OPEN(ph, left, pos, st, sp, nb, need, KB_out, u0)                                  \
-      while (left == 0 && ph < n_ph) {                                                            \
-        int site_, l_;                                                                            \
-        mega_phase(p, ph++, site_, l_);                                                           \
-        if (site_ < 0) {                                                                          \
-          pos += n_att;                                                                           \
-          st += n_att;                                                                            \
-          if (st >= NS) { sp ^= (uint32_t)(st / NS) & 1u; st %= NS; }                             \
-          continue;                                                                               \
-        }                                                                                         \
-        need = nb;                                                                                \
-        nb += (site_ == SITE_QKV) ? 3 : 1;                                                        \
-        const SiteInfo si_ = site_info(site_, dm, 0, 1);                                          \
-        const unsigned U_ = (unsigned)si_.n_tiles * (unsigned)si_.KB;                             \
-        const unsigned lo_ = (unsigned)c * U_ / (unsigned)G, hi_ = (unsigned)(c + 1) * U_ / (unsigned)G; \
-        left = (int)(hi_ - lo_);                                                                  \
-        KB_out = si_.KB;                                                                          \
-        u0 = (int)lo_;                                                                            \
-      }
-      int cc_ph = 0, cc_left = 0, cc_pos = 0, cc_st = 0, cc_nb = p.do_embed ? 1 : 0, cc_need = 0;
-      int cm_ph = 0, cm_left = 0, cm_pos = 0, cm_st = 0, cm_nb = p.do_embed ? 1 : 0, cm_need = 0;
-      uint32_t cc_sp = 0, cm_sp = 0;
-      // slot of the copy / MMA cursor's unit, the parity its slot barriers are waited with, and how far the
-      // copy cursor is ahead (units parked in TMEM)
-      int cc_slot = 0, cm_slot = 0, ahead = 0;
-      uint32_t cc_par = 1, cm_par = 0;       // slot_free is first waited for in the slot's second round
-      bool cc_first = true;                  // the copy cursor is in the slots' first round: nothing to wait for
-      int kb_c = 0, u_c = 0, KB_m = 1, u_m = 0, to_tile_end = 0;
-      MEGA_OPEN(cc_ph, cc_left, cc_pos, cc_st, cc_sp, cc_nb, cc_need, kb_c, u_c)
-      MEGA_OPEN(cm_ph, cm_left, cm_pos, cm_st, cm_sp, cm_nb, cm_need, KB_m, u_m)
-      to_tile_end = KB_m - u_m % KB_m;
-      int seg = 0, sidx = 0, n_done = 0;
-      bool seg_open = false;     // the current segment's accumulator has been claimed
-      bool seg_fresh = true;     // its first MMA overwrites the accumulator
-      uint32_t idle = 0;
-      (void)kb_c; (void)u_c;
-      while (cm_left > 0) {
-        bool did = false;
-        // MMA step: the next unit in order, from its TMEM slot if it was parked there, else straight from its
-        // ring stage (the steady state inside a phase: no copy at all)
-        {
-          const int acc = seg & 1;
-          if (!seg_open && (seg < 2 || mbar_test_wait(smem_u32(&ctl->tmem_empty[acc]), (uint32_t)((seg >> 1) - 1) & 1u))) seg_open = true;
-          if (seg_open && mbar_test_wait(bar_afull + 8u * (uint32_t)cm_slot, cm_par)) {
-            const bool parked = ahead > 0;
-            if (parked || (*issued > cm_pos && mbar_test_wait(bar_full + 8u * (uint32_t)cm_st, cm_sp))) {
-              tc_fence_after();
-              const uint32_t dcol = tmem_base + (uint32_t)(acc * 2 * Rp);
-              const uint64_t da = smem_desc_sw128(act0 + (uint32_t)cm_slot * a_bytes);
-              const uint32_t fresh = seg_fresh ? 0u : 1u;
-              if (parked) {
-                const uint32_t ta = tmem_w + (uint32_t)(32 * cm_slot);
-#pragma unroll
-                for (int k = 0; k < kBK / 16; ++k) tc_mma_bf16_ta(dcol, ta + (uint32_t)(8 * k), da + 2 * k, idesc, (k > 0) ? 1u : fresh);
-                --ahead;
-              } else {
-                const uint64_t dw = smem_desc_sw128(ring0 + (uint32_t)cm_st * s_bytes);
-#pragma unroll
-                for (int k = 0; k < kBK / 16; ++k) tc_mma_bf16(dcol, dw + 2 * k, da + 2 * k, idesc, (k > 0) ? 1u : fresh);
-                tc_commit(bar_empty + 8u * (uint32_t)cm_st);
-                // the copy cursor skips this unit
-                ++cc_pos; --cc_left;
-                if (++cc_st == NS) { cc_st = 0; cc_sp ^= 1u; }
-                if (++cc_slot == NT) { cc_slot = 0; cc_par ^= 1u; cc_first = false; }
-                MEGA_OPEN(cc_ph, cc_left, cc_pos, cc_st, cc_sp, cc_nb, cc_need, kb_c, u_c)
-              }
-              seg_fresh = false;
-              tc_commit(bar_sfree + 8u * (uint32_t)cm_slot);
-              ++cm_pos; --cm_left; ++n_done;
-              if (++cm_st == NS) { cm_st = 0; cm_sp ^= 1u; }
-              if (++cm_slot == NT) { cm_slot = 0; cm_par ^= 1u; }
-              if (--to_tile_end == 0 || cm_left == 0) {   // the segment ends with its tile or with the block's range
-                tc_commit(smem_u32(&ctl->tmem_full[acc]));
-                ++seg;
-                seg_open = false;
-                seg_fresh = true;
-                to_tile_end = KB_m;
-              }
-              if (cm_left == 0) {
-                MEGA_EV(sidx, 3);
-                ++sidx;
-                MEGA_OPEN(cm_ph, cm_left, cm_pos, cm_st, cm_sp, cm_nb, cm_need, KB_m, u_m)
-                to_tile_end = KB_m - u_m % KB_m;
-              }
-              did = true;
-            }
+      const uint32_t tmem_base = ctl->tmem_base;
+      RingPos rp{0, 0, NS};
+      int seg = 0, sidx = 0, nb = p.do_embed ? 1 : 0;
+      bool alive = true;
+      auto fsite = [&](int site, int l) {
+        if (!alive) return;
+        const SiteSplit ss = site_split(site, dm, c, G);
+        bool first = true;
+        unsigned u = ss.g_lo;
+        // Do not look at this phase's stages before the phase has begun: the attention phase in between
+        // may reuse a stage several times, and a parity wait started two uses early would be satisfied by
+        // the wrong one.
+        if (u < ss.g_hi && !mega_wait_bars(nb, ctl, p, w.status, 10)) { alive = false; return; }
+        nb += (site == SITE_QKV) ? 3 : 1;
+        Seg sg;
+        while (seg_next(ss, u, sg)) {
+          const int len = sg.b - sg.a;
+          if (len == 0) continue;   // no share of this segment: no accumulator is used
+          const int acc = seg & 1, use = seg >> 1;
+          if (use > 0 && !mega_wait(smem_u32(&ctl->tmem_empty[acc]), (uint32_t)(use - 1) & 1u, ctl, p, w.status, 4, seg)) {
+            alive = false;
+            return;
           }
-        }
-        // Copy step, only for tiles of a phase that has not begun (its activations cannot exist yet; inside a
-        // phase a tile waits for its slice in the ring: copies and MMAs share one pipe): park the next landed
-        // tile in a free TMEM slot and release its ring stage.
-        if (!did && cc_left > 0 && ahead < NT && cc_need > *bars_passed) {
-          if (*issued > cc_pos && mbar_test_wait(bar_full + 8u * (uint32_t)cc_st, cc_sp) &&
-              (cc_first || mbar_test_wait(bar_sfree + 8u * (uint32_t)cc_slot, cc_par))) {
+          tc_fence_after();
+          const uint32_t dcol = tmem_base + (uint32_t)(acc * 2 * Rp);
+          for (int i = 0; i < len; ++i) {
+            if (!mega_wait(smem_u32(&ctl->full[rp.s]), (uint32_t)rp.r & 1u, ctl, p, w.status, 5, rp.r)) { alive = false; return; }
             tc_fence_after();
-            const uint64_t dw = smem_desc_sw128(ring0 + (uint32_t)cc_st * s_bytes);
-            const uint32_t ta = tmem_w + (uint32_t)(32 * cc_slot);
+            if (first) { MEGA_EV(sidx, 2); first = false; }
+            const uint32_t wa = stage_addr(rp.s);
+            const uint64_t dw = smem_desc_sw128(wa), da = smem_desc_sw128(wa + kWTileBytes);
 #pragma unroll
-            for (int k = 0; k < kBK / 16; ++k) tc_cp_128x256b(ta + (uint32_t)(8 * k), dw + 2 * k);
-            tc_commit(bar_empty + 8u * (uint32_t)cc_st);   // the stage is free once the copy has read it
-            ++ahead;
-            ++cc_pos; --cc_left;
-            if (++cc_st == NS) { cc_st = 0; cc_sp ^= 1u; }
-            if (++cc_slot == NT) { cc_slot = 0; cc_par ^= 1u; cc_first = false; }
-            MEGA_OPEN(cc_ph, cc_left, cc_pos, cc_st, cc_sp, cc_nb, cc_need, kb_c, u_c)
-            did = true;
+            for (int k = 0; k < kBK / 16; ++k) tc_mma_bf16(dcol, dw + 2 * k, da + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            tc_commit(smem_u32(&ctl->empty[rp.s]));
+            rp.next();
           }
+          tc_commit(smem_u32(&ctl->tmem_full[acc]));
+          ++seg;
         }
-        if (did) { idle = 0; continue; }
-        if (++idle > 64) {
-          if (*af) break;
-          if ((idle & 255) == 0 && *reinterpret_cast<volatile int*>(p.abort_g)) { *af = 1; break; }
-          __nanosleep(idle > 4096 ? 128 : 20);
-          if (idle >= kMegaSpin) {
-            *af = 1;
-            att_note_timeout(p.abort_g, 5, n_done);
-            *reinterpret_cast<volatile int*>(p.abort_g) = 1;
-            atomicCAS(w.status, DEV_OK, DEV_TIMEOUT);
-            break;
-          }
-        }
-      }
+        MEGA_EV(sidx, 3);
+        ++sidx;
+      };
+      auto fatt = [&](int l) { rp.advance(n_att); };
+      mega_walk(p, fsite, fatt);
     }
-#undef MEGA_OPEN
   } else if (warp == 2) {
     // ------------------------------ activation producer ------------------------------
     if (lane == 0) {
       const uint64_t pol_a = l2_policy_evict_last();
       const uint32_t a_tx = (uint32_t)(2 * Rp) * 128u;
-      const uint32_t act0 = smem_u32(ring + (size_t)NS * p.stage_bytes);
-      const int NT = p.slots;
-      int nb = p.do_embed ? 1 : 0, sidx = 0, n = 0;   // n: units served so far (slot = n % NT)
+      RingPos rp{0, 0, NS};
+      int nb = p.do_embed ? 1 : 0, sidx = 0;
       bool alive = true;
       auto fsite = [&](int site, int l) {
         if (!alive) return;
@@ -1231,15 +1107,15 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           unsigned u = ss.g_lo;
           Seg sg;
           while (seg_next(ss, u, sg)) {
-            for (int kb = sg.a; kb < sg.b; ++kb, ++n) {
-              const int slot = n % NT;
-              if (n >= NT && !mega_wait(smem_u32(&ctl->slot_free[slot]), (uint32_t)(n / NT - 1) & 1u, ctl, p, w.status, 2, n)) {
+            for (int kb = sg.a; kb < sg.b; ++kb) {
+              if (rp.r > 0 && !mega_wait(smem_u32(&ctl->empty[rp.s]), (uint32_t)(rp.r - 1) & 1u, ctl, p, w.status, 2, rp.r)) {
                 alive = false;
                 return;
               }
-              const uint32_t bar = smem_u32(&ctl->afull[slot]);
+              const uint32_t bar = smem_u32(&ctl->full[rp.s]);
               mbar_expect_tx(bar, a_tx);
-              tma_load_2d(act0 + (uint32_t)slot * (uint32_t)p.a_bytes, tm, bar, kb * kBK, 0, pol_a);
+              tma_load_2d(stage_addr(rp.s) + kWTileBytes, tm, bar, kb * kBK, 0, pol_a);
+              rp.next();
             }
           }
           MEGA_EV(sidx, 1);
@@ -1247,7 +1123,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         ++sidx;
         nb += (site == SITE_QKV) ? 3 : 1;
       };
-      auto fatt = [&](int l) {};
+      auto fatt = [&](int l) { rp.advance(n_att); };
       mega_walk(p, fsite, fatt);
     }
   }
