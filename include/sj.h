@@ -102,6 +102,10 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *   "attn_impl"  0 = CUDA-core kernel,  1 = tensor-core (mma.sync) kernel (bf16 only; default for bf16)
  *   "step_impl"  1 = the whole step as one persistent cooperative kernel (bf16, tcgen05 GEMMs, at most 80
  *                block rows; default when the shape allows), 0 = one kernel per stage
+ *   "attn_two_term_layers"  n >= 0 (default 1): in layers [0, n) the tensor-core attention carries queries and
+ *                probabilities as a sum of two fp16 terms (twice the MMAs).  Where the residual stream is still
+ *                small (the first layer: an embedding row), the attention output is most of what the next
+ *                norm sees, and the 2^-11 rounding of one-term operands would dominate the step's error.
  *   "ring_stages" persistent kernel: cap on the shared-memory ring depth (0 = as many as fit, the default)
  *   "trace"      k > 0 = the persistent kernel records a timeline with the nanosecond global timer
  *                (sj_step_trace()): block k - 1 stamps its arrival at and release from every device-wide

@@ -208,7 +208,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_att_precise = 1;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -380,6 +380,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   ALLOC(tmp, uint8_t, act_rows * c.d_model * esz); W.A = tmp;
   ALLOC(W.Q, float, (size_t)R * qd);
   if (t->bf) ALLOC(W.Qb, __half, (size_t)R * qd);
+  if (t->bf) ALLOC(W.Qlo, __half, (size_t)R * qd);
   if (t->bf) ALLOC(W.KVn, __half, (size_t)R * 2 * kd);
   ALLOC(tmp, uint8_t, act_rows * qd * esz); W.ATT = tmp;
   ALLOC(tmp, uint8_t, act_rows * c.d_ffn * esz); W.H = tmp;
@@ -537,6 +538,11 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
   } else if (n == "ring_stages") {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
+  } else if (n == "attn_two_term_layers") {
+    if (value < 0) return fail(SJ_ERR_INVALID_ARG, "attn_two_term_layers must be >= 0");
+    cudaStreamSynchronize(t->stream);
+    clear_graphs(t);
+    t->opt_att_precise = value;
   } else if (n == "trace") {
     const size_t n_tr = kMegaTraceEntries;
     if (value && !t->d_trace) {
@@ -937,7 +943,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
                   (size_t)R * (qd + 2 * kd), l, (const T*)L.bq, (const T*)L.bk, (const T*)L.bv));
     // attention
     if (attn_tc) {
-      AttArgs aa{W.Qb, W.KVn, AttPartials{W.tc_m, W.tc_l, W.tc_o}, t->sm_count + B * dm.Hkv, l};
+      AttArgs aa{W.Qb, l < t->opt_att_precise ? W.Qlo : nullptr, W.KVn, AttPartials{W.tc_m, W.tc_l, W.tc_o}, t->sm_count + B * dm.Hkv, l};
       const size_t tc_smem = kAttStages * kAttStageBytes + sizeof(AttSmemCtl) + 1024;
       const AttPartials parts{W.tc_m, W.tc_l, W.tc_o};
       const int items = B * dm.Hkv * nq, cgrid = std::max(1, std::min(4 * t->sm_count, (items + 7) / 8));
@@ -1036,6 +1042,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.gbar = t->d_sync;
   p.abort_g = reinterpret_cast<int*>(t->d_sync + 1);
   p.n_tail_base = t->sm_count + B * dm.Hkv;
+  p.att_precise_layers = t->opt_att_precise;
   p.trace = t->opt_trace ? t->d_trace : nullptr;
   p.trace_block = t->opt_trace ? (unsigned)std::min(t->opt_trace - 1, t->sm_count - 1) : 0u;
   const int grid = t->sm_count;

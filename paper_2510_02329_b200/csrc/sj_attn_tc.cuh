@@ -59,6 +59,11 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
   __half2 t = __floats2half2_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&t);
 }
+// what packing (lo, hi) into fp16 dropped: (lo - fp16(lo), hi - fp16(hi)) as packed fp16; `packed` = pack_f16(lo, hi)
+__device__ __forceinline__ uint32_t pack_f16_rest(float lo, float hi, uint32_t packed) {
+  const float2 r = __half22float2(*reinterpret_cast<const __half2*>(&packed));
+  return pack_f16(lo - r.x, hi - r.y);
+}
 // two packed bf16 -> two packed fp16
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t x) {
   return pack_f16(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
@@ -176,7 +181,14 @@ struct AttWarp {
   // [page][half] of 2 KiB (16 slots x 64 dims, 128-byte swizzle) then, 8 KiB in, the V boxes.
   // kw0: first key of this warp's share inside the tile; key_abs0: absolute index of that key; L: keys
   // >= L are masked.
-  __device__ __forceinline__ void tile(uint32_t stage, int kw0, int key_abs0, int L, int lane) {
+  // qlo != nullptr: two-term mode.  The scores also take q_lo . k (the part of the query that its fp16 rounding
+  // dropped; qa is overwritten with those fragments and reloaded from qhi afterwards: no second fragment
+  // array has to stay in registers), and the probabilities enter the second MMA as p_hi + p_lo.
+  // (TWO is a template parameter so that the one-term code, which nearly every layer runs, is compiled exactly as
+  // it would be without the two-term mode.)
+  template <bool TWO>
+  __device__ __forceinline__ void tile(uint32_t stage, int kw0, int key_abs0, int L, int lane, const __half* qhi = nullptr,
+                                       const __half* qlo = nullptr, int row0 = 0, int nq = 0) {
     constexpr int HB = HD / 64;
     const int lr = lane & 7, mid = lane >> 3;
     // All K fragments of this warp's keys first (the ldmatrix results are not needed until the MMA chain
@@ -220,6 +232,18 @@ struct AttWarp {
         mma_16816(s[n], qa[2 * kp + 1], kf[kp][n][2], kf[kp][n][3]);
       }
     }
+    if constexpr (TWO) {
+      load_q(qlo, row0, nq, lane);
+#pragma unroll
+      for (int kp = 0; kp < HD / 32; ++kp) {
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+          mma_16816(s[n], qa[2 * kp], kf[kp][n][0], kf[kp][n][1]);
+          mma_16816(s[n], qa[2 * kp + 1], kf[kp][n][2], kf[kp][n][3]);
+        }
+      }
+      load_q(qhi, row0, nq, lane);
+    }
 #pragma unroll
     for (int n = 0; n < NT; ++n) {
       const int k = key_abs0 + n * 8 + (lane & 3) * 2;
@@ -239,6 +263,18 @@ struct AttWarp {
         mma_16816(o[2 * dp], pa, vf[kk2][dp][0], vf[kk2][dp][1]);
         mma_16816(o[2 * dp + 1], pa, vf[kk2][dp][2], vf[kk2][dp][3]);
       }
+      if constexpr (TWO) {
+        uint32_t pl[4];
+        pl[0] = pack_f16_rest(s[2 * kk2][0], s[2 * kk2][1], pa[0]);
+        pl[1] = pack_f16_rest(s[2 * kk2][2], s[2 * kk2][3], pa[1]);
+        pl[2] = pack_f16_rest(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1], pa[2]);
+        pl[3] = pack_f16_rest(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3], pa[3]);
+#pragma unroll
+        for (int dp = 0; dp < HD / 16; ++dp) {
+          mma_16816(o[2 * dp], pl, vf[kk2][dp][0], vf[kk2][dp][1]);
+          mma_16816(o[2 * dp + 1], pl, vf[kk2][dp][2], vf[kk2][dp][3]);
+        }
+      }
     }
   }
 
@@ -246,8 +282,9 @@ struct AttWarp {
   // copy written earlier in this step (the pages hold the same rows rounded to bf16 for later steps;
   // reading the copy keeps 11 significant bits of the rows that weigh most when the cache is short).
   // Query row q = g*rows + j sees kq <= j.  krow(kq) / vrow(kq) return the fp16 row pointers [HD].
-  template <typename KFn, typename VFn>
-  __device__ __forceinline__ void tail(KFn krow, VFn vrow, int rows, int row0, int nq, int lane) {
+  template <bool TWO, typename KFn, typename VFn>
+  __device__ __forceinline__ void tail(KFn krow, VFn vrow, int rows, int row0, int nq, int lane, const __half* qhi = nullptr,
+                                       const __half* qlo = nullptr) {
     const int q0 = row0 + (lane >> 2), q1 = q0 + 8;
     const int j0 = q0 % rows, j1 = q1 % rows;
     for (int kbase = 0; kbase < rows; kbase += NT * 8) {
@@ -255,17 +292,22 @@ struct AttWarp {
 #pragma unroll
       for (int n = 0; n < NT; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
 #pragma unroll
-      for (int n = 0; n < NT; ++n) {
-        const int key = kbase + n * 8 + (lane >> 2);
-        if (kbase + n * 8 < rows) {   // warp-uniform
-          const __half* kr = key < rows ? krow(key) : nullptr;
+      for (int pass = 0; pass < (TWO ? 2 : 1); ++pass) {   // two-term mode: q_hi . k, then q_lo . k (see tile())
+        if (pass == 1) load_q(qlo, row0, nq, lane);
 #pragma unroll
-          for (int k = 0; k < HD / 16; ++k) {
-            uint32_t b0 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2) : 0u;
-            uint32_t b1 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2 + 8) : 0u;
-            mma_16816(s[n], qa[k], b0, b1);
+        for (int n = 0; n < NT; ++n) {
+          const int key = kbase + n * 8 + (lane >> 2);
+          if (kbase + n * 8 < rows) {   // warp-uniform
+            const __half* kr = key < rows ? krow(key) : nullptr;
+#pragma unroll
+            for (int k = 0; k < HD / 16; ++k) {
+              uint32_t b0 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2) : 0u;
+              uint32_t b1 = kr ? ldcg_u32(kr + k * 16 + (lane & 3) * 2 + 8) : 0u;
+              mma_16816(s[n], qa[k], b0, b1);
+            }
           }
         }
+        if (pass == 1) load_q(qhi, row0, nq, lane);
       }
 #pragma unroll
       for (int n = 0; n < NT; ++n) {
@@ -284,6 +326,13 @@ struct AttWarp {
         pa[1] = pack_f16(s[2 * kk2][2], s[2 * kk2][3]);
         pa[2] = pack_f16(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1]);
         pa[3] = pack_f16(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3]);
+        uint32_t pl[4] = {0u, 0u, 0u, 0u};
+        if constexpr (TWO) {
+          pl[0] = pack_f16_rest(s[2 * kk2][0], s[2 * kk2][1], pa[0]);
+          pl[1] = pack_f16_rest(s[2 * kk2][2], s[2 * kk2][3], pa[1]);
+          pl[2] = pack_f16_rest(s[2 * kk2 + 1][0], s[2 * kk2 + 1][1], pa[2]);
+          pl[3] = pack_f16_rest(s[2 * kk2 + 1][2], s[2 * kk2 + 1][3], pa[3]);
+        }
         const int ka = kbase + kk2 * 16 + (lane & 3) * 2;   // keys ka, ka+1 (b0) and ka+8, ka+9 (b1)
         const __half* v00 = ka < rows ? vrow(ka) : nullptr;
         const __half* v01 = ka + 1 < rows ? vrow(ka + 1) : nullptr;
@@ -295,6 +344,7 @@ struct AttWarp {
           uint32_t b0 = (v00 ? ldcg_u16(v00 + d) : 0u) | ((v01 ? ldcg_u16(v01 + d) : 0u) << 16);
           uint32_t b1 = (v10 ? ldcg_u16(v10 + d) : 0u) | ((v11 ? ldcg_u16(v11 + d) : 0u) << 16);
           mma_16816(o[dn], pa, b0, b1);
+          if constexpr (TWO) mma_16816(o[dn], pl, b0, b1);
         }
       }
     }
@@ -354,6 +404,7 @@ __device__ __forceinline__ int att_find_seq(const int* pre, int B, int t) {
 
 struct AttArgs {
   const __half* Qb;        // [B][Hkv][nq][HD] scaled queries (fp16)
+  const __half* Qlo;       // same layout: the part of the queries that Qb's rounding dropped; null = one-term operands
   const __half* KVn;       // [B][Hkv][2][rows][HD] this step's own key / value rows (fp16)
   AttPartials P;
   int n_tail_base;         // slot of tail (b, h): n_tail_base + b*Hkv + h
@@ -483,11 +534,14 @@ template <int HD, int NT>
 __device__ __forceinline__ void att_tail_task(AttWarp<HD, NT>& st, const AttGeom& g, const AttArgs& a, int x, int row0, int lane) {
   const int rows = g.rows;
   st.reset();
-  st.load_q(a.Qb + (size_t)x * g.nq * HD, row0, g.nq, lane);
+  const __half* qhi = a.Qb + (size_t)x * g.nq * HD;
+  const __half* qlo = a.Qlo ? a.Qlo + (size_t)x * g.nq * HD : nullptr;
+  st.load_q(qhi, row0, g.nq, lane);
   const __half* kn = a.KVn + (size_t)x * 2 * rows * HD;
   auto krow = [&](int kq) -> const __half* { return kn + (size_t)kq * HD; };
   auto vrow = [&](int kq) -> const __half* { return kn + (size_t)(rows + kq) * HD; };
-  st.tail(krow, vrow, rows, row0, g.nq, lane);
+  if (qlo) st.template tail<true>(krow, vrow, rows, row0, g.nq, lane, qhi, qlo);   // warp-uniform
+  else st.template tail<false>(krow, vrow, rows, row0, g.nq, lane);
   st.store(a.P, (size_t)a.n_tail_base + x, 0, row0, g.nq, lane);
 }
 
@@ -515,7 +569,9 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
     const AttTile x = att_locate(pl, B, g.KPS, (int)t);
     const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
     st.reset();
-    st.load_q(a.Qb + ((size_t)x.b * Hkv + x.h) * g.nq * HD, row0, g.nq, lane);
+    const __half* qhi = a.Qb + ((size_t)x.b * Hkv + x.h) * g.nq * HD;
+    const __half* qlo = a.Qlo ? a.Qlo + ((size_t)x.b * Hkv + x.h) * g.nq * HD : nullptr;
+    st.load_q(qhi, row0, g.nq, lane);
     if (rg.ev && cw == 0 && lane == 0) { rg.ev[3] = st.qa[0][0]; rg.ev[0] = att_timer_ns(); }
     for (int i = 0; i < n; ++i, ++it) {
       const int s = it % rg.stages;
@@ -526,7 +582,11 @@ __device__ __forceinline__ bool att_consume(const AttRing& rg, int& it, const At
       if (!ok) return false;
       att_mbar_try(bar, par);   // every lane observes the completed phase
       __syncwarp();
-      st.tile(att_smem_u32(rg.base + (size_t)s * rg.stage_stride), ks * g.KW, (x.ti + i) * g.KPS + ks * g.KW, x.L, lane);
+      if (qlo)   // warp-uniform
+        st.template tile<true>(att_smem_u32(rg.base + (size_t)s * rg.stage_stride), ks * g.KW, (x.ti + i) * g.KPS + ks * g.KW, x.L,
+                               lane, qhi, qlo, row0, g.nq);
+      else
+        st.template tile<false>(att_smem_u32(rg.base + (size_t)s * rg.stage_stride), ks * g.KW, (x.ti + i) * g.KPS + ks * g.KW, x.L, lane);
       __syncwarp();
       if (lane == 0) {
         __threadfence_block();

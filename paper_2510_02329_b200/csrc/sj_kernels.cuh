@@ -17,6 +17,8 @@ struct Work {
   float* Q;          // [R, Hq*hd]    fp32 rotated queries
   __half* Qb;        // [B, Hkv, group*(gamma+1), hd] fp16 rotated queries times log2(e)/sqrt(hd), query row
                      // g*(gamma+1)+j of a KV head's group (tensor-core attention), or null
+  __half* Qlo;       // same layout: what the fp16 rounding of Qb dropped (q - Qb, rounded to fp16), for the layers in
+                     // which the attention runs with two-term operands
   __half* KVn;       // [B, Hkv, 2 (K|V), gamma+1, hd] fp16 copy of this step's own key / value rows (the rows the
                      // pages receive in bf16): the tensor-core attention reads the block's own rows from here
   void* ATT;         // attention output (input of the O projection), K = Hq*hd
@@ -188,8 +190,12 @@ __global__ void k_qkv_rope(const StepArgs* __restrict__ args, KvView kv, Work w,
         const int group = dm.Hq / dm.Hkv, j = r % rows;
         const float qs = 1.4426950408889634f / sqrtf((float)dm.hd);
         __half* qb = w.Qb + ((((size_t)b * dm.Hkv + head / group) * group + head % group) * rows + j) * dm.hd;
-        qb[i] = __float2half_rn(y1 * qs);
-        qb[i + half] = __float2half_rn(y2 * qs);
+        const __half h1 = __float2half_rn(y1 * qs), h2 = __float2half_rn(y2 * qs);
+        qb[i] = h1;
+        qb[i + half] = h2;
+        __half* ql = w.Qlo + (qb - w.Qb);
+        ql[i] = __float2half_rn(y1 * qs - __half2float(h1));
+        ql[i + half] = __float2half_rn(y2 * qs - __half2float(h2));
       }
     } else {
       T* krow = kv_row<T>(kv, layer, page, 0, head - dm.Hq, slot);

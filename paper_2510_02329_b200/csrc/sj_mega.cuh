@@ -87,6 +87,7 @@ struct MegaParams {
   unsigned* gbar;             // device-wide barrier counter   } zeroed before every launch
   int* abort_g;               // device-wide abort word        }
   int n_tail_base;
+  int att_precise_layers;     // layers [0, n) run the attention with two-term (hi + lo fp16) queries and probabilities
   // optional timeline (global-timer nanoseconds), block `trace_block`:
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
   //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
@@ -580,9 +581,16 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
         // ((((layer*n_pages + page)*2 + K|V)*Hkv + head)*page_size + slot)*HD: the per-row parts are tabulated
         if (kind == 0) {
           __half* qb = w.Qb + (size_t)head * rows * HD + dim;
+          __half* ql = w.Qlo + (size_t)head * rows * HD + dim;
+          const bool two_term = l < p.att_precise_layers;   // block-uniform
 #pragma unroll
           for (int i = 0; i < NS; ++i)
-            if (i < nr) qb[ctl->row_qoff[c0 + i]] = __float2half_rn(v[i] * qscale);
+            if (i < nr) {
+              const float qv = v[i] * qscale;
+              const __half hq = __float2half_rn(qv);
+              qb[ctl->row_qoff[c0 + i]] = hq;
+              if (two_term) ql[ctl->row_qoff[c0 + i]] = __float2half_rn(qv - __half2float(hq));
+            }
         } else {
           bf16* kvb = reinterpret_cast<bf16*>(kv.pool) +
                       ((size_t)l * kv.n_pages * 2 * dm.Hkv + (size_t)(kind - 1) * dm.Hkv + head) * kv.page_size * HD + dim;
@@ -1159,7 +1167,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
                                      ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8
                                      : nullptr;
         AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status, ev};
-        AttArgs aa{w.Qb, w.KVn, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
+        AttArgs aa{w.Qb, l < p.att_precise_layers ? w.Qlo : nullptr, w.KVn, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
         int it2 = it;
         att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
       }
