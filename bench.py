@@ -37,11 +37,11 @@ UNIT = "tokens/s"
 # ----------------------------------------------------------------------------------------------
 # helpers
 # ----------------------------------------------------------------------------------------------
-# DRAM bytes the persistent kernel moved per algorithmic byte in the ncu capture of a 4-layer cut
-# (2.8875 GB moved for 2.8626 GB of weights and cache; the ncu summary of that cut is under profiles/).
-# Traffic grows in proportion to the streamed bytes (nothing is re-read), so the full step's traffic
-# is the same ratio times its algorithmic bytes.  Set to None whenever the kernel changes until recaptured.
-MEGA_DRAM_TRAFFIC_RATIO = 1.0087
+# DRAM bytes per algorithmic byte of the persistent kernel, per workload, from the ncu capture of a cut of that
+# workload's shape (summaries under profiles/); traffic grows in proportion to the streamed bytes (nothing is
+# re-read), so a full step's traffic is this ratio times its algorithmic bytes.  A workload without a capture
+# of the kernel as it stands has no entry and reports null.
+MEGA_DRAM_TRAFFIC_RATIO = {}
 
 
 def measured_peaks():
@@ -124,7 +124,7 @@ class OracleSample:
 
     The sample is `n_layers` decoder layers, the LM head over the first vocab/`vocab_div` tokens, and
     (once, in `acceptance_seconds`) the acceptance rule on full-vocabulary logits, for at most two
-    sequences with the cache capped at 2048 tokens.  `time_step()` runs the sample once and returns
+    sequences with their full caches.  `time_step()` runs the sample once and returns
     the seconds scaled to the whole step (layers by count, head by vocabulary share, total by
     sequence count).  Weight conversion to fp64 is done at set-up, outside the timing.
     """
@@ -138,7 +138,7 @@ class OracleSample:
         cut = shape.cut(n_layers)
         gen = "cuda" if torch.cuda.is_available() else "cpu"
         dtype = torch.bfloat16
-        self.lens = [int(min(x, 2048)) for x in synth.kv_lengths(wl, seed)[:2]]
+        self.lens = [int(x) for x in synth.kv_lengths(wl, seed)[:2]]
         self.nseq = len(self.lens)
         self.osh = helpers.oracle_shape(cut)
         self.vs = shape.vocab // vocab_div
@@ -175,7 +175,7 @@ class OracleSample:
 
     def describe(self) -> str:
         return (f"{self.n_layers} of {self.wl.shape.n_layers} layers + LM head over 1/{self.vocab_div} of the vocabulary "
-                f"+ acceptance rule, {self.nseq} of {self.wl.batch} sequence(s), cache capped at 2048 tokens; scaled by "
+                f"+ acceptance rule, {self.nseq} of {self.wl.batch} sequence(s) with their full caches; extrapolated by "
                 f"layer count, vocabulary share and sequence count")
 
     def time_step(self) -> float:
@@ -192,6 +192,60 @@ class OracleSample:
         per_seq = (t_layers * self.wl.shape.n_layers / self.n_layers + t_head * self.vocab_div) / self.nseq \
             + self.acceptance_seconds
         return per_seq * self.wl.batch
+
+
+def time_whole_oracle_step(wl: synth.Workload, seed: int = 0, budget_s: float = 45.0):
+    """Seconds the CPU oracle needs for ONE whole verification step of `wl`: every layer, every sequence, the
+    full cache, the full vocabulary and the acceptance rule, calling the oracle's own functions in its own order.
+
+    One layer's weights and cache rows are drawn and widened to fp64 at a time (set-up, not timed; the whole
+    model in fp64 would not fit the host).  If the timed seconds pass `budget_s` before the last layer, the
+    remaining layers are extrapolated from those done and the result says so.
+    Returns (seconds, description, extrapolated, threads).
+    """
+    import helpers
+    from oracle import sj_oracle as orc
+    shape = wl.shape
+    gen = "cuda" if torch.cuda.is_available() else "cpu"
+    dtype = torch.bfloat16
+    lens = [int(x) for x in synth.kv_lengths(wl, seed)]
+    B = len(lens)
+    osh = helpers.oracle_shape(shape)
+    si = synth.step_inputs(shape.vocab, B, wl.gamma, seed)
+    tokens = [np.concatenate([[int(si.pending[b])], si.draft_ids[b].astype(np.int64)]) for b in range(B)]
+    top = synth.top_weights(shape, dtype, gen, seed)
+    xs = [helpers.np64(top["embed"][torch.from_numpy(t).to(top["embed"].device)]) for t in tokens]
+    timed, done = 0.0, 0
+    for l in range(shape.n_layers):
+        w64 = {k: helpers.np64(v) for k, v in synth.layer_weights(shape, l, dtype, gen, seed).items()}
+        for b in range(B):
+            ck, cv = (helpers.np64(t) for t in synth.cache_fill(shape, l, b, lens[b], dtype, gen, seed))
+            t0 = time.perf_counter()
+            xs[b], _, _ = orc.layer_forward(xs[b], w64, ck, cv, osh)
+            timed += time.perf_counter() - t0
+        done = l + 1
+        if timed > budget_s and done < shape.n_layers:
+            break
+    extrapolated = done < shape.n_layers
+    t_layers = timed * shape.n_layers / done
+    lm64, fn64, jw = helpers.np64(top["lm_head"]), helpers.np64(top["final_norm"]), helpers.np64(synth.judge_head(shape, gen, seed))
+    del top
+    t0 = time.perf_counter()
+    for b in range(B):
+        h = orc.rmsnorm(xs[b], fn64, osh.rms_eps)
+        logits = h @ lm64.T
+        orc.verdict(logits, h, si.draft_ids[b], lens[b], mode=orc.GREEDY, judge_w=jw, theta=0.5)
+    t_head = time.perf_counter() - t0
+    try:
+        import threadpoolctl
+        threads = max([p.get("num_threads", 1) for p in threadpoolctl.threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    what = (f"the whole step: {shape.n_layers} layers, {B} sequence(s) with their full caches, LM head over the full "
+            f"vocabulary, acceptance rule") if not extrapolated else \
+           (f"{done} of {shape.n_layers} layers (all {B} sequences, full caches) extrapolated by layer count, plus the "
+            f"LM head over the full vocabulary and the acceptance rule in full")
+    return t_layers + t_head, what, extrapolated, threads
 
 
 def run_reference(args, wl, rank, world):
@@ -212,7 +266,7 @@ def run_reference(args, wl, rank, world):
             "config": {"workload": wl.name, "batch": wl.batch, "gamma": wl.gamma, "kv_len": wl.kv_len,
                        "positions_per_step": R},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": sample.threads, "kind": "oracle",
-                             "sample": sample.describe()},
+                             "sample": sample.describe(), "extrapolated": True},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -372,9 +426,12 @@ def main():
             per_launch_bytes = (w_bytes + kv_bytes) / mega_launches
             per_launch_s = (v_ms / v_n) / 1e3
             roofline.update({"kernel": "k_verify_mega", "launches_per_step": mega_launches,
-                             "traffic": per_launch_bytes * MEGA_DRAM_TRAFFIC_RATIO, "traffic_unit": "bytes per launch",
+                             "traffic": (per_launch_bytes * MEGA_DRAM_TRAFFIC_RATIO[args.workload]
+                                         if args.workload in MEGA_DRAM_TRAFFIC_RATIO and not args.layers else None),
+                             "traffic_unit": "bytes per launch",
                              "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum on a 4-layer cut of the "
-                                               "same shape, scaled by algorithmic bytes",
+                                               "same shape, scaled by algorithmic bytes (null: no capture of this "
+                                               "workload's shape with the kernel as it stands)",
                              "achieved": per_launch_bytes / per_launch_s / 1e9,
                              "avg_launch_us": per_launch_s * 1e6, "algorithmic_bytes_per_launch": per_launch_bytes})
         else:
@@ -389,10 +446,10 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:
         t0 = time.perf_counter()
-        sample = OracleSample(wl, min(4, wl.shape.n_layers), vocab_div=1)
-        full = min(sample.time_step() for _ in range(2))
-        cpu_baseline = {"value": R / full, "unit": UNIT, "cores": sample.threads, "kind": "oracle",
-                        "sample": sample.describe(), "seconds_spent": time.perf_counter() - t0}
+        full, what, extrapolated, threads = time_whole_oracle_step(wl, seed=rank)
+        cpu_baseline = {"value": R / full, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what,
+                        "extrapolated": extrapolated, "oracle_seconds_per_step": full,
+                        "seconds_spent": time.perf_counter() - t0}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

@@ -225,7 +225,7 @@ struct sj_target {
   size_t tc_part_cap = 0;   // floats in tc_m / tc_l
   size_t logits_rows = 0;
   std::map<StepKey, cudaGraphExec_t> graphs;
-  std::map<int, CUtensorMap> mapA_d, mapA_q, mapA_f;  // activation maps per R
+  std::map<int, CUtensorMap> mapA_d, mapA_q, mapA_f, mapA_sel;  // activation maps per R (mapA_sel: per B)
   std::vector<void*> owned;
 };
 
@@ -384,6 +384,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   if (t->bf) ALLOC(W.KVn, __half, (size_t)R * 2 * kd);
   ALLOC(tmp, uint8_t, act_rows * qd * esz); W.ATT = tmp;
   ALLOC(tmp, uint8_t, act_rows * c.d_ffn * esz); W.H = tmp;
+  ALLOC(tmp, uint8_t, act_rows * c.d_model * esz); W.Asel = tmp;   // at most one row per sequence is used
   ALLOC(W.Hf, float, (size_t)R * c.d_model);
   ALLOC(W.rope, float2, (size_t)R * (c.head_dim / 2));
   ALLOC(W.row_pos, int, R);
@@ -478,6 +479,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     cudaMemset(W.A, 0, act_rows * c.d_model * esz);
     cudaMemset(W.ATT, 0, act_rows * qd * esz);
     cudaMemset(W.H, 0, act_rows * c.d_ffn * esz);
+    cudaMemset(W.Asel, 0, act_rows * c.d_model * esz);
     t->opt_step = 1;
   }
 #undef ALLOC
@@ -861,7 +863,8 @@ static sj_status activation_map(sj_target* t, std::map<int, CUtensorMap>& cache,
 }
 
 static cudaError_t launch_tc(sj_target* t, const TcSite& s, const CUtensorMap* mA, const CUtensorMap* w0,
-                             const CUtensorMap* w1, const CUtensorMap* w2, int R, bool pdl, bool planes) {
+                             const CUtensorMap* w1, const CUtensorMap* w2, int R, bool pdl, bool planes, int lm_mode = -1,
+                             const Work* work = nullptr) {
   RowGeom g = feed_geom(R, planes);
   TcGemmParams p;
   memset(&p, 0, sizeof(p));
@@ -873,9 +876,25 @@ static cudaError_t launch_tc(sj_target* t, const TcSite& s, const CUtensorMap* m
   p.stages = g.stages; p.a_stage_bytes = g.a_stage_bytes; p.tmem_cols = g.tmem_cols;
   p.acc_bufs = g.acc_bufs; p.acc_stride = g.acc_stride;
   p.P = t->work.P; p.slot_stride = (size_t)R * s.N; p.tile_slots = s.d_tile_slots;
-  p.lm_mode = s.lm ? 1 : 0; p.status = t->work.status;
+  p.lm_mode = lm_mode >= 0 ? lm_mode : (s.lm ? 1 : 0); p.status = t->work.status;
   return launch(k_gemm_tc, dim3(s.G), dim3(kTcThreads), g.smem_bytes, t->stream, pdl, *mA, *w0, *(w1 ? w1 : w0),
-                *(w2 ? w2 : w0), p, (const StepArgs*)t->d_args, t->work, t->dm.V);
+                *(w2 ? w2 : w0), p, (const StepArgs*)t->d_args, work ? *work : t->work, t->dm.V);
+}
+
+// a14 in sampling mode with the tensor-core LM head: re-normalise the one row per sequence that the emitted
+// token is drawn from, run the LM head over those B rows into the [B, V] logit scratch, draw the token.
+template <typename T>
+static sj_status enqueue_resample(sj_target* t, sj_kv* kv, int B, const Work& W, bool pdl) {
+  const Dims& dm = t->dm;
+  cudaStream_t s = t->stream;
+  const CUtensorMap* mA = nullptr;
+  sj_status st = activation_map(t, t->mapA_sel, W.Asel, B, dm.d, &mA);
+  if (st != SJ_OK) return st;
+  CU_TRY(launch(k_select_rows<T>, dim3(B), dim3(256), sizeof(float) * dm.d, s, pdl, (const StepArgs*)t->d_args, W, dm,
+                (const T*)t->final_norm));
+  CU_TRY(launch_tc(t, t->s_lm, mA, &t->m_lm, nullptr, nullptr, B, pdl, true, 2, &W));
+  CU_TRY(launch(k_resample, dim3(B), dim3(1024), 0, s, pdl, (const StepArgs*)t->d_args, kv->view, W, dm, 1));
+  return SJ_OK;
 }
 
 template <typename T>
@@ -998,7 +1017,14 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
     TIMED("lm_stats", launch(k_lm_stats_from_logits, dim3(n_vtiles, (R + 7) / 8), dim3(256), 0, s, pdl, args, W, dm, R));
   }
   TIMED("finalize", launch(k_finalize, dim3(B), dim3(256), 0, s, pdl, args, kv->view, W, dm, n_vtiles, R));
-  if (mode == SJ_MODE_SAMPLING) TIMED("resample", launch(k_resample, dim3(B), dim3(1024), 0, s, pdl, args, kv->view, W, dm));
+  if (mode == SJ_MODE_SAMPLING) {
+    if (tc) {
+      sj_status st = enqueue_resample<T>(t, kv, B, t->work, pdl);   // t->work: with the [B, V] logit scratch
+      if (st != SJ_OK) return st;
+    } else {
+      TIMED("resample", launch(k_resample, dim3(B), dim3(1024), 0, s, pdl, args, kv->view, W, dm, 0));
+    }
+  }
   return SJ_OK;
 }
 
@@ -1084,8 +1110,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
       t->timed.push_back({"verify_step", ea, eb});
     }
   }
-  if (mode == SJ_MODE_SAMPLING)
-    CU_TRY(launch(k_resample, dim3(B), dim3(1024), 0, s, false, (const StepArgs*)t->d_args, kv->view, W, dm));
+  if (mode == SJ_MODE_SAMPLING) return enqueue_resample<bf16>(t, kv, B, t->work, false);
   return SJ_OK;
 }
 
@@ -1173,7 +1198,10 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
   for (int i = 0; i < B; ++i) chunk_need_base += (size_t)(kv->len_hi[a->seq_ids[i]] + rows + chunk_len - 1) / chunk_len;
 
   const bool use_mega = mega_usable(t, kv, B, gamma);
-  const bool use_scratch = a->mode == SJ_MODE_SAMPLING || (t->opt_gemm == 0 && !use_mega);
+  // [R, V] logits exist only for the CUDA-core LM head (fp32 models, cross-checks); the tensor-core paths keep
+  // softmax statistics per vocabulary tile and, in sampling mode, the logits of one row per sequence ([B, V])
+  const bool use_scratch = t->opt_gemm == 0 && !use_mega;
+  const size_t logit_rows_needed = use_scratch ? (size_t)R : (a->mode == SJ_MODE_SAMPLING ? (size_t)B : 0);
   // grow lazily-sized buffers (outside any capture)
   if (chunk_need_base > t->att_chunks_cap || rows > t->att_rows_cap) {
     CU_TRY(cudaStreamSynchronize(t->stream));
@@ -1218,7 +1246,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
       t->tc_part_cap = need;
     }
   }
-  if (use_scratch && (size_t)R > t->logits_rows) {
+  if (logit_rows_needed > t->logits_rows) {
     CU_TRY(cudaStreamSynchronize(t->stream));
     clear_graphs(t);
     if (t->work.logits) {
@@ -1226,8 +1254,8 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
       t->owned.erase(std::remove(t->owned.begin(), t->owned.end(), (void*)t->work.logits), t->owned.end());
       t->work.logits = nullptr;
     }
-    if ((st = dev_alloc(t, &t->work.logits, (size_t)R * t->dm.V)) != SJ_OK) return st;
-    t->logits_rows = R;
+    if ((st = dev_alloc(t, &t->work.logits, logit_rows_needed * t->dm.V)) != SJ_OK) return st;
+    t->logits_rows = logit_rows_needed;
   }
 
   // per-call arguments: one small copy (the driver stages pageable memory before returning)

@@ -49,7 +49,8 @@ struct TcGemmParams {
   float* P;             // partial buffer (split mode)
   size_t slot_stride;
   const int2* tile_slots;
-  int lm_mode;          // 1: fused LM-head epilogue, split at whole tiles
+  int lm_mode;          // 1: fused LM-head epilogue, split at whole tiles; 2: same split, raw logits stored to w.logits
+                        // [R, V] and nothing else (the second pass over one row per sequence in sampling mode)
   int* status;
 };
 
@@ -323,7 +324,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     pdl_wait();
     const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
     const int et = threadIdx.x - 64;
-    if (p.lm_mode) {
+    if (p.lm_mode == 1) {
       const int rows = args->gamma + 1;
       for (int r = et; r < p.R; r += 128) {
         int b = r / rows, j = r % rows;
@@ -369,6 +370,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             tc_ld16(taddr + p.lo_off + c0, lo);
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] += lo[i];
+          }
+          if (p.lm_mode == 2) {
+            if (n < V) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                if (c0 + i < p.R) w.logits[(size_t)(c0 + i) * V + n] = v[i];
+            }
+            continue;
           }
 #pragma unroll
           for (int i = 0; i < 16; ++i) {

@@ -37,7 +37,9 @@ struct Work {
   RowStat* stats;    // [vocab tiles, R]
   float* tgt_logit;  // [R]   logit of the drafted token d_{j+1} in row j
   RowStat* rowstat;  // [R]   merged statistics
-  float* logits;     // [R, V] fp32 scratch (sampling mode / debugging / CUDA-core LM head), or null
+  float* logits;     // fp32 logit scratch, or null: [R, V] for the CUDA-core LM head; [B, V] in sampling mode with
+                     // the tensor-core LM head (only the one row per sequence that the emitted token is drawn from)
+  void* Asel;        // GEMM input planes of those B rows (final-norm hidden states), K = d
   const double* inv_freq;  // [hd/2] rope_theta^(-2i/hd)
   const float* judge_w;    // [d]
   int* status;
@@ -578,9 +580,26 @@ __global__ void k_finalize(const StepArgs* __restrict__ args, KvView kv, Work w,
   }
 }
 
+// a14, sampling mode, first half: the row the emitted token is drawn from (row n_b of sequence b, known only
+// after the first-rejection scan) is normalised again into a compact set of GEMM input planes, one row per
+// sequence; a second LM-head pass over those B rows then yields the only logits the step ever stores.
+template <typename T>
+__global__ void k_select_rows(const StepArgs* __restrict__ args, Work w, Dims dm, const T* __restrict__ gain) {
+  extern __shared__ float xs[];
+  __shared__ float red[32];
+  pdl_wait();
+  pdl_launch();
+  const int b = blockIdx.x, rows = args->gamma + 1;
+  const int r = b * rows + min(max(args->accepted_len[b], 0), rows - 1);
+  for (int i = threadIdx.x; i < dm.d; i += blockDim.x) xs[i] = w.X[(size_t)r * dm.d + i];
+  __syncthreads();
+  norm_row_from_smem<T>(xs, dm.d, gain, dm.eps, w.Asel, gridDim.x, b, nullptr, nullptr, red);
+}
+
 // a14, sampling mode: inverse CDF over the vocabulary of norm(max(0, p_n - q_{n+1})) (first
 // rejection) or of p_gamma (everything accepted), driven by uniforms[:, gamma].  fp64 prefix sums.
-__global__ void k_resample(const StepArgs* __restrict__ args, KvView kv, Work w, Dims dm) {
+// per_seq: the logit scratch holds one row per sequence (row b) instead of every block row.
+__global__ void k_resample(const StepArgs* __restrict__ args, KvView kv, Work w, Dims dm, int per_seq) {
   pdl_wait();
   pdl_launch();
   __shared__ double part[1024];
@@ -591,7 +610,7 @@ __global__ void k_resample(const StepArgs* __restrict__ args, KvView kv, Work w,
   const int r = b * rows + n;
   const RowStat st = w.rowstat[r];
   const float invT = args->inv_temperature;
-  const float* lg = w.logits + (size_t)r * dm.V;
+  const float* lg = w.logits + (size_t)(per_seq ? b : r) * dm.V;
   const float* q = (n < gamma) ? args->q_full + ((size_t)b * gamma + n) * dm.V : nullptr;
   const int per = (dm.V + T - 1) / T, v0 = tid * per, v1 = min(v0 + per, dm.V);
   const double inv_s = 1.0 / (double)st.s;
