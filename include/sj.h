@@ -173,6 +173,12 @@ typedef struct {
   int use_align, use_judge;  /* which of the two tests may accept (App. D.2 ablation) */
   float theta_override;      /* >= 0: use instead of the loaded theta */
   int commit;                /* 1: kv_len <- kv_len + 1 + accepted_len, pending <- next_token */
+  const float *theta_per_seq;/* host [B] or NULL: a judge threshold per sequence (takes precedence; each in [0, 1e30]) */
+  int top_k;                 /* GREEDY alignment test: 0 or 1 = the draft must be the target's arg max (strict matching);
+                                2 = it must be among the target's two most likely tokens (the top-k baseline of the
+                                paper's Sec. 4, k = 2).  Equal logits rank by token id, lowest first */
+  int accept_all;            /* 1: accept every drafted position whatever the tests say: the block is a forced
+                                continuation (prefill of known tokens, teacher-forced scoring, Eq. 2 alone) */
 } sj_verify_args;
 
 typedef struct {
@@ -185,12 +191,37 @@ typedef struct {
   int *new_kv_len;      /* device [B]         kv_len + 1 + n */
   float *dbg_hidden;    /* device [B, gamma+1, d_model] or NULL: hidden states after the final norm */
   float *dbg_logits;    /* device [B, gamma+1, vocab]   or NULL: raw logits (tests only) */
+  float *logp_draft;    /* device [B, gamma] or NULL: log p_j(d_j) (natural log; the teacher-forced log-likelihood
+                                              terms of the semantic-preservation score, Eq. 6-7) */
 } sj_verify_out;
 
 /* One verification step (see the file comment).  Appends gamma+1 K/V rows per sequence at
  * [kv_len, kv_len+gamma]; with commit the sequence keeps the first 1+n of them.
  * Errors before launch: INVALID_ARG, SHAPE (B*(gamma+1) > max_rows), OOM (page pool), STATE. */
 sj_status sj_verify(sj_target *t, sj_kv *kv, const sj_verify_args *args, const sj_verify_out *out);
+
+/* Chunked prefill through the verification step's own kernels: Eq. 2 applied to tokens that are known
+ * rather than drafted.  Appends the n_tokens tokens `tokens` (host) to sequence `seq` in blocks of up to
+ * min(32, 96 / (Hq/Hkv), max_rows) tokens: each block runs as a verification step whose first row is the
+ * block's first token and whose "drafts" are the following ones, every position accepted and committed
+ * (accept_all), so the cache receives exactly the K/V rows a verification step would read.  On return (the
+ * work is queued on the target's stream) the sequence is n_tokens longer and its pending token is the target's
+ * greedy token after the last appended one; with next_token != NULL (host) that token is also copied out,
+ * which waits for the stream.  The sequence's previous pending token is dropped: the first appended token
+ * takes its place.  Errors: INVALID_ARG, SHAPE, OOM (page pool), and whatever sj_verify() reports. */
+sj_status sj_prefill(sj_target *t, sj_kv *kv, int seq, const int *tokens, int n_tokens, int *next_token);
+
+/* Semantic-preservation score of a token replacement (Sec. 3.3, Eq. 6 in the autoregressive form of Eq. 7):
+ *   s = [log P(z_i | y_<i) - log P(y_i | y_<i)]
+ *       + sum_{k=1..N} [log P(y_{i+k} | y_<i, z_i, y_{i+1..i+k-1}) - log P(y_{i+k} | y_<i, y_i, y_{i+1..i+k-1})]
+ * the quantity whose threshold labels the verifier's training tokens.  Sequence `seq` must hold y_{<i-1} in the
+ * cache and y_{i-1} as its pending token; `future` (host) are the N = n_future <= 30 tokens y_{i+1..i+N}.  Two
+ * uncommitted verification steps over [y_{i-1}; z_i or y_i, future...] give the teacher-forced log-probabilities
+ * (sj_verify_out.logp_draft); the cache, the length and the pending token are left as they were.
+ * score (host, two floats): s and its prefix term log P(z_i | y_<i) - log P(y_i | y_<i).  Waits for the stream.
+ * Errors: INVALID_ARG, SHAPE, and whatever sj_verify() reports. */
+sj_status sj_semantic_score(sj_target *t, sj_kv *kv, int seq, int y_i, int z_i, const int *future, int n_future,
+                            float *score);
 
 /* Truncate sequences to new_len <= current length (host arrays [B]) and return the whole pages
  * past new_len to the pool (the KV-length rollback that follows the first-rejection scan, Sec. 3.1).

@@ -309,3 +309,38 @@ def verify(shape: Shape, top, layer_provider, pending: Sequence[int], draft_ids:
             uniforms=None if uniforms is None else uniforms[b],
             judge_w=judge_w, judge_b=judge_b, theta=theta, use_align=use_align, use_judge=use_judge))
     return out, fwd
+
+
+# --------------------------------------------------------------------------------------
+# semantic-preservation score (labels for the verifier's training data)
+# --------------------------------------------------------------------------------------
+
+
+def log_softmax_rows(z: np.ndarray) -> np.ndarray:
+    z = np.asarray(z, F64)
+    z = z - z.max(axis=-1, keepdims=True)
+    return z - np.log(np.exp(z).sum(axis=-1, keepdims=True))
+
+
+def teacher_forced_logp(shape: Shape, top, layer_provider, cache, prev_token: int, tokens: Sequence[int]) -> np.ndarray:
+    """log P(tokens[k] | cache, prev_token, tokens[:k]) for every k: one block [prev_token, tokens...] fed to the
+    target (Eq. 2), row k's distribution read at tokens[k]."""
+    block = np.concatenate([[int(prev_token)], np.asarray(tokens, np.int64)])
+    bf = forward_blocks(shape, top, layer_provider, [block], [cache])[0]
+    lp = log_softmax_rows(bf.logits)
+    return np.array([lp[k, int(tokens[k])] for k in range(len(tokens))])
+
+
+def semantic_preservation_score(shape: Shape, top, layer_provider, cache, prev_token: int, y_i: int, z_i: int,
+                                future: Sequence[int]) -> Tuple[float, float]:
+    """s(y, z_i) of Sec. 3.3 with N = len(future) future tokens (Eq. 6, in the autoregressive form of Eq. 7):
+
+        s = [log P(z_i | y_<i) - log P(y_i | y_<i)]
+            + sum_k [log P(y_{i+k} | y_<i, z_i, y_{i+1..i+k-1}) - log P(y_{i+k} | y_<i, y_i, y_{i+1..i+k-1})]
+
+    cache holds y_{<i-1}, prev_token is y_{i-1} (the row that predicts position i), future = y_{i+1..i+N}.
+    The replaced-token probabilities come from feeding the token-substituted response to the target.
+    Returns (s, s_prefix)."""
+    lp_z = teacher_forced_logp(shape, top, layer_provider, cache, prev_token, [int(z_i)] + [int(t) for t in future])
+    lp_y = teacher_forced_logp(shape, top, layer_provider, cache, prev_token, [int(y_i)] + [int(t) for t in future])
+    return float(np.sum(lp_z - lp_y)), float(lp_z[0] - lp_y[0])

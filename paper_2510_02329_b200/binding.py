@@ -24,7 +24,7 @@ MODE_GREEDY, MODE_SAMPLING = 0, 1
 EXPORTS = ["sj_create_target", "sj_destroy_target", "sj_load_judge_head", "sj_set_option", "sj_sync",
            "sj_kv_create", "sj_kv_destroy", "sj_kv_fill", "sj_kv_read", "sj_kv_set_len", "sj_kv_set_pending",
            "sj_kv_len", "sj_verify", "sj_rollback_kv", "sj_gemm_skinny", "sj_gemm_skinny_noalloc", "sj_last_error",
-           "sj_kernel_time", "sj_step_trace", "sj_device_memory_calls", "sj_debug_expire_wait"]
+           "sj_kernel_time", "sj_step_trace", "sj_device_memory_calls", "sj_debug_expire_wait", "sj_prefill", "sj_semantic_score"]
 
 
 class SjError(RuntimeError):
@@ -52,12 +52,13 @@ class VerifyArgs(C.Structure):
     _fields_ = [("B", C.c_int), ("gamma", C.c_int), ("seq_ids", C.POINTER(C.c_int)), ("draft_ids", C.c_void_p),
                 ("draft_q_tok", C.c_void_p), ("draft_q_full", C.c_void_p), ("uniforms", C.c_void_p),
                 ("mode", C.c_int), ("temperature", C.c_float), ("use_align", C.c_int), ("use_judge", C.c_int),
-                ("theta_override", C.c_float), ("commit", C.c_int)]
+                ("theta_override", C.c_float), ("commit", C.c_int), ("theta_per_seq", C.POINTER(C.c_float)),
+                ("top_k", C.c_int), ("accept_all", C.c_int)]
 
 
 class VerifyOut(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("accepted_len", "next_token", "judge_scores", "p_draft", "new_kv_len",
-                                          "dbg_hidden", "dbg_logits")]
+                                          "dbg_hidden", "dbg_logits", "logp_draft")]
 
 
 _lib = None
@@ -81,6 +82,9 @@ def load(build_if_needed: bool = True) -> C.CDLL:
         if name != "sj_last_error":
             getattr(lib, name).restype = C.c_int
     lib.sj_debug_expire_wait.argtypes = [C.c_void_p, C.c_int, C.c_uint]
+    lib.sj_semantic_score.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int), C.c_int,
+                                      C.POINTER(C.c_float)]
+    lib.sj_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_int), C.c_int, C.POINTER(C.c_int)]
     lib.sj_device_memory_calls.restype = C.c_long
     lib.sj_device_memory_calls.argtypes = []
     lib.sj_create_target.argtypes = [C.POINTER(ModelConfig), C.POINTER(Weights), C.c_void_p, C.POINTER(C.c_void_p)]
@@ -224,6 +228,22 @@ class KVCache:
         check(self._lib.sj_kv_len(self.handle, _iarr(seq_ids), out, len(seq_ids)))
         return list(out)
 
+    def prefill(self, seq: int, tokens, want_next: bool = True) -> Optional[int]:
+        """``sj_prefill``: append known tokens to a sequence through the verification kernels; returns the
+        target's greedy token after the last one (or None without ``want_next``)."""
+        nxt = C.c_int(-1)
+        check(self._lib.sj_prefill(self.target.handle, self.handle, int(seq), _iarr(tokens), len(tokens),
+                                   C.byref(nxt) if want_next else None))
+        return int(nxt.value) if want_next else None
+
+    def semantic_score(self, seq: int, y_i: int, z_i: int, future):
+        """``sj_semantic_score``: (s, s_prefix) of replacing y_i by z_i given the sequence's cache, its pending
+        token y_{i-1} and the future tokens."""
+        out = (C.c_float * 2)()
+        check(self._lib.sj_semantic_score(self.target.handle, self.handle, int(seq), int(y_i), int(z_i), _iarr(future),
+                                          len(future), out))
+        return float(out[0]), float(out[1])
+
     def rollback(self, seq_ids, new_len) -> None:
         check(self._lib.sj_rollback_kv(self.handle, _iarr(seq_ids), _iarr(new_len), len(seq_ids)))
 
@@ -251,22 +271,26 @@ class VerifyBuffers:
         self.new_kv_len = torch.zeros(B, dtype=torch.int32, device=dev)
         self.dbg_hidden = torch.zeros(B, gamma + 1, d_model, dtype=torch.float32, device=dev) if debug else None
         self.dbg_logits = torch.zeros(B, gamma + 1, vocab, dtype=torch.float32, device=dev) if debug else None
+        self.logp_draft = torch.zeros(B, gamma, dtype=torch.float32, device=dev)
 
     def struct(self) -> VerifyOut:
         return VerifyOut(_ptr(self.accepted_len), _ptr(self.next_token), _ptr(self.judge_scores), _ptr(self.p_draft),
-                         _ptr(self.new_kv_len), _ptr(self.dbg_hidden), _ptr(self.dbg_logits))
+                         _ptr(self.new_kv_len), _ptr(self.dbg_hidden), _ptr(self.dbg_logits), _ptr(self.logp_draft))
 
 
 def verify(target: Target, kv: KVCache, seq_ids: Sequence[int], draft_ids: torch.Tensor, out: VerifyBuffers, *,
            mode: int = MODE_GREEDY, temperature: float = 1.0, draft_q_tok: Optional[torch.Tensor] = None,
            draft_q_full: Optional[torch.Tensor] = None, uniforms: Optional[torch.Tensor] = None,
-           use_align: bool = True, use_judge: bool = True, theta: float = -1.0, commit: bool = True) -> None:
+           use_align: bool = True, use_judge: bool = True, theta: float = -1.0, commit: bool = True,
+           theta_per_seq: Optional[Sequence[float]] = None, top_k: int = 0, accept_all: bool = False) -> None:
     """``sj_verify``: asynchronous on the target's stream; results land in ``out``."""
     B, gamma = draft_ids.shape
     assert draft_ids.dtype == torch.int32
     ids = _iarr(seq_ids)
     args = VerifyArgs(B, gamma, ids, _ptr(draft_ids), _ptr(draft_q_tok), _ptr(draft_q_full), _ptr(uniforms), mode,
-                      temperature, int(use_align), int(use_judge), theta, int(commit))
+                      temperature, int(use_align), int(use_judge), theta, int(commit),
+                      (C.c_float * B)(*[float(x) for x in theta_per_seq]) if theta_per_seq is not None else None,
+                      int(top_k), int(accept_all))
     o = out.struct()
     target.stream.wait_stream(torch.cuda.current_stream())   # inputs were produced on the caller's stream
     check(target._lib.sj_verify(target.handle, kv.handle, C.byref(args), C.byref(o)))

@@ -205,6 +205,7 @@ struct sj_target {
   Work work;
   StepArgs* d_args = nullptr;
   float* d_judge_w = nullptr;
+  int* d_prefill = nullptr;        // device scratch of sj_prefill(): one block's token ids and outputs
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
@@ -1175,6 +1176,11 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
     return fail(SJ_ERR_INVALID_ARG, "null output pointer");
   if (a->theta_override == a->theta_override && a->theta_override > 1e30f) return fail(SJ_ERR_INVALID_ARG, "bad theta");
   if (a->theta_override != a->theta_override) return fail(SJ_ERR_INVALID_ARG, "theta is NaN");
+  if (a->theta_per_seq)
+    for (int i = 0; i < a->B; ++i)
+      if (!(a->theta_per_seq[i] >= 0.f && a->theta_per_seq[i] <= 1e30f)) return fail(SJ_ERR_INVALID_ARG, "theta_per_seq[%d] is not in [0, 1e30]", i);
+  if (a->top_k < 0 || a->top_k > 2) return fail(SJ_ERR_UNSUPPORTED, "top_k must be 0, 1 or 2");
+  if (a->top_k == 2 && a->mode != SJ_MODE_GREEDY) return fail(SJ_ERR_UNSUPPORTED, "top_k = 2 is a greedy-mode test");
   const int group = t->dm.Hq / t->dm.Hkv;
   if (group * rows > kAttMaxQ) return fail(SJ_ERR_SHAPE, "(Hq/Hkv)*(gamma+1) = %d exceeds %d", group * rows, kAttMaxQ);
 
@@ -1267,7 +1273,11 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
   h.B = B; h.gamma = gamma; h.mode = a->mode; h.use_align = a->use_align ? 1 : 0; h.use_judge = a->use_judge ? 1 : 0;
   h.commit = a->commit ? 1 : 0;
   h.inv_temperature = a->mode == SJ_MODE_SAMPLING ? 1.0f / a->temperature : 1.0f;
-  h.theta = a->theta_override >= 0.f ? a->theta_override : t->theta;
+  for (int i = 0; i < B; ++i)
+    h.theta[i] = a->theta_per_seq ? a->theta_per_seq[i] : (a->theta_override >= 0.f ? a->theta_override : t->theta);
+  h.top_k = a->top_k >= 2 ? 2 : 1;
+  h.accept_all = a->accept_all ? 1 : 0;
+  h.logp_draft = o->logp_draft;
   h.judge_bias = t->judge_bias;
   h.has_judge = t->has_judge ? 1 : 0;
   memcpy(h.seq_ids, a->seq_ids, sizeof(int) * B);
@@ -1312,6 +1322,133 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
       kv->len_hi[s] += rows;
       kv->exact[s] = 0;
     }
+  }
+  return SJ_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// chunked prefill and teacher-forced scoring: the verification step applied to known tokens
+// ---------------------------------------------------------------------------------------------
+// device scratch of one such block, in ints: [0,32) token ids, [32,64) accepted_len / next_token / new_kv_len,
+// [64,96) judge scores, [96,128) p_draft, [128,160) and [160,192) log-probabilities of two blocks, [192,194) a score
+constexpr int kBlockScratchInts = 8 * (SJ_MAX_GAMMA + 1);
+
+// s = sum_k (lp_z[k] - lp_y[k]) in index order (fp64), s_prefix = lp_z[0] - lp_y[0]
+__global__ void k_score_diff(const float* __restrict__ lp_z, const float* __restrict__ lp_y, int n, float* __restrict__ out) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    double s = 0.0;
+    for (int k = 0; k < n; ++k) s += (double)lp_z[k] - (double)lp_y[k];
+    out[0] = (float)s;
+    out[1] = lp_z[0] - lp_y[0];
+  }
+}
+
+extern "C" sj_status sj_semantic_score(sj_target* t, sj_kv* kv, int seq, int y_i, int z_i, const int* future, int n_future,
+                                       float* score) {
+  if (!t || !kv || !score || (n_future > 0 && !future)) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (kv->t != t) return fail(SJ_ERR_INVALID_ARG, "KV cache belongs to another target");
+  if (seq < 0 || seq >= kv->max_seqs) return fail(SJ_ERR_INVALID_ARG, "sequence id %d out of range", seq);
+  if (n_future < 0 || n_future + 1 > SJ_MAX_GAMMA) return fail(SJ_ERR_SHAPE, "n_future must be in [0, %d]", SJ_MAX_GAMMA - 1);
+  for (int k = -2; k < n_future; ++k) {
+    const int tok = k == -2 ? y_i : (k == -1 ? z_i : future[k]);
+    if (tok < 0 || tok >= t->dm.V) return fail(SJ_ERR_INVALID_ARG, "token id out of range");
+  }
+  if (!t->d_prefill) {
+    sj_status st = dev_alloc(t, &t->d_prefill, (size_t)kBlockScratchInts);
+    if (st != SJ_OK) return st;
+  }
+  const int W = SJ_MAX_GAMMA + 1, gamma = n_future + 1;
+  sj_verify_out o;
+  memset(&o, 0, sizeof(o));
+  o.accepted_len = t->d_prefill + W;
+  o.next_token = o.accepted_len + 1;
+  o.new_kv_len = o.accepted_len + 2;
+  o.judge_scores = reinterpret_cast<float*>(t->d_prefill + 2 * W);
+  o.p_draft = reinterpret_cast<float*>(t->d_prefill + 3 * W);
+  float* lp[2] = {reinterpret_cast<float*>(t->d_prefill + 4 * W), reinterpret_cast<float*>(t->d_prefill + 5 * W)};
+  float* d_score = reinterpret_cast<float*>(t->d_prefill + 6 * W);
+  int block[SJ_MAX_GAMMA + 1];
+  for (int k = 0; k < n_future; ++k) block[1 + k] = future[k];
+  for (int pass = 0; pass < 2; ++pass) {   // the token-substituted response, then the original one
+    block[0] = pass == 0 ? z_i : y_i;
+    CU_TRY(cudaMemcpyAsync(t->d_prefill, block, sizeof(int) * gamma, cudaMemcpyHostToDevice, t->stream));
+    sj_verify_args a;
+    memset(&a, 0, sizeof(a));
+    a.B = 1;
+    a.gamma = gamma;
+    a.seq_ids = &seq;
+    a.draft_ids = t->d_prefill;
+    a.mode = SJ_MODE_GREEDY;
+    a.temperature = 1.f;
+    a.theta_override = -1.f;
+    a.accept_all = 1;
+    a.commit = 0;          // the cache and the pending token stay as they are
+    o.logp_draft = lp[pass];
+    sj_status st = sj_verify(t, kv, &a, &o);
+    if (st != SJ_OK) return st;
+  }
+  CU_TRY(launch(k_score_diff, dim3(1), dim3(32), 0, t->stream, false, (const float*)lp[0], (const float*)lp[1], gamma, d_score));
+  CU_TRY(cudaMemcpyAsync(score, d_score, 2 * sizeof(float), cudaMemcpyDeviceToHost, t->stream));
+  CU_TRY(cudaStreamSynchronize(t->stream));
+  return SJ_OK;
+}
+
+extern "C" sj_status sj_prefill(sj_target* t, sj_kv* kv, int seq, const int* tokens, int n_tokens, int* next_token) {
+  if (!t || !kv || !tokens) return fail(SJ_ERR_INVALID_ARG, "null argument");
+  if (kv->t != t) return fail(SJ_ERR_INVALID_ARG, "KV cache belongs to another target");
+  if (seq < 0 || seq >= kv->max_seqs) return fail(SJ_ERR_INVALID_ARG, "sequence id %d out of range", seq);
+  if (n_tokens <= 0) return fail(SJ_ERR_INVALID_ARG, "n_tokens must be positive");
+  for (int i = 0; i < n_tokens; ++i)
+    if (tokens[i] < 0 || tokens[i] >= t->dm.V) return fail(SJ_ERR_INVALID_ARG, "token id out of range");
+  const int group = t->dm.Hq / t->dm.Hkv;
+  const int c_max = std::min({SJ_MAX_GAMMA + 1, kAttMaxQ / group, t->max_rows});
+  if (c_max < 2) return fail(SJ_ERR_SHAPE, "max_rows = %d is too small for a prefill block", t->max_rows);
+  if (!t->d_prefill) {   // draft ids and the step's outputs of one block
+    sj_status st = dev_alloc(t, &t->d_prefill, (size_t)kBlockScratchInts);
+    if (st != SJ_OK) return st;
+  }
+  int* d_draft = t->d_prefill;
+  sj_verify_out o;
+  memset(&o, 0, sizeof(o));
+  o.accepted_len = t->d_prefill + (SJ_MAX_GAMMA + 1);
+  o.next_token = o.accepted_len + 1;
+  o.new_kv_len = o.accepted_len + 2;
+  o.judge_scores = reinterpret_cast<float*>(t->d_prefill + 2 * (SJ_MAX_GAMMA + 1));
+  o.p_draft = reinterpret_cast<float*>(t->d_prefill + 3 * (SJ_MAX_GAMMA + 1));
+  for (int i = 0; i < n_tokens;) {
+    const int c = std::min(c_max, n_tokens - i);
+    sj_status st = sj_kv_set_pending(kv, &seq, tokens + i, 1);
+    if (st != SJ_OK) return st;
+    sj_verify_args a;
+    memset(&a, 0, sizeof(a));
+    a.B = 1;
+    a.seq_ids = &seq;
+    a.draft_ids = d_draft;
+    a.mode = SJ_MODE_GREEDY;
+    a.temperature = 1.f;
+    a.theta_override = -1.f;
+    a.commit = 1;
+    const int before = kv->len_hi[seq];
+    if (c >= 2) {
+      // block [x_i, x_{i+1} .. x_{i+c-1}]: the c - 1 known continuations are the "drafts", all accepted
+      a.gamma = c - 1;
+      a.accept_all = 1;
+      CU_TRY(cudaMemcpyAsync(d_draft, tokens + i + 1, sizeof(int) * (c - 1), cudaMemcpyHostToDevice, t->stream));
+    } else {
+      // a lone last token: a block of two rows whose second row (a dummy draft) is rejected outright
+      a.gamma = 1;
+      a.use_align = 0;
+      a.use_judge = 0;
+      CU_TRY(cudaMemsetAsync(d_draft, 0, sizeof(int), t->stream));
+    }
+    if ((st = sj_verify(t, kv, &a, &o)) != SJ_OK) return st;
+    kv->len_hi[seq] = before + c;   // the host knows exactly how many rows such a block keeps
+    kv->exact[seq] = 1;
+    i += c;
+  }
+  if (next_token) {
+    CU_TRY(cudaMemcpyAsync(next_token, o.next_token, sizeof(int), cudaMemcpyDeviceToHost, t->stream));
+    CU_TRY(cudaStreamSynchronize(t->stream));
   }
   return SJ_OK;
 }

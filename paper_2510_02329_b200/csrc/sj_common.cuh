@@ -38,10 +38,14 @@ struct StepArgs {
   int* new_kv_len;
   float* dbg_hidden;
   float* dbg_logits;
+  float* logp_draft;      // optional: natural log of p_j(d_j)
   int B, gamma, mode, use_align, use_judge, commit;
-  float inv_temperature, theta, judge_bias;
+  int top_k;              // greedy alignment test: the draft must be among the target's top_k tokens (1 or 2)
+  int accept_all;         // every drafted position is accepted whatever the tests say (prefill, teacher forcing)
+  float inv_temperature, judge_bias;
   int has_judge;
   int seq_ids[kMaxBatch];
+  float theta[kMaxBatch]; // judge threshold per sequence of the batch
 };
 
 // Paged KV cache view.  Element (layer, page, kv in {0,1}, head, slot, dim):

@@ -556,13 +556,15 @@ __global__ void k_finalize(const StepArgs* __restrict__ args, KvView kv, Work w,
       const int j = lane + 1;  // drafted position
       const int d = args->draft_ids[b * gamma + lane];
       const RowStat st = rs[j - 1];
-      const float p = expf(w.tgt_logit[b * rows + j - 1] - st.m) / st.s;
+      const float zd = w.tgt_logit[b * rows + j - 1] - st.m;
+      const float p = expf(zd) / st.s;
       args->p_draft[b * gamma + lane] = p;
+      if (args->logp_draft) args->logp_draft[b * gamma + lane] = zd - logf(st.s);
       bool align;
       if (args->mode == 0) align = (d == st.arg);
       else align = args->uniforms[b * rows + lane] * args->q_tok[b * gamma + lane] < p;
-      bool judge = args->has_judge && (score[j] > args->theta);
-      ok = (args->use_align && align) || (args->use_judge && judge);
+      bool judge = args->has_judge && (score[j] > args->theta[b]);
+      ok = (args->use_align && align) || (args->use_judge && judge) || args->accept_all;
     }
     unsigned rej = __ballot_sync(0xffffffffu, !ok);
     int n = rej ? (__ffs(rej) - 1) : gamma;

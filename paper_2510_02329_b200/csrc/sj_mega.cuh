@@ -890,13 +890,15 @@ __device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p,
       const int j = lane + 1;
       const int d = args->draft_ids[b * gamma + lane];
       const RowStat st = ctl->rs[j - 1];
-      const float pr = expf(__ldcg(w.tgt_logit + b * rows + j - 1) - st.m) / st.s;
+      const float zd = __ldcg(w.tgt_logit + b * rows + j - 1) - st.m;
+      const float pr = expf(zd) / st.s;
       args->p_draft[b * gamma + lane] = pr;
+      if (args->logp_draft) args->logp_draft[b * gamma + lane] = zd - logf(st.s);
       bool align;
       if (args->mode == 0) align = (d == st.arg);
       else align = args->uniforms[b * rows + lane] * args->q_tok[b * gamma + lane] < pr;
-      const bool judge = args->has_judge && (ctl->score[j] > args->theta);
-      ok = (args->use_align && align) || (args->use_judge && judge);
+      const bool judge = args->has_judge && (ctl->score[j] > args->theta[b]);
+      ok = (args->use_align && align) || (args->use_judge && judge) || args->accept_all;
     }
     const unsigned rej = __ballot_sync(0xffffffffu, !ok);
     const int n = rej ? (__ffs(rej) - 1) : gamma;

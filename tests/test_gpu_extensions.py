@@ -1,0 +1,136 @@
+"""GPU parity of the calls built around the verification step: chunked prefill (Eq. 2 on known tokens),
+per-sequence thresholds and log-probabilities, the top-2 alignment test (Sec. 4's top-k baseline) and the
+semantic-preservation score (Eq. 6-7), each against the CPU oracle on the same seeded bytes."""
+import numpy as np
+import pytest
+import torch
+
+import harness
+import helpers
+from oracle import sj_oracle as orc
+from paper_2510_02329_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+GQA = synth.ModelShape("gqa-small", 3, 256, 4, 2, 64, 512, 1024, rope_theta=5e5)
+
+
+def _binding():
+    from paper_2510_02329_b200 import binding
+    return binding
+
+
+def _empty_case(shape, dtype, n_seqs=1, gamma=4, seed=0, room=200):
+    """A target and a cache with `n_seqs` empty sequences and room for `room` tokens each."""
+    b = _binding()
+    case = harness.Case(shape, dtype, [0] * n_seqs, gamma, seed=seed, cache="fill")
+    dev = "cuda"
+    top = {k: v.to(dev) for k, v in case.model.top.items()}
+    if shape.tied_embeddings:
+        top["lm_head"] = top["embed"]
+    layers = [{k: v.to(dev) for k, v in lw.items()} for lw in case.model.layers]
+    case.target = b.Target(shape, top, layers, max_rows=64)
+    case.target.load_judge_head(case.model.judge_w, 0.0, 0.5)
+    case.kv = b.KVCache(case.target, n_seqs, n_seqs * (room // 16 + 2))
+    case.seq_ids = list(range(n_seqs))
+    return case
+
+
+PREFILL_CASES = [("tiny-f32", synth.TINY, torch.float32), ("tiny-bf16", synth.TINY, torch.bfloat16),
+                 ("gqa-bf16", GQA, torch.bfloat16), ("llama-1b-cut2-bf16", synth.LLAMA_1B.cut(2), torch.bfloat16)]
+
+
+@pytest.mark.parametrize("name,shape,dtype", PREFILL_CASES, ids=[c[0] for c in PREFILL_CASES])
+@pytest.mark.parametrize("n_prompt", [77, 33, 1])
+def test_prefill_builds_the_cache_the_oracle_prefill_builds(name, shape, dtype, n_prompt):
+    """Blocks of up to 32 (24 with four query heads per KV head) tokens, a ragged last block, a lone last token."""
+    b = _binding()
+    case = _empty_case(shape, dtype)
+    try:
+        prompt = synth.token_ids(shape.vocab, n_prompt, seed=21, stream=7)
+        nxt = case.kv.prefill(0, prompt)
+        assert case.kv.lengths([0]) == [n_prompt]
+        bf, cache = orc.prefill(case.osh, case.top64, case.model.layer64, prompt)
+        tol = harness.tol_for(dtype, float(np.abs(bf.logits).max()))
+        for l in range(shape.n_layers):
+            k, v = case.kv.read(0, l, 0, n_prompt)
+            ek = np.abs(k.cpu().double().numpy() - cache[l][0])
+            ev = np.abs(v.cpu().double().numpy() - cache[l][1])
+            assert (ek <= tol.delta(cache[l][0])).all() and (ev <= tol.delta(cache[l][1])).all(), (l, ek.max(), ev.max())
+        last = bf.logits[-1]
+        assert nxt == int(np.argmax(last)) or last.max() - last[nxt] <= 2 * tol.delta(np.abs(last).max())
+        # a verification step on top of the prefilled cache, against the oracle on the rows the library stored
+        if n_prompt > 1:
+            gamma = 4
+            si = synth.step_inputs(shape.vocab, 1, gamma, seed=22)
+            stored = [tuple(helpers.np64(t) for t in case.kv.read(0, l, 0, n_prompt)) for l in range(shape.n_layers)]
+            v2, f2 = orc.verify(case.osh, case.top64, case.model.layer64, [nxt], si.draft_ids, [stored], mode=orc.GREEDY,
+                                judge_w=case.judge_w64, theta=0.5)
+            out = b.VerifyBuffers(1, gamma, shape.d_model, shape.vocab, debug=True)
+            b.verify(case.target, case.kv, [0], torch.from_numpy(si.draft_ids).cuda(), out, commit=False)   # pending = nxt
+            case.target.sync()
+            err = np.abs(out.dbg_logits.cpu().numpy()[0] - f2[0].logits)
+            assert (err <= tol.delta(f2[0].logits)).all(), err.max()
+            assert np.abs(out.judge_scores.cpu().numpy()[0] - v2[0].judge).max() <= tol.judge_abs
+    finally:
+        case.close()
+
+
+@pytest.mark.parametrize("options", [{"gemm_impl": 1, "step_impl": 1}, {"gemm_impl": 1, "step_impl": 0}, {"gemm_impl": 0}],
+                         ids=["persistent", "tcgen05", "cudacore"])
+def test_per_sequence_thresholds_and_log_probabilities(options):
+    b = _binding()
+    thetas = [0.0, 0.5, 1.0, 0.3]
+    case = harness.Case(GQA, torch.bfloat16, [20, 33, 7, 48], 6, seed=9).gpu_setup()
+    try:
+        for k, v in options.items():
+            case.target.set_option(k, v)
+        fwd = case.oracle_forward()
+        case.kv.set_pending(case.seq_ids, case.inputs.pending)
+        out = b.VerifyBuffers(case.B, case.gamma, GQA.d_model, GQA.vocab, debug=True)
+        b.verify(case.target, case.kv, case.seq_ids, case.d_draft, out, commit=False, theta_per_seq=thetas)
+        case.target.sync()
+        g = {k: getattr(out, k).cpu().numpy() for k in ("accepted_len", "next_token", "judge_scores", "p_draft", "new_kv_len")}
+        g["hidden"], g["logits"] = out.dbg_hidden.cpu().numpy(), out.dbg_logits.cpu().numpy()
+        logp = out.logp_draft.cpu().numpy()
+        for i, th in enumerate(thetas):      # sequence by sequence: each has its own threshold
+            v = orc.verdict(fwd[i].logits, fwd[i].hidden, case.inputs.draft_ids[i], case.kv_lens[i], mode=orc.GREEDY,
+                            judge_w=case.judge_w64, theta=th)
+            near = np.abs(v.judge - th) <= 1e-3
+            if not near.any():
+                assert int(g["accepted_len"][i]) == v.accepted_len, (i, th)
+            lp = orc.log_softmax_rows(fwd[i].logits)
+            want = np.array([lp[j, case.inputs.draft_ids[i][j]] for j in range(case.gamma)])
+            assert np.abs(logp[i] - want).max() <= 4e-2 + 2e-2 * np.abs(fwd[i].logits).max()
+            assert np.allclose(np.exp(logp[i]), g["p_draft"][i], rtol=1e-4)
+        assert int(g["accepted_len"][0]) == case.gamma          # theta 0: a sigmoid is positive
+    finally:
+        case.close()
+
+
+SCORE_CASES = [("tiny-f32", synth.TINY, torch.float32, 20), ("gqa-bf16", GQA, torch.bfloat16, 20),
+               ("llama-1b-cut2-bf16", synth.LLAMA_1B.cut(2), torch.bfloat16, 20), ("tiny-bf16-n0", synth.TINY, torch.bfloat16, 0)]
+
+
+@pytest.mark.parametrize("name,shape,dtype,N", SCORE_CASES, ids=[c[0] for c in SCORE_CASES])
+def test_semantic_preservation_score(name, shape, dtype, N):
+    """N = 20 future tokens as in the paper's implementation details: two teacher-forced blocks of N + 2 rows."""
+    case = _empty_case(shape, dtype)
+    try:
+        toks = synth.token_ids(shape.vocab, 40 + 2 + N, seed=31, stream=8)
+        prefix, y_prev, y_i, future = toks[:40], int(toks[40]), int(toks[41]), toks[42:]
+        z_i = int((y_i + 17) % shape.vocab)
+        case.kv.prefill(0, prefix, want_next=False)
+        case.kv.set_pending([0], [y_prev])
+        s, s_prefix = case.kv.semantic_score(0, y_i, z_i, future)
+        assert case.kv.lengths([0]) == [40]                      # nothing was committed
+        stored = [tuple(helpers.np64(t) for t in case.kv.read(0, l, 0, 40)) for l in range(shape.n_layers)]
+        want, want_prefix = orc.semantic_preservation_score(case.osh, case.top64, case.model.layer64, stored, y_prev, y_i,
+                                                            z_i, future)
+        per_term = 1e-4 if dtype == torch.float32 else 2e-2
+        assert abs(s_prefix - want_prefix) <= 2 * per_term, (s_prefix, want_prefix)
+        assert abs(s - want) <= 2 * per_term * np.sqrt(N + 1) + per_term, (s, want)
+        same, _ = case.kv.semantic_score(0, y_i, y_i, future)    # replacing a token by itself changes nothing
+        assert same == 0.0
+    finally:
+        case.close()
