@@ -227,7 +227,7 @@ def verdict(logits: np.ndarray, hidden: np.ndarray, draft_ids: np.ndarray, n_cac
             mode: int, temperature: float = 1.0, q_tok: Optional[np.ndarray] = None,
             q_full: Optional[np.ndarray] = None, uniforms: Optional[np.ndarray] = None,
             judge_w: Optional[np.ndarray] = None, judge_b: float = 0.0, theta: float = 0.5,
-            use_align: bool = True, use_judge: bool = True) -> Verdict:
+            use_align: bool = True, use_judge: bool = True, top_k: int = 1) -> Verdict:
     """Acceptance decision for one sequence from the block's logits and hidden states.
 
     logits [gamma+1, V], hidden [gamma+1, d] (rows as in the module docstring),
@@ -236,6 +236,10 @@ def verdict(logits: np.ndarray, hidden: np.ndarray, draft_ids: np.ndarray, n_cac
 
     Decisions that compare floating-point numbers are taken in fp32, the precision the
     compared quantities are handed over in (q and u are fp32 inputs).
+
+    top_k > 1 (greedy mode) relaxes strict matching to the top-k baseline of the paper's experiments
+    (Sec. 4): d_j is aligned when it is among the k most likely target tokens, equal logits ranking
+    by token id, lowest first.
     """
     gamma = int(len(draft_ids))
     f32 = np.float32
@@ -256,7 +260,11 @@ def verdict(logits: np.ndarray, hidden: np.ndarray, draft_ids: np.ndarray, n_cac
         # strict matching: accept d_j iff it is the target's greedy token (Sec. 3.1)
         p = None
         for j in range(1, gamma + 1):
-            align[j - 1] = int(draft_ids[j - 1]) == argmax_lowest(logits[j - 1])
+            if top_k <= 1:
+                align[j - 1] = int(draft_ids[j - 1]) == argmax_lowest(logits[j - 1])
+            else:
+                ranked = np.lexsort((np.arange(logits.shape[1]), -np.asarray(logits[j - 1], F64)))   # by logit, then id
+                align[j - 1] = int(draft_ids[j - 1]) in set(int(v) for v in ranked[:top_k])
             p_draft[j - 1] = softmax_rows(logits[j - 1])[int(draft_ids[j - 1])]
     else:
         p = softmax_rows(np.asarray(logits, F64) / float(temperature))

@@ -393,6 +393,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   const int n_vtiles = (c.vocab + kTileN - 1) / kTileN;
   ALLOC(W.stats, RowStat, (size_t)n_vtiles * R);
   ALLOC(W.tgt_logit, float, R);
+  ALLOC(W.tgt_pre, float, R);
   ALLOC(W.rowstat, RowStat, R);
   ALLOC(W.status, int, 1);
   ALLOC(t->d_args, StepArgs, 1);
@@ -1011,6 +1012,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   // LM head + statistics
   const int n_vtiles = (dm.V + kTileN - 1) / kTileN;
   if (tc) {
+    TIMED("target_logits", launch(k_target_logits, dim3((R + 7) / 8), dim3(256), 0, s, pdl, args, W, dm, (const bf16*)t->lm_head, R));
     TIMED("gemm_lm_head", launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl, true));
   } else {
     GemmSegs g{{t->lm_head, nullptr, nullptr}, {dm.V, 0, 0}, 1};
@@ -1063,6 +1065,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.tmem_cols = tc;
   p.lp = t->d_layer_ptrs;
   p.embed = (const bf16*)t->embed;
+  p.lm_head = (const bf16*)t->lm_head;
   p.gain0 = (const bf16*)t->layers[0].na;
   p.sumsq = t->d_sumsq;
   p.pbuf = reinterpret_cast<unsigned long long*>(t->d_sync + 64);

@@ -125,7 +125,7 @@ __device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.laun
 struct RowStat {
   float m, s;
   int arg;
-  int pad;
+  int pad;   // top-k test: how many of the set's logits rank before the drafted token's (larger, or equal with a lower id)
 };
 __device__ __forceinline__ RowStat stat_merge(const RowStat& a, const RowStat& b) {
   // a precedes b in vocabulary order: on equal maxima the lower index (a) is kept
@@ -136,7 +136,7 @@ __device__ __forceinline__ RowStat stat_merge(const RowStat& a, const RowStat& b
   float sa = (a.m == -INFINITY) ? 0.f : a.s * expf(a.m - r.m);
   float sb = (b.m == -INFINITY) ? 0.f : b.s * expf(b.m - r.m);
   r.s = sa + sb;
-  r.pad = 0;
+  r.pad = a.pad + b.pad;
   return r;
 }
 

@@ -195,6 +195,7 @@ struct TcSmemCtl {
   uint32_t tmem_base;
   int abort_flag;
   int tgt_tok[kMaxRows];
+  float tgt_pre[kMaxRows];   // top-k test: the drafted tokens' logits, known before the head runs
   RowStat wstat[4][16];  // per epilogue warp, one group of 16 rows at a time
 };
 
@@ -329,10 +330,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       for (int r = et; r < p.R; r += 128) {
         int b = r / rows, j = r % rows;
         ctl->tgt_tok[r] = (j < args->gamma) ? args->draft_ids[b * args->gamma + j] : -1;
+        ctl->tgt_pre[r] = args->top_k >= 2 ? w.tgt_pre[r] : 0.f;
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
     }
     const float invT = p.lm_mode ? args->inv_temperature : 1.f;
+    const bool topk = p.lm_mode == 1 && args->top_k >= 2;
     float* dbg_logits = p.lm_mode ? args->dbg_logits : nullptr;
     int seg = 0;
     long long u = u_lo;
@@ -399,8 +402,15 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
             float e = (z == -INFINITY) ? 0.f : expf(z - m);
             e = warp_sum(e);
+            int before = 0;
+            if (topk) {   // block-uniform
+              const int tg = r < p.R ? ctl->tgt_tok[r] : -1;
+              const float zd = r < p.R ? ctl->tgt_pre[r] : 0.f;
+              const bool bf = r < p.R && n < V && tg >= 0 && n != tg && (v[i] > zd || (v[i] == zd && n < tg));
+              before = __popc(__ballot_sync(0xffffffffu, bf));
+            }
             if (lane == 0) {
-              RowStat st; st.m = m; st.s = e; st.arg = arg; st.pad = 0;
+              RowStat st; st.m = m; st.s = e; st.arg = arg; st.pad = before;
               ctl->wstat[quarter][i] = st;
             }
           }

@@ -36,6 +36,7 @@ struct Work {
   float* tc_o;       // [slots][4][nq][hd]              unnormalised outputs
   RowStat* stats;    // [vocab tiles, R]
   float* tgt_logit;  // [R]   logit of the drafted token d_{j+1} in row j
+  float* tgt_pre;    // [R]   the same logit (raw), computed BEFORE the LM head when the top-k test needs it to count ranks
   RowStat* rowstat;  // [R]   merged statistics
   float* logits;     // fp32 logit scratch, or null: [R, V] for the CUDA-core LM head; [B, V] in sampling mode with
                      // the tensor-core LM head (only the one row per sequence that the emitted token is drawn from)
@@ -465,6 +466,32 @@ __global__ void k_attn_combine(const StepArgs* __restrict__ args, Work w, Dims d
   }
 }
 
+// Dot product of GEMM-input row r (both bf16 planes) with one weight row, over the whole warp.
+__device__ __forceinline__ float planes_dot(const bf16* __restrict__ A, int R, int K, int r, const bf16* __restrict__ wrow,
+                                            int lane) {
+  const bf16* hi = A + (size_t)r * K;
+  const bf16* lo = A + ((size_t)pad16(R) + r) * K;
+  float acc = 0.f;
+  for (int k = lane; k < K; k += 32) acc = fmaf(__bfloat162float(hi[k]) + __bfloat162float(lo[k]), __bfloat162float(wrow[k]), acc);
+  return warp_sum(acc);
+}
+
+// Top-k alignment test with the tensor-core LM head, which stores no logits: the logit of row j's drafted token
+// d_{j+1} is computed ahead of the LM head (one dot product per row), so that the head's epilogue can count, tile
+// by tile, how many logits rank before it.  One warp per row; idle unless the step asks for top_k >= 2.
+__global__ void k_target_logits(const StepArgs* __restrict__ args, Work w, Dims dm, const bf16* __restrict__ lm_head, int R) {
+  pdl_wait();
+  pdl_launch();
+  if (args->top_k < 2) return;
+  const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= R) return;
+  const int rows = args->gamma + 1, b = r / rows, j = r % rows;
+  if (j >= args->gamma) return;
+  const int tok = min(max(args->draft_ids[b * args->gamma + j], 0), dm.V - 1);
+  const float z = planes_dot(reinterpret_cast<const bf16*>(w.A), R, dm.d, r, lm_head + (size_t)tok * dm.d, lane);
+  if (lane == 0) w.tgt_pre[r] = z;
+}
+
 // ---------------------------------------------------------------------------------------------
 // a10 (CUDA-core path): per-(128-token vocabulary tile, row) softmax statistics from stored logits
 // ---------------------------------------------------------------------------------------------
@@ -500,8 +527,19 @@ __global__ void k_lm_stats_from_logits(const StepArgs* __restrict__ args, Work w
 #pragma unroll
   for (int i = 0; i < 4; ++i) s += (z[i] == -INFINITY) ? 0.f : expf(z[i] - m);
   s = warp_sum(s);
+  int before = 0;   // top-k test: this tile's logits that rank before the drafted token's (the logits are stored here)
+  if (args->top_k >= 2 && tgt >= 0) {
+    const float zd = lg[min(tgt, dm.V - 1)];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int v = tile * kTileN + i * 32 + lane;
+      const float raw = (v < dm.V) ? lg[v] : -INFINITY;
+      const bool bf = v < dm.V && v != tgt && (raw > zd || (raw == zd && v < tgt));
+      before += __popc(__ballot_sync(0xffffffffu, bf));
+    }
+  }
   if (lane == 0) {
-    RowStat st; st.m = m; st.s = s; st.arg = arg; st.pad = 0;
+    RowStat st; st.m = m; st.s = s; st.arg = arg; st.pad = before;
     w.stats[(size_t)tile * R + r] = st;
   }
 }
@@ -561,7 +599,7 @@ __global__ void k_finalize(const StepArgs* __restrict__ args, KvView kv, Work w,
       args->p_draft[b * gamma + lane] = p;
       if (args->logp_draft) args->logp_draft[b * gamma + lane] = zd - logf(st.s);
       bool align;
-      if (args->mode == 0) align = (d == st.arg);
+      if (args->mode == 0) align = args->top_k >= 2 ? st.pad < args->top_k : (d == st.arg);
       else align = args->uniforms[b * rows + lane] * args->q_tok[b * gamma + lane] < p;
       bool judge = args->has_judge && (score[j] > args->theta[b]);
       ok = (args->use_align && align) || (args->use_judge && judge) || args->accept_all;

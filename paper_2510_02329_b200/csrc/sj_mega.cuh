@@ -76,6 +76,7 @@ struct MegaParams {
   uint32_t tmem_cols;
   const MegaLayerPtrs* lp;    // [n_layers], device
   const bf16* embed;
+  const bf16* lm_head;        // rows of the LM head (top-k test: the drafted tokens' logits are computed ahead of the head)
   const bf16* gain0;          // first layer's attention-norm gain
   float* sumsq;               // [2][d/128][kMegaMaxRows]
   // Split-K partial sums, [blocks][Rp][128] words of 64 bits: the fp32 value in the low half and, in the
@@ -129,6 +130,7 @@ struct MegaCtl {
   int bars_passed;
   int bcast[6];   // [2 * group + accumulator]: the group's wait on that accumulator succeeded; [4], [5] spare
   float inv[kMegaMaxRows];
+  float zd[kMegaMaxRows];      // top-k test: raw logit of each row's drafted token, computed before the LM head
   int row_b[kMegaMaxRows], row_j[kMegaMaxRows], row_page[kMegaMaxRows], row_slot[kMegaMaxRows], tgt_tok[kMegaMaxRows];
   int row_qoff[kMegaMaxRows];         // element offset of row r's queries in the query buffer, without the head part
   int row_nkvoff[kMegaMaxRows];       // element offset of row r in the fp16 copy of the step's own K/V rows, without head / K|V part
@@ -410,6 +412,21 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
     }
     bar_sync(bar_id, 128);
   }
+  const bool topk = site == SITE_LM && args->top_k >= 2;   // block-uniform
+  if (topk) {
+    // The LM head stores no logits, so the rank of a drafted token is counted tile by tile against its own
+    // logit, which therefore has to exist first: one dot product per row (this group's rows, a warp each).
+    const int gamma = rows - 1;
+    for (int r = quarter; r < R; r += 4) {
+      if (mega_row_group(r, R) != grp) continue;
+      const int tok = ctl->tgt_tok[r];
+      float z = 0.f;
+      if (tok >= 0) z = planes_dot(reinterpret_cast<const bf16*>(w.A), R, dm.d, r, p.lm_head + (size_t)min(tok, dm.V - 1) * dm.d, lane) * ctl->inv[r];
+      if (lane == 0) ctl->zd[r] = z;
+    }
+    (void)gamma;
+    bar_sync(bar_id, 128);
+  }
   const int qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd, tq = qd / kTileN, tk = kd / kTileN;
   const float invT = (site == SITE_LM) ? args->inv_temperature : 1.f;
   float* dbg_logits = (site == SITE_LM) ? args->dbg_logits : nullptr;
@@ -677,8 +694,15 @@ __device__ __forceinline__ void mega_epilogue(int site, int l, int gseq, int& se
           }
           float e = (z == -INFINITY) ? 0.f : expf(z - m);
           e = warp_sum(e);
+          int before = 0;
+          if (topk) {
+            const int rr = min(r, R - 1), tg = ctl->tgt_tok[rr];
+            const float raw = v[i] * ctl->inv[rr], zd = ctl->zd[rr];
+            const bool bf = r < rend && n < dm.V && tg >= 0 && n != tg && (raw > zd || (raw == zd && n < tg));
+            before = __popc(__ballot_sync(0xffffffffu, bf));
+          }
           if (lane == 0) {
-            RowStat st; st.m = m; st.s = e; st.arg = arg; st.pad = 0;
+            RowStat st; st.m = m; st.s = e; st.arg = arg; st.pad = before;
             ctl->wstat[grp][quarter][i] = st;
           }
         }
@@ -844,7 +868,7 @@ __device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p,
     for (int t = t0; t < t1; ++t) {
       RowStat x;
       const float4 raw = __ldcg(reinterpret_cast<const float4*>(w.stats + (size_t)t * R + r));
-      x.m = raw.x; x.s = raw.y; x.arg = __float_as_int(raw.z); x.pad = 0;
+      x.m = raw.x; x.s = raw.y; x.arg = __float_as_int(raw.z); x.pad = __float_as_int(raw.w);
       a = stat_merge(a, x);
     }
     ctl->u.sred[wt] = a;
@@ -895,7 +919,7 @@ __device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p,
       args->p_draft[b * gamma + lane] = pr;
       if (args->logp_draft) args->logp_draft[b * gamma + lane] = zd - logf(st.s);
       bool align;
-      if (args->mode == 0) align = (d == st.arg);
+      if (args->mode == 0) align = args->top_k >= 2 ? st.pad < args->top_k : (d == st.arg);
       else align = args->uniforms[b * rows + lane] * args->q_tok[b * gamma + lane] < pr;
       const bool judge = args->has_judge && (ctl->score[j] > args->theta[b]);
       ok = (args->use_align && align) || (args->use_judge && judge) || args->accept_all;

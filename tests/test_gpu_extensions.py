@@ -134,3 +134,64 @@ def test_semantic_preservation_score(name, shape, dtype, N):
         assert same == 0.0
     finally:
         case.close()
+
+
+@pytest.mark.parametrize("dtype,options", [(torch.float32, {}), (torch.bfloat16, {"gemm_impl": 0}),
+                                            (torch.bfloat16, {"gemm_impl": 1, "step_impl": 0}),
+                                            (torch.bfloat16, {"gemm_impl": 1, "step_impl": 1})],
+                         ids=["f32", "bf16-cudacore", "bf16-tcgen05", "bf16-persistent"])
+def test_top_two_alignment(dtype, options):
+    """Drafts built from the oracle's own ranking: the target's best token, its second best, its third best, a
+    random one.  With top_k = 2 the first two kinds are aligned, the others are not (judge off)."""
+    b = _binding()
+    gamma = 6
+    probe = harness.Case(GQA, dtype, [30, 9, 41], gamma, seed=17)
+    # the ranking of row j depends on drafts 1..j only: build the drafts position by position
+    kinds = np.array([[0, 1, 0, 1, 2, 0], [1, 1, 1, 0, 0, 3], [0, 0, 2, 0, 0, 0]])   # 0 best, 1 second, 2 third, 3 random
+    drafts = probe.inputs.draft_ids.copy()
+    caches = [[(helpers.np64(k), helpers.np64(v)) for k, v in seq] for seq in probe.cache_t]
+    for j in range(gamma):
+        for i in range(3):
+            toks = np.concatenate([[int(probe.inputs.pending[i])], drafts[i, :j]])
+            row = orc.forward_blocks(probe.osh, probe.top64, probe.model.layer64, [toks], [caches[i]])[0].logits[-1]
+            ranked = np.lexsort((np.arange(row.size), -row))
+            if kinds[i, j] < 3:
+                drafts[i, j] = ranked[kinds[i, j]]
+    case = harness.Case(GQA, dtype, [30, 9, 41], gamma, seed=17, draft_ids=drafts).gpu_setup()
+    try:
+        for k, v in options.items():
+            case.target.set_option(k, v)
+        fwd = case.oracle_forward()
+        tol = harness.tol_for(dtype, float(max(np.abs(f.logits).max() for f in fwd)))
+        checked = 0
+        for top_k in (1, 2):
+            case.kv.set_pending(case.seq_ids, case.inputs.pending)
+            out = b.VerifyBuffers(case.B, gamma, GQA.d_model, GQA.vocab, debug=True)
+            b.verify(case.target, case.kv, case.seq_ids, case.d_draft, out, commit=False, use_judge=False, top_k=top_k)
+            case.target.sync()
+            got = out.accepted_len.cpu().numpy()
+            glog = out.dbg_logits.cpu().numpy()
+            for i in range(3):
+                v = orc.verdict(fwd[i].logits, fwd[i].hidden, drafts[i], case.kv_lens[i], mode=orc.GREEDY, use_judge=False,
+                                top_k=top_k)
+                err = np.abs(glog[i] - fwd[i].logits)
+                assert (err <= tol.delta(fwd[i].logits)).all()
+                # a decision can only come out differently where the draft's logit is within twice the actual
+                # logit error of the boundary between ranks top_k - 1 and top_k
+                crisp = True
+                for j in range(min(v.accepted_len + 1, gamma)):
+                    row = fwd[i].logits[j]
+                    srt = np.sort(row)[::-1]
+                    zd = row[drafts[i, j]]
+                    edge = srt[top_k] if zd >= srt[top_k - 1] else srt[top_k - 1]
+                    crisp = crisp and abs(zd - edge) > 2 * err[j].max()
+                if crisp:
+                    assert int(got[i]) == v.accepted_len, (top_k, i, got, v.accepted_len)
+                    checked += 1
+        assert checked >= 5
+        # the construction itself: with k = 2 sequence 0 stops at its third-best draft, sequence 1 at the random one
+        v0 = orc.verdict(fwd[0].logits, fwd[0].hidden, drafts[0], 30, mode=orc.GREEDY, use_judge=False, top_k=2)
+        v1 = orc.verdict(fwd[0].logits, fwd[0].hidden, drafts[0], 30, mode=orc.GREEDY, use_judge=False, top_k=1)
+        assert v0.accepted_len == 4 and v1.accepted_len == 1
+    finally:
+        case.close()

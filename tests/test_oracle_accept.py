@@ -189,3 +189,27 @@ def test_residual_with_zero_mass_falls_back_to_the_target_distribution():
     v = orc.verdict(logits, hidden, np.array([1]), 5, mode=orc.SAMPLING, q_tok=np.array([1.0]), q_full=q_full,
                     uniforms=np.array([0.99, 0.5]), use_judge=False)
     assert v.accepted_len == 0 and v.next_token == 2
+
+
+def test_top_k_alignment_is_rank_below_k_brute_force():
+    """Top-k baseline (Sec. 4): a draft is aligned iff fewer than k tokens rank before it, a token ranking before
+    another when its logit is larger or equal with a lower id.  k = 1 is strict matching."""
+    rng = np.random.default_rng(5)
+    for trial in range(200):
+        gamma, V = int(rng.integers(1, 6)), int(rng.integers(3, 10))
+        logits = np.round(rng.standard_normal((gamma + 1, V)) * 2.0) / 2.0      # coarse values: many exact ties
+        hidden = np.zeros((gamma + 1, 4))
+        drafts = rng.integers(0, V, gamma)
+        for k in (1, 2, 3):
+            v = orc.verdict(logits, hidden, drafts, 3, mode=orc.GREEDY, use_judge=False, top_k=k)
+            n = 0
+            for j in range(gamma):
+                d = int(drafts[j])
+                before = sum(1 for t in range(V) if t != d and (logits[j, t] > logits[j, d] or (logits[j, t] == logits[j, d] and t < d)))
+                if before >= k:
+                    break
+                n += 1
+            assert v.accepted_len == n, (trial, k)
+            assert v.next_token == int(np.argmax(logits[n]))
+        strict = orc.verdict(logits, hidden, drafts, 3, mode=orc.GREEDY, use_judge=False)
+        assert strict.accepted_len == orc.verdict(logits, hidden, drafts, 3, mode=orc.GREEDY, use_judge=False, top_k=1).accepted_len
