@@ -195,3 +195,72 @@ def test_top_two_alignment(dtype, options):
         assert v0.accepted_len == 4 and v1.accepted_len == 1
     finally:
         case.close()
+
+
+def _target_and_cache(shape, dtype, seed, n_seqs, room=128):
+    b = _binding()
+    model = helpers.HostModel(shape, dtype, "cpu", seed)
+    top = {k: v.cuda() for k, v in model.top.items()}
+    layers = [{k: v.cuda() for k, v in lw.items()} for lw in model.layers]
+    t = b.Target(shape, top, layers, max_rows=64)
+    t.load_judge_head(model.judge_w, 0.0, 0.5)
+    return model, t, b.KVCache(t, n_seqs, n_seqs * (room // 16 + 2))
+
+
+def test_speculative_loop_reproduces_the_targets_greedy_decoding():
+    """Draft passes + verification + cache roll-back as a loop.  With the judge off, speculative decoding at
+    temperature 0 must emit exactly what the target alone would (Sec. 3.1: the target distribution is kept);
+    the first tokens are also checked against the oracle's own greedy continuation."""
+    from paper_2510_02329_b200 import loop
+    shape, gamma, n_out = synth.TINY, 4, 14
+    tm, target, target_kv = _target_and_cache(shape, torch.float32, 0, 2)
+    _, draft, draft_kv = _target_and_cache(shape, torch.float32, 1, 2)        # another random model of the same shape
+    _, solo, solo_kv = _target_and_cache(shape, torch.float32, 0, 2)
+    try:
+        prompts = [list(synth.token_ids(shape.vocab, 9, seed=41, stream=3)), list(synth.token_ids(shape.vocab, 5, seed=42, stream=3))]
+        dec = loop.SpeculativeDecoder(draft, draft_kv, target, target_kv, [0, 1], gamma)
+        dec.prefill(prompts)
+        got = dec.generate(n_out, use_judge=False)
+        want = [loop.greedy_decode(solo, solo_kv, s, prompts[s], n_out) for s in (0, 1)]
+        assert got == want
+        assert 0.0 <= dec.mean_accepted_length < gamma       # an unrelated draft is mostly rejected
+        # oracle: greedy continuation by full recomputes (tiny model)
+        osh, top64 = helpers.oracle_shape(shape), tm.top64()
+        seq = list(prompts[0])
+        for k in range(4):
+            bf, _ = orc.prefill(osh, top64, tm.layer64, np.asarray(seq))
+            row = bf.logits[-1]
+            srt = np.sort(row)
+            if srt[-1] - srt[-2] < 1e-3:
+                break
+            assert got[0][k] == int(np.argmax(row))
+            seq.append(got[0][k])
+        # with the judge threshold at 0 every draft is accepted: the loop then follows the draft model
+        dec2 = loop.SpeculativeDecoder(draft, draft_kv, target, target_kv, [0, 1], gamma)
+        target_kv.rollback([0, 1], [0, 0]); draft_kv.rollback([0, 1], [0, 0])
+        dec2.prefill(prompts)
+        dec2.generate(10, use_judge=True, theta=0.0)
+        assert dec2.mean_accepted_length == gamma
+    finally:
+        for kv in (target_kv, draft_kv, solo_kv):
+            kv.close()
+        for t in (target, draft, solo):
+            t.close()
+
+
+def test_speculative_loop_with_the_target_as_its_own_draft_accepts_everything():
+    from paper_2510_02329_b200 import loop
+    shape, gamma = GQA, 5
+    _, target, target_kv = _target_and_cache(shape, torch.bfloat16, 0, 1)
+    _, draft, draft_kv = _target_and_cache(shape, torch.bfloat16, 0, 1)
+    try:
+        prompt = list(synth.token_ids(shape.vocab, 20, seed=43, stream=3))
+        dec = loop.SpeculativeDecoder(draft, draft_kv, target, target_kv, [0], gamma)
+        dec.prefill([prompt])
+        out = dec.generate(24, use_judge=False)
+        # a draft pass sees one row, the verification gamma + 1: same model, slightly different rounding, so a
+        # rejection can only happen at a near-tie of the two best logits
+        assert dec.mean_accepted_length >= gamma - 1.0
+        assert len(out[0]) == 24
+    finally:
+        target_kv.close(); draft_kv.close(); target.close(); draft.close()
