@@ -8,6 +8,10 @@ drafted token (Eq. 4, Eq. 5), the either-test-accepts rule (Sec. 3.2, App. D.2),
 accept-until-first-rejection scan (Sec. 3.1), the token emitted after the accepted prefix
 and the resulting cache length.
 
+Also here, for the calls built around the step: the top-k alignment baseline of the paper's
+experiments (Sec. 4) and the semantic-preservation score that labels the verifier's training
+tokens (Sec. 3.3, Eq. 6 in the autoregressive form of Eq. 7).
+
 It is independent of the CUDA library: it imports nothing from it, shares no helper,
 table or constant with it, and is only ever called from tests, the smoke check and the
 benchmark's CPU-baseline leg.  numpy's matmul is the only library primitive used; there
