@@ -12,7 +12,7 @@
 // Roles per block (384 threads):
 //   warp 0      weight / cache-tile producer (TMA into the ring; never stops at a phase boundary)
 //   warp 1      tcgen05.mma issuer, owns the TMEM allocation
-//   warp 2      activation producer: TMA of the activation K-slices, gated by the device-wide barrier
+//   warps 2, 3  activation producers: TMA of the activation K-slices (alternate units), gated by the device-wide barrier
 //   warps 4..11 workers: all eight drain TMEM (fused epilogues, two groups of four warps) and run attention,
 //               the combine, the embedding and the final acceptance phase
 //
@@ -1120,9 +1120,14 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       auto fatt = [&](int l) { rp.advance(n_att); };
       mega_walk(p, fsite, fatt);
     }
-  } else if (warp == 2) {
-    // ------------------------------ activation producer ------------------------------
+  } else {
+    // ------------------------------ activation producers (warps 2 and 3) ------------------------------
+    // Two threads, alternate units: right after a device-wide barrier the ring already holds the phase's first
+    // weight tiles, and the MMAs can start only as fast as their activation slices are requested (a wait, an
+    // expect and a TMA per slice cost one thread about a quarter of a microsecond).
     if (lane == 0) {
+      const int mine = warp - 2;
+      int n_unit = 0;
       const uint64_t pol_a = l2_policy_evict_last();
       const uint32_t a_tx = (uint32_t)(2 * Rp) * 128u;
       RingPos rp{0, 0, NS};
@@ -1136,23 +1141,25 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           if (!mega_wait_bars(nb, ctl, p, w.status, 3)) { alive = false; return; }
           __threadfence();
           fence_proxy_async();
-          MEGA_EV(sidx, 0);
+          if (mine == 0) MEGA_EV(sidx, 0);
           const CUtensorMap* tm = (site == SITE_O) ? &mp.a_q : (site == SITE_DOWN ? &mp.a_f : &mp.a_d);
           unsigned u = ss.g_lo;
           Seg sg;
           while (seg_next(ss, u, sg)) {
-            for (int kb = sg.a; kb < sg.b; ++kb) {
-              if (rp.r > 0 && !mega_wait(smem_u32(&ctl->empty[rp.s]), (uint32_t)(rp.r - 1) & 1u, ctl, p, w.status, 2, rp.r)) {
-                alive = false;
-                return;
+            for (int kb = sg.a; kb < sg.b; ++kb, ++n_unit) {
+              if ((n_unit & 1) == mine) {
+                if (rp.r > 0 && !mega_wait(smem_u32(&ctl->empty[rp.s]), (uint32_t)(rp.r - 1) & 1u, ctl, p, w.status, 2, rp.r)) {
+                  alive = false;
+                  return;
+                }
+                const uint32_t bar = smem_u32(&ctl->full[rp.s]);
+                mbar_expect_tx(bar, a_tx);
+                tma_load_2d(stage_addr(rp.s) + kWTileBytes, tm, bar, kb * kBK, 0, pol_a);
               }
-              const uint32_t bar = smem_u32(&ctl->full[rp.s]);
-              mbar_expect_tx(bar, a_tx);
-              tma_load_2d(stage_addr(rp.s) + kWTileBytes, tm, bar, kb * kBK, 0, pol_a);
               rp.next();
             }
           }
-          MEGA_EV(sidx, 1);
+          if (mine == 0) MEGA_EV(sidx, 1);
         }
         ++sidx;
         nb += (site == SITE_QKV) ? 3 : 1;
