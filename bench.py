@@ -386,6 +386,17 @@ def main():
             barrier()
             ms_total = e0.elapsed_time(e1)
             dw.target.sync()
+            # latency spread: every step between its own pair of events (same steps, a second short pass)
+            n_lat = min(args.steps, 50)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_lat)]
+            for a_ev, b_ev in evs:
+                a_ev.record(stream)
+                dw.step(mode)
+                b_ev.record(stream)
+            stream.synchronize()
+            lat = sorted(a_ev.elapsed_time(b_ev) for a_ev, b_ev in evs)
+            latency = {"p10": lat[int(0.1 * (n_lat - 1))], "p50": lat[(n_lat - 1) // 2], "p90": lat[int(0.9 * (n_lat - 1))],
+                       "steps": n_lat, "unit": "ms"}
 
             # ---------------- end to end: host buffers in, results out, every step ----------------
             si = dw.inputs
@@ -509,7 +520,7 @@ def main():
         "config": {"workload": wl.name, "shape": dw.shape.name, "layers": dw.shape.n_layers, "batch": wl.batch,
                    "gamma": wl.gamma, "kv_len_total": int(sum(dw.kv_lens)), "mode": args.mode, "replicas": world,
                    "positions_per_step": R, "l2": "inputs larger than L2 (weights stream from HBM every step)"},
-        "verify_steps_per_s": world * 1e3 / ms_step,
+        "verify_steps_per_s": world * 1e3 / ms_step, "step_latency_ms": latency,
         "committed_tokens_per_s": float((accepted + 1).sum()) * world * 1e3 / ms_step,
         "step_hbm_gbs": step_gbs, "step_hbm_frac_of_measured_copy": step_gbs / peak, "step_hbm_frac_of_8tbs": step_gbs / 8000.0,
         "algorithmic_bytes_per_step": w_bytes + kv_bytes,
