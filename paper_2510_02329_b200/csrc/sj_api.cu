@@ -14,6 +14,7 @@
 
 #include "../../include/sj.h"
 #include "sj_attn_tc.cuh"
+#include "sj_attn_t5.cuh"
 #include "sj_gemm_tc.cuh"
 #include "sj_mega.cuh"
 
@@ -485,6 +486,10 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     t->opt_step = 1;
   }
 #undef ALLOC
+  if (t->bf && c.head_dim == 128) {
+    cudaError_t e = cudaFuncSetAttribute(k_attn_t5, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kT5SmemBytes + sizeof(T5Ctl) + 1024));
+    if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "smem opt-in: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
+  }
   if (t->bf) {
     const int att_smem = kAttStages * kAttStageBytes + (int)sizeof(AttSmemCtl) + 1024;
     cudaError_t e = c.head_dim == 128
@@ -532,8 +537,9 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
     if (value == 1 && !tc_shapes_ok(t->cfg)) return fail(SJ_ERR_UNSUPPORTED, "tensor-core GEMM needs bf16 and 128-multiples");
     t->opt_gemm = value;
   } else if (n == "attn_impl") {
-    if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "attn_impl must be 0 or 1");
-    if (value == 1 && !t->bf) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention needs a bf16 model");
+    if (value < 0 || value > 2) return fail(SJ_ERR_INVALID_ARG, "attn_impl must be 0, 1 or 2");
+    if (value >= 1 && !t->bf) return fail(SJ_ERR_UNSUPPORTED, "tensor-core attention needs a bf16 model");
+    if (value == 2 && t->dm.hd != 128) return fail(SJ_ERR_UNSUPPORTED, "the tcgen05 attention needs head_dim 128");
     t->opt_attn = value;
   } else if (n == "step_impl") {
     if (value != 0 && value != 1) return fail(SJ_ERR_INVALID_ARG, "step_impl must be 0 or 1");
@@ -928,7 +934,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   const int R = B * (gamma + 1), qd = dm.Hq * dm.hd, kd = dm.Hkv * dm.hd;
   const bool timing = t->opt_timing != 0 && !t->opt_graph;
   const bool pdl = t->opt_pdl != 0 && !timing, tc = t->opt_gemm == 1;
-  const bool attn_tc = t->opt_attn == 1 && t->bf && kv->has_tm_pool;
+  const bool attn_tc = t->opt_attn >= 1 && t->bf && kv->has_tm_pool;
   const StepArgs* args = t->d_args;
   Work W = t->work;
   if (!use_scratch) W.logits = nullptr;
@@ -968,12 +974,16 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
       const size_t tc_smem = kAttStages * kAttStageBytes + sizeof(AttSmemCtl) + 1024;
       const AttPartials parts{W.tc_m, W.tc_l, W.tc_o};
       const int items = B * dm.Hkv * nq, cgrid = std::max(1, std::min(4 * t->sm_count, (items + 7) / 8));
-      if (dm.hd == 128) {
+      if (dm.hd == 128 && t->opt_attn == 2) {
+        const size_t t5_smem = kT5SmemBytes + sizeof(T5Ctl) + 1024;
+        TIMED("attn", launch(k_attn_t5, dim3(t->sm_count), dim3(kT5Threads), t5_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, kT5Keys));
+      } else if (dm.hd == 128) {
         TIMED("attn", launch(k_attn_tc<128>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0));
       } else {
         TIMED("attn", launch(k_attn_tc<64>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<64>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base));
+        TIMED("attn_combine", launch(k_attn_combine_tc<64>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0));
       }
     } else {
       TIMED("attn", launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
@@ -1013,7 +1023,7 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
   const int n_vtiles = (dm.V + kTileN - 1) / kTileN;
   if (tc) {
     TIMED("target_logits", launch(k_target_logits, dim3((R + 7) / 8), dim3(256), 0, s, pdl, args, W, dm, (const bf16*)t->lm_head, R));
-    TIMED("gemm_lm_head", launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl, true));
+    TIMED("gemm_lm_head", launch_tc(t, t->s_lm, mA_d, &t->m_lm, nullptr, nullptr, R, pdl, true, -1, &W));   // W: no [R, V] logit store
   } else {
     GemmSegs g{{t->lm_head, nullptr, nullptr}, {dm.V, 0, 0}, 1};
     TIMED("gemm_cudacore", launch_simt<T>(t, W.A, g, W.logits, R, dm.V, dm.d, pdl));
@@ -1231,7 +1241,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
     t->att_chunks_cap = cap;
     t->att_rows_cap = rcap;
   }
-  if ((t->opt_attn == 1 || use_mega) && t->bf && kv->has_tm_pool) {
+  if ((t->opt_attn >= 1 || use_mega) && t->bf && kv->has_tm_pool) {
     const size_t slots = (size_t)t->sm_count + 2 * (size_t)B * t->dm.Hkv;
     const size_t need = slots * kAttMaxSub * (size_t)(group * rows);
     if (need > t->tc_part_cap) {

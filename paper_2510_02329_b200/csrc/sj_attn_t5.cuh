@@ -1,0 +1,380 @@
+// Attention of the verification step on the 5th-generation tensor cores (head dimension 128, bf16 cache):
+// the cached keys of the multi-kernel path, split along the keys over all SMs like sj_attn_tc.cuh's kernel,
+// but with both contractions on tcgen05.mma and the scores in tensor memory.
+//
+// One work tile is 128 cached keys of one (sequence, KV head): K and V of its 8 pages arrive by TMA (boxes of
+// 16 slots x 64 dims, 128-byte swizzle) as two 32 KiB shared-memory tiles laid out [half of the head dim][page]
+// [16 keys x 128 B], so that the 128 key rows of a half sit 128 bytes apart.
+//   S = Q K^T   M = 128 query-row slots (the group's gamma+1 rows of every query head; unused slots are zero),
+//               N = 128 keys, K = head dim: Q from shared memory (K-major), the key tile as a K-major B operand.
+//               The cache is bf16, and both operands of an MMA have one type, so a query enters as the sum of two
+//               bf16 terms (hi + lo, 16 significant bits): two MMAs per 16-dim step into the same accumulator.
+//   softmax     one thread per query-row slot reads its row of S from tensor memory (no cross-lane traffic),
+//               keeps a stabiliser m (raised only when the row maximum exceeds it by more than 8 in the log2
+//               domain: then the thread rescales its row of O), and writes P = exp2(S - m) back to tensor memory
+//               as two bf16 terms.
+//   O += P V    A = P from tensor memory (M = 128 slots, K = 16 keys per step = one page), B = the page's V rows
+//               as an MN-major operand (the head dim is the contiguous one: leading byte offset = the 16 KiB
+//               between the two halves, stride byte offset = the 1 KiB between 8-key groups), N = head dim.
+// A segment (the block's run of tiles of one (sequence, KV head)) ends with the unnormalised partial (m, l, o)
+// per query row, in the format of sj_attn_tc.cuh, whose combine pass merges them; the block's own gamma+1 rows
+// (the causal tail) are handled by two extra warps with that file's mma.sync routine.
+//
+// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer (owns tensor memory: S twice, P, O = 512
+// columns), warps 2..5 softmax (TMEM lane quarter = warp % 4), warps 6..7 tails.  Every wait is bounded.
+#pragma once
+
+#include "sj_attn_tc.cuh"
+#include "sj_gemm_tc.cuh"
+
+namespace sj {
+
+constexpr int kT5Keys = 128;               // keys per tile
+constexpr int kT5Threads = 256;
+constexpr int kT5TileBytes = 32768;        // one K or V tile: 2 halves x 8 pages x 2 KiB
+constexpr int kT5SmemBytes = 2 * kT5TileBytes /* Q hi, lo */ + 4 * kT5TileBytes /* K, V double-buffered */;
+
+struct T5Ctl {
+  uint64_t kfull[2], kempty[2], vfull[2], vempty[2], s_full[2], s_free[2], p_full, o_done, q_ready;
+  uint32_t tmem_base;
+  int abort_flag;
+  AttPlan plan;
+  int pages[kAttPageCache];
+};
+
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,"
+      "%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tc_st32f(uint32_t taddr, const float* v) {
+  uint32_t r[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+  tc_st16(taddr, r);
+  tc_st16(taddr + 16, r + 16);
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory descriptor of an MN-major operand in the [half][page][16 x 128 B] layout: 16 keys (one page) by
+// 128 dims; the two 64-dim halves are `half_stride` bytes apart, the two 8-key groups 1024 bytes.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t saddr, uint32_t half_stride) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((half_stride >> 4) & 0x3FFF) << 16;   // leading byte offset: along the contiguous (head) dimension
+  d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset: along the keys
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// bf16 x bf16 -> fp32, M = 128, N = n; b_mn: the B operand is MN-major
+__device__ __forceinline__ uint32_t instr_desc_bf16_mn(int n, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+// byte offset of (row, dim) in a K-major tile of two [rows x 128 B] halves 16 KiB apart, 128-byte swizzle
+__device__ __forceinline__ uint32_t t5_q_off(int row, int dim) {
+  const int h = dim >> 6, c = (dim & 63) >> 3;
+  return (uint32_t)(h * 16384 + row * 128 + ((c ^ (row & 7)) << 4) + (dim & 7) * 2);
+}
+// TMEM lane of query row q: the rows are dealt round-robin to the four lane quarters (one softmax warp each)
+__device__ __forceinline__ int t5_lane_of_row(int q) { return 32 * (q & 3) + (q >> 2); }
+
+__device__ __forceinline__ bool t5_wait(uint64_t* bar, uint32_t parity, T5Ctl* ctl, int* status, int where) {
+  return att_mbar_wait(att_smem_u32(bar), parity, &ctl->abort_flag, status, nullptr, where, 0);
+}
+
+__global__ void __launch_bounds__(kT5Threads, 1)
+k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__ args, KvView kv, Work w, Dims dm, AttArgs a) {
+  constexpr int HD = 128;
+  extern __shared__ uint8_t t5_smem_raw[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(t5_smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t *sQ = sm, *sK = sm + 2 * kT5TileBytes, *sV = sm + 4 * kT5TileBytes;
+  T5Ctl* ctl = reinterpret_cast<T5Ctl*>(sm + kT5SmemBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_wait();
+  pdl_launch();
+  const int B = args->B, rows = args->gamma + 1, Hkv = dm.Hkv, group = dm.Hq / dm.Hkv, nq = group * rows;
+  const int G = gridDim.x, c = blockIdx.x;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2; ++i) {
+      att_mbar_init(att_smem_u32(&ctl->kfull[i]), 1);
+      att_mbar_init(att_smem_u32(&ctl->kempty[i]), 1);
+      att_mbar_init(att_smem_u32(&ctl->vfull[i]), 1);
+      att_mbar_init(att_smem_u32(&ctl->vempty[i]), 1);
+      att_mbar_init(att_smem_u32(&ctl->s_full[i]), 1);
+      att_mbar_init(att_smem_u32(&ctl->s_free[i]), 128);
+    }
+    att_mbar_init(att_smem_u32(&ctl->p_full), 128);
+    att_mbar_init(att_smem_u32(&ctl->o_done), 1);
+    att_mbar_init(att_smem_u32(&ctl->q_ready), 128);
+    ctl->abort_flag = 0;
+    att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, kT5Keys);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // unused query-row slots stay zero for the whole kernel
+  for (int i = threadIdx.x; i < 2 * kT5TileBytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(att_smem_u32(&ctl->tmem_base)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const AttPlan& pl = ctl->plan;
+  const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
+  att_fill_pages(ctl->pages, pl, kv, args, B, kT5Keys, t_lo, t_hi, threadIdx.x, blockDim.x);
+  __syncthreads();
+  const uint32_t tmem = ctl->tmem_base;   // columns: [0,256) S twice, [256,384) P (hi 64, lo 64), [384,512) O
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      int g = 0;
+      for (long long t = t_lo; t < t_hi; ++t, ++g) {
+        const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
+        const int st = g & 1, seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
+        int page[8];
+        for (int p = 0; p < 8; ++p) {
+          int pi = x.ti * 8 + p;
+          if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
+          page[p] = (g + 1) * 8 <= kAttPageCache ? ctl->pages[g * 8 + p]
+                                                 : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+        }
+        for (int which = 0; which < 2; ++which) {   // the key tile, then the value tile
+          uint64_t* full = which ? &ctl->vfull[st] : &ctl->kfull[st];
+          uint64_t* empty = which ? &ctl->vempty[st] : &ctl->kempty[st];
+          if (g >= 2 && !t5_wait(empty, (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 1)) goto producer_done;
+          const uint32_t bar = att_smem_u32(full);
+          const uint32_t dst = att_smem_u32((which ? sV : sK) + (size_t)st * kT5TileBytes);
+          att_mbar_expect_tx(bar, kT5TileBytes);
+          for (int p = 0; p < 8; ++p) {
+            const long long row = ((((long long)a.layer * kv.n_pages + page[p]) * 2 + which) * kv.n_kv_heads + x.h) * 16;
+            att_tma_2d(dst + (uint32_t)(p * 2048), &tmKV, bar, 0, (int)row);
+            att_tma_2d(dst + 16384u + (uint32_t)(p * 2048), &tmKV, bar, 64, (int)row);
+          }
+        }
+      }
+    }
+  producer_done:;
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      const uint32_t id_s = instr_desc_bf16_mn(kT5Keys, 0), id_o = instr_desc_bf16_mn(HD, 1);
+      const uint32_t q0 = att_smem_u32(sQ), k0 = att_smem_u32(sK), v0 = att_smem_u32(sV);
+      int it = 0, seg = 0;
+      long long t = t_lo;
+      bool alive = true;
+      while (t < t_hi && alive) {
+        const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
+        const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+        if (!t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2)) break;
+        tc_fence_after();
+        for (int i = 0; i <= n && alive; ++i) {
+          if (i < n) {   // scores of tile i
+            const int g = it + i, st = g & 1;
+            if (!t5_wait(&ctl->kfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 3) ||
+                (g >= 2 && !t5_wait(&ctl->s_free[st], (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 4))) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t kb = k0 + (uint32_t)st * kT5TileBytes, d_s = tmem + (uint32_t)(st * 128);
+#pragma unroll
+            for (int k = 0; k < HD / 16; ++k) {
+              const uint32_t off = (uint32_t)((k >> 2) * 16384 + (k & 3) * 32);
+              const uint64_t db = smem_desc_sw128(kb + off);
+              tc_mma_bf16(d_s, smem_desc_sw128(q0 + off), db, id_s, k > 0 ? 1u : 0u);
+              tc_mma_bf16(d_s, smem_desc_sw128(q0 + kT5TileBytes + off), db, id_s, 1u);
+            }
+            tc_commit(att_smem_u32(&ctl->kempty[st]));
+            tc_commit(att_smem_u32(&ctl->s_full[st]));
+          }
+          if (i >= 1) {  // output of tile i - 1
+            const int g = it + i - 1, st = g & 1;
+            if (!t5_wait(&ctl->p_full, (uint32_t)g & 1u, ctl, w.status, 5) ||
+                !t5_wait(&ctl->vfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 6)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t vb = v0 + (uint32_t)st * kT5TileBytes;
+#pragma unroll
+            for (int pg = 0; pg < 8; ++pg) {
+              const uint64_t db = smem_desc_mn_sw128(vb + (uint32_t)(pg * 2048), 16384u);
+              tc_mma_bf16_ta(tmem + 384, tmem + 256 + (uint32_t)(8 * pg), db, id_o, (i > 1 || pg > 0) ? 1u : 0u);
+              tc_mma_bf16_ta(tmem + 384, tmem + 320 + (uint32_t)(8 * pg), db, id_o, 1u);
+            }
+            tc_commit(att_smem_u32(&ctl->vempty[st]));
+            tc_commit(att_smem_u32(&ctl->o_done));
+          }
+        }
+        it += n;
+        t += n;
+        ++seg;
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------ softmax: one thread per query-row slot ------------------------------
+    const int sl = 32 * (warp & 3) + lane;                  // TMEM lane == query-row slot
+    const int q = 4 * (sl & 31) + (sl >> 5);                // the query row of this slot (inverse of t5_lane_of_row)
+    const bool active = q < nq;
+    const uint32_t lane_addr = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+    int it = 0, seg = 0;
+    long long t = t_lo;
+    bool alive = true;
+    while (t < t_hi && alive) {
+      const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
+      const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+      // queries of this (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16 terms
+      if (active) {
+        const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD;
+        const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD : nullptr;
+        for (int d = 0; d < HD; d += 8) {
+          const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(qh + d));
+          uint4 rawl = make_uint4(0, 0, 0, 0);
+          if (ql) rawl = __ldcg(reinterpret_cast<const uint4*>(ql + d));
+          const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+          const __half2* l2 = reinterpret_cast<const __half2*>(&rawl);
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float2 v = __half22float2(h2[e]);
+            const float2 vl = __half22float2(l2[e]);
+            v.x += vl.x; v.y += vl.y;
+            const __nv_bfloat162 bh = __floats2bfloat162_rn(v.x, v.y);
+            const float2 back = __bfloat1622float2(bh);
+            const __nv_bfloat162 bl = __floats2bfloat162_rn(v.x - back.x, v.y - back.y);
+            hi[e] = *reinterpret_cast<const uint32_t*>(&bh);
+            lo[e] = *reinterpret_cast<const uint32_t*>(&bl);
+          }
+          *reinterpret_cast<uint4*>(sQ + t5_q_off(sl, d)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(sQ + kT5TileBytes + t5_q_off(sl, d)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read these generic-proxy stores
+      att_mbar_arrive(att_smem_u32(&ctl->q_ready));
+      float m_used = -INFINITY, l_sum = 0.f;
+      for (int i = 0; i < n && alive; ++i) {
+        const int g = it + i, sb = g & 1;
+        int ok = 1;
+        if (lane == 0) ok = t5_wait(&ctl->s_full[sb], (uint32_t)(g >> 1) & 1u, ctl, w.status, 7) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) { alive = false; break; }
+        att_mbar_try(att_smem_u32(&ctl->s_full[sb]), (uint32_t)(g >> 1) & 1u);   // every lane observes the completed phase
+        tc_fence_after();
+        const uint32_t s_addr = lane_addr + (uint32_t)(sb * 128);
+        const int key0 = (x.ti + i) * kT5Keys, n_valid = min(kT5Keys, x.L - key0);   // keys >= L are masked
+        // pass 1: the row maximum
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c0 = 0; c0 < kT5Keys; c0 += 32) {
+          float s[32];
+          tc_ld32(s_addr + c0, s);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, (c0 + j < n_valid) ? s[j] : -INFINITY);
+        }
+        // the stabiliser only moves when the maximum outgrows it by more than 8 (p stays below 256)
+        float m_new = m_used, f = 1.f;
+        if (m_used == -INFINITY) m_new = mx;
+        else if (mx > m_used + 8.f) { m_new = mx; f = exp2f(m_used - m_new); }
+        if (i > 0) {   // P and O may be touched once the previous tile's P V has completed
+          if (lane == 0) ok = t5_wait(&ctl->o_done, (uint32_t)(g - 1) & 1u, ctl, w.status, 8) ? 1 : 0;
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) { alive = false; break; }
+          att_mbar_try(att_smem_u32(&ctl->o_done), (uint32_t)(g - 1) & 1u);
+          tc_fence_after();
+          if (__any_sync(0xffffffffu, f != 1.f)) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+              float o[32];
+              tc_ld32(lane_addr + 384 + c0, o);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) o[j] *= f;
+              tc_st32f(lane_addr + 384 + c0, o);
+            }
+            l_sum *= f;
+          }
+        }
+        // pass 2: probabilities as two bf16 terms
+#pragma unroll 1
+        for (int c0 = 0; c0 < kT5Keys; c0 += 32) {
+          float s[32];
+          tc_ld32(s_addr + c0, s);
+          uint32_t hi[16], lo[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = (c0 + j < n_valid) ? exp2f(s[j] - m_new) : 0.f;
+            const float p1 = (c0 + j + 1 < n_valid) ? exp2f(s[j + 1] - m_new) : 0.f;
+            l_sum += p0 + p1;
+            const __nv_bfloat162 bh = __floats2bfloat162_rn(p0, p1);
+            const float2 back = __bfloat1622float2(bh);
+            const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - back.x, p1 - back.y);
+            hi[j >> 1] = *reinterpret_cast<const uint32_t*>(&bh);
+            lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&bl);
+          }
+          tc_st16(lane_addr + 256 + (uint32_t)(c0 >> 1), hi);
+          tc_st16(lane_addr + 320 + (uint32_t)(c0 >> 1), lo);
+        }
+        tc_wait_st();
+        tc_fence_before();
+        att_mbar_arrive(att_smem_u32(&ctl->p_full));
+        att_mbar_arrive(att_smem_u32(&ctl->s_free[sb]));
+        m_used = m_new;
+      }
+      if (!alive) break;
+      // the segment's partial: wait for the last P V, then (m, l, o) of every real query row
+      {
+        const int g = it + n - 1;
+        int ok = 1;
+        if (lane == 0) ok = t5_wait(&ctl->o_done, (uint32_t)g & 1u, ctl, w.status, 9) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        att_mbar_try(att_smem_u32(&ctl->o_done), (uint32_t)g & 1u);
+        tc_fence_after();
+        const size_t base = (((size_t)c + (size_t)x.b * Hkv + x.h) * kAttMaxSub + 0) * (size_t)nq;
+        if (active) { a.P.m[base + q] = m_used; a.P.l[base + q] = l_sum; }
+#pragma unroll 1
+        for (int c0 = 0; c0 < HD; c0 += 32) {
+          float o[32];
+          tc_ld32(lane_addr + 384 + c0, o);
+          if (active) {
+            float4* dst = reinterpret_cast<float4*>(a.P.o + (base + q) * HD + c0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+          }
+        }
+        tc_fence_before();
+      }
+      it += n;
+      t += n;
+      ++seg;
+    }
+  } else {
+    // ------------------------------ tails: the block's own rows, one m-tile of one (sequence, KV head) per task ------------------------------
+    const AttGeom g = att_geom(HD, group, rows);
+    AttWarp<HD, 2> st;
+    for (int task = (G - 1 - c) * 2 + (warp - 6); task < B * Hkv * g.MT; task += G * 2)
+      att_tail_task<HD, 2>(st, g, a, task / g.MT, (task % g.MT) * 16, lane);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    if (*abort_flag) __nanosleep(20000);   // let copies in flight land before the block retires
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+}  // namespace sj

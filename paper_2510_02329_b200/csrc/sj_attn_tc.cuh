@@ -818,14 +818,17 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
   for (int i = 0; i < DPL; ++i) store_act<T>(ATT, R, Hq * HD, r, head * HD + (part * 32 + lane) * DPL + i, acc[i] * inv);
 }
 
+// keys_per_tile > 0: the partials come from a pass that cut the cache into tiles of that many keys with one
+// sub-partial per block segment (the tcgen05 attention); 0: this file's own geometry.
 template <int HD>
 __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dims dm, AttPartials P, int G_att,
-                                  int n_tail_base) {
+                                  int n_tail_base, int keys_per_tile) {
   __shared__ AttPlan pl;
   pdl_wait();
   pdl_launch();
   const int B = args->B, rows = args->gamma + 1;
-  const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+  AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+  if (keys_per_tile > 0) { g.KPS = keys_per_tile; g.KS = 1; g.KW = keys_per_tile; }
   if (threadIdx.x == 0) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS);
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;

@@ -104,8 +104,9 @@ def test_ragged_batches_and_page_edges(dtype, options, kv_lens, gamma):
         case.close()
 
 
-@pytest.mark.parametrize("options", [{"gemm_impl": 0}, {"gemm_impl": 1, "step_impl": 0}, {"gemm_impl": 1, "step_impl": 1}],
-                         ids=["cudacore", "tcgen05", "persistent"])
+@pytest.mark.parametrize("options", [{"gemm_impl": 0}, {"gemm_impl": 1, "step_impl": 0}, {"gemm_impl": 1, "step_impl": 1},
+                                     {"gemm_impl": 1, "step_impl": 0, "attn_impl": 2}],
+                         ids=["cudacore", "tcgen05", "persistent", "tcgen05-attention"])
 def test_head_dim_128_with_qkv_bias(options):
     case = harness.Case(GQA128, torch.bfloat16, [70, 300], 8, seed=4).gpu_setup()
     try:
@@ -348,6 +349,32 @@ def test_full_size_benchmark_workloads(name, key, thetas):
                 assert rep.exact + rep.margin == len(kv_lens)
                 print(name, "mode", mode, "theta", theta, "margin positions", rep.margin, "of", rep.sequences,
                       "mean accepted length %.2f" % float(np.mean(g["accepted_len"])), rep)
+    finally:
+        case.close()
+
+
+T5_CASES = [
+    ("gqa128-ragged", GQA128, [70, 300, 1, 128, 129, 0, 2047], 8),     # tile edges: 1, 128, 129 keys; an empty cache
+    ("llama-8b-cut2", synth.LLAMA_8B.cut(2), [210, 4096], 8),          # config 3 / 4 widths: group 4, 36 query rows
+    ("llama-8b-cut1-g16", synth.LLAMA_8B.cut(1), [777], 16),           # 68 query rows
+    ("qwen-32b-cut1", synth.QWEN_32B.cut(1), [40, 1300, 515], 8),      # group 5, qkv bias
+]
+
+
+@pytest.mark.parametrize("name,shape,kv_lens,gamma", T5_CASES, ids=[c[0] for c in T5_CASES])
+def test_tcgen05_attention(name, shape, kv_lens, gamma):
+    """The attention of the multi-kernel path on tcgen05 (scores in tensor memory), against the oracle and against
+    the mma.sync attention on the same inputs."""
+    cache = "prefill" if shape is GQA128 else "fill"
+    case = harness.Case(shape, torch.bfloat16, kv_lens, gamma, seed=8, cache=cache,
+                        gen_device="cpu" if shape is GQA128 else "cuda").gpu_setup(max_rows=len(kv_lens) * (gamma + 1))
+    try:
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 1.0)]:
+            rep, g = _run(case, mode, T, options={"gemm_impl": 1, "step_impl": 0, "attn_impl": 2})
+            assert rep.exact + rep.margin == len(kv_lens)
+            rep1, g1 = _run(case, mode, T, options={"gemm_impl": 1, "step_impl": 0, "attn_impl": 1})
+            assert np.abs(g["hidden"] - g1["hidden"]).max() < 5e-3
+            print(name, "mode", mode, rep)
     finally:
         case.close()
 
