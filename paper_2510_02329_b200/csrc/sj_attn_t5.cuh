@@ -9,10 +9,11 @@
 //               N = 128 keys, K = head dim: Q from shared memory (K-major), the key tile as a K-major B operand.
 //               The cache is bf16, and both operands of an MMA have one type, so a query enters as the sum of two
 //               bf16 terms (hi + lo, 16 significant bits): two MMAs per 16-dim step into the same accumulator.
-//   softmax     one thread per query-row slot reads its row of S from tensor memory (no cross-lane traffic),
-//               keeps a stabiliser m (raised only when the row maximum exceeds it by more than 8 in the log2
-//               domain: then the thread rescales its row of O), and writes P = exp2(S - m) back to tensor memory
-//               as two bf16 terms.
+//   softmax     one thread per query-row slot reads its row of S from tensor memory into registers (no cross-lane
+//               traffic), keeps a stabiliser m (raised only when the row maximum exceeds it by more than 8 in the
+//               log2 domain: then the thread rescales its row of O), and writes P = exp2(S - m) over the scores it
+//               has just read, as two bf16 terms per 32-key chunk ([hi 16 columns | lo 16 columns]).  S is double-
+//               buffered, so the next tile's scores are computed while this tile's P V runs.
 //   O += P V    A = P from tensor memory (M = 128 slots, K = 16 keys per step = one page), B = the page's V rows
 //               as an MN-major operand (the head dim is the contiguous one: leading byte offset = the 16 KiB
 //               between the two halves, stride byte offset = the 1 KiB between 8-key groups), N = head dim.
@@ -20,8 +21,9 @@
 // per query row, in the format of sj_attn_tc.cuh, whose combine pass merges them; the block's own gamma+1 rows
 // (the causal tail) are handled by two extra warps with that file's mma.sync routine.
 //
-// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer (owns tensor memory: S twice, P, O = 512
-// columns), warps 2..5 softmax (TMEM lane quarter = warp % 4), warps 6..7 tails.  Every wait is bounded.
+// Roles (384 threads): warps 0 and 11 TMA producers (keys, values), warp 1 MMA issuer (owns tensor memory: S twice,
+// O = 384 of the 512 columns it allocates), warps 2..9 softmax (two threads per query row, TMEM lane quarter =
+// warp % 4), warp 10 tails.  Every wait is bounded.
 #pragma once
 
 #include "sj_attn_tc.cuh"
@@ -30,14 +32,15 @@
 namespace sj {
 
 constexpr int kT5Keys = 128;               // keys per tile
-constexpr int kT5Threads = 256;
+constexpr int kT5Threads = 384;
 constexpr int kT5TileBytes = 32768;        // one K or V tile: 2 halves x 8 pages x 2 KiB
 constexpr int kT5SmemBytes = 2 * kT5TileBytes /* Q hi, lo */ + 4 * kT5TileBytes /* K, V double-buffered */;
 
 struct T5Ctl {
-  uint64_t kfull[2], kempty[2], vfull[2], vempty[2], s_full[2], s_free[2], p_full, o_done, q_ready;
+  uint64_t kfull[2], kempty[2], vfull[2], vempty[2], s_full[2], p_full[2], o_done[2], q_ready;
   uint32_t tmem_base;
   int abort_flag;
+  float mx[2][2][128];   // [tile parity][key half][query-row slot]: row maxima (and, at a segment's end, sums) of the two threads of a row
   AttPlan plan;
   int pages[kAttPageCache];
 };
@@ -56,6 +59,17 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tc_ld32_nowait(uint32_t taddr, float* v) {   // results valid after tc_wait_ld()
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,"
+      "%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7]), "=f"(v[8]), "=f"(v[9]),
+        "=f"(v[10]), "=f"(v[11]), "=f"(v[12]), "=f"(v[13]), "=f"(v[14]), "=f"(v[15]), "=f"(v[16]), "=f"(v[17]), "=f"(v[18]),
+        "=f"(v[19]), "=f"(v[20]), "=f"(v[21]), "=f"(v[22]), "=f"(v[23]), "=f"(v[24]), "=f"(v[25]), "=f"(v[26]), "=f"(v[27]),
+        "=f"(v[28]), "=f"(v[29]), "=f"(v[30]), "=f"(v[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
@@ -95,6 +109,12 @@ __device__ __forceinline__ uint32_t t5_q_off(int row, int dim) {
 // TMEM lane of query row q: the rows are dealt round-robin to the four lane quarters (one softmax warp each)
 __device__ __forceinline__ int t5_lane_of_row(int q) { return 32 * (q & 3) + (q >> 2); }
 
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void bar_sync_n(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ bool t5_wait(uint64_t* bar, uint32_t parity, T5Ctl* ctl, int* status, int where) {
   return att_mbar_wait(att_smem_u32(bar), parity, &ctl->abort_flag, status, nullptr, where, 0);
 }
@@ -118,11 +138,10 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       att_mbar_init(att_smem_u32(&ctl->vfull[i]), 1);
       att_mbar_init(att_smem_u32(&ctl->vempty[i]), 1);
       att_mbar_init(att_smem_u32(&ctl->s_full[i]), 1);
-      att_mbar_init(att_smem_u32(&ctl->s_free[i]), 128);
+      att_mbar_init(att_smem_u32(&ctl->p_full[i]), 256);
+      att_mbar_init(att_smem_u32(&ctl->o_done[i]), 1);
     }
-    att_mbar_init(att_smem_u32(&ctl->p_full), 128);
-    att_mbar_init(att_smem_u32(&ctl->o_done), 1);
-    att_mbar_init(att_smem_u32(&ctl->q_ready), 128);
+    att_mbar_init(att_smem_u32(&ctl->q_ready), 256);
     ctl->abort_flag = 0;
     att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, kT5Keys);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -141,39 +160,37 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
   const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
   att_fill_pages(ctl->pages, pl, kv, args, B, kT5Keys, t_lo, t_hi, threadIdx.x, blockDim.x);
   __syncthreads();
-  const uint32_t tmem = ctl->tmem_base;   // columns: [0,256) S twice, [256,384) P (hi 64, lo 64), [384,512) O
+  const uint32_t tmem = ctl->tmem_base;   // columns: [0,256) S twice (P overwrites S in place), [256,384) O
   volatile int* abort_flag = &ctl->abort_flag;
 
-  if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
+  if (warp == 0 || warp == 11) {
+    // ------------------------------ TMA producers: warp 0 the key tiles, warp 11 the value tiles ------------------------------
+    // (two threads, so that the key tiles, which the scores need first, never queue behind a value stage that is
+    // still waiting for its P V)
     if (lane == 0) {
+      const int which = warp == 0 ? 0 : 1;
+      uint64_t* full = which ? ctl->vfull : ctl->kfull;
+      uint64_t* empty = which ? ctl->vempty : ctl->kempty;
+      uint8_t* base = which ? sV : sK;
       int g = 0;
       for (long long t = t_lo; t < t_hi; ++t, ++g) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
         const int st = g & 1, seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
-        int page[8];
+        if (g >= 2 && !t5_wait(&empty[st], (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 1)) break;
+        const uint32_t bar = att_smem_u32(&full[st]);
+        const uint32_t dst = att_smem_u32(base + (size_t)st * kT5TileBytes);
+        att_mbar_expect_tx(bar, kT5TileBytes);
         for (int p = 0; p < 8; ++p) {
           int pi = x.ti * 8 + p;
           if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
-          page[p] = (g + 1) * 8 <= kAttPageCache ? ctl->pages[g * 8 + p]
-                                                 : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
-        }
-        for (int which = 0; which < 2; ++which) {   // the key tile, then the value tile
-          uint64_t* full = which ? &ctl->vfull[st] : &ctl->kfull[st];
-          uint64_t* empty = which ? &ctl->vempty[st] : &ctl->kempty[st];
-          if (g >= 2 && !t5_wait(empty, (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 1)) goto producer_done;
-          const uint32_t bar = att_smem_u32(full);
-          const uint32_t dst = att_smem_u32((which ? sV : sK) + (size_t)st * kT5TileBytes);
-          att_mbar_expect_tx(bar, kT5TileBytes);
-          for (int p = 0; p < 8; ++p) {
-            const long long row = ((((long long)a.layer * kv.n_pages + page[p]) * 2 + which) * kv.n_kv_heads + x.h) * 16;
-            att_tma_2d(dst + (uint32_t)(p * 2048), &tmKV, bar, 0, (int)row);
-            att_tma_2d(dst + 16384u + (uint32_t)(p * 2048), &tmKV, bar, 64, (int)row);
-          }
+          const int page = (g + 1) * 8 <= kAttPageCache ? ctl->pages[g * 8 + p]
+                                                        : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+          const long long row = ((((long long)a.layer * kv.n_pages + page) * 2 + which) * kv.n_kv_heads + x.h) * 16;
+          att_tma_2d(dst + (uint32_t)(p * 2048), &tmKV, bar, 0, (int)row);
+          att_tma_2d(dst + 16384u + (uint32_t)(p * 2048), &tmKV, bar, 64, (int)row);
         }
       }
     }
-  producer_done:;
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0) {
@@ -182,17 +199,31 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       int it = 0, seg = 0;
       long long t = t_lo;
       bool alive = true;
+#ifdef SJ_T5_PROF
+      long long pc_k = 0, pc_p = 0, pc_v = 0, pc_iss = 0, pc_q = 0, pc_t0 = clock64(), pc_x;
+#define T5P(acc, stmt) pc_x = clock64(); stmt; acc += clock64() - pc_x;
+#else
+#define T5P(acc, stmt) stmt;
+#endif
       while (t < t_hi && alive) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
         const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-        if (!t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2)) break;
+        bool okq;
+        T5P(pc_q, okq = t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2))
+        if (!okq) break;
         tc_fence_after();
         for (int i = 0; i <= n && alive; ++i) {
           if (i < n) {   // scores of tile i
             const int g = it + i, st = g & 1;
-            if (!t5_wait(&ctl->kfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 3) ||
-                (g >= 2 && !t5_wait(&ctl->s_free[st], (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 4))) { alive = false; break; }
+            // S buffer `st` still holds P of tile g - 2 for that tile's P V, which this thread issued earlier: the
+            // tensor pipe executes one thread's MMAs in issue order, so these may overwrite it
+            bool okk;
+            T5P(pc_k, okk = t5_wait(&ctl->kfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 3))
+            if (!okk) { alive = false; break; }
             tc_fence_after();
+#ifdef SJ_T5_PROF
+            pc_x = clock64();
+#endif
             const uint32_t kb = k0 + (uint32_t)st * kT5TileBytes, d_s = tmem + (uint32_t)(st * 128);
 #pragma unroll
             for (int k = 0; k < HD / 16; ++k) {
@@ -203,45 +234,67 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
             }
             tc_commit(att_smem_u32(&ctl->kempty[st]));
             tc_commit(att_smem_u32(&ctl->s_full[st]));
+#ifdef SJ_T5_PROF
+            pc_iss += clock64() - pc_x;
+#endif
           }
           if (i >= 1) {  // output of tile i - 1
             const int g = it + i - 1, st = g & 1;
-            if (!t5_wait(&ctl->p_full, (uint32_t)g & 1u, ctl, w.status, 5) ||
-                !t5_wait(&ctl->vfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 6)) { alive = false; break; }
+            bool okp, okv;
+            T5P(pc_p, okp = t5_wait(&ctl->p_full[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 5))
+            T5P(pc_v, okv = okp && t5_wait(&ctl->vfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 6))
+            if (!okv) { alive = false; break; }
             tc_fence_after();
-            const uint32_t vb = v0 + (uint32_t)st * kT5TileBytes;
+#ifdef SJ_T5_PROF
+            pc_x = clock64();
+#endif
+            const uint32_t vb = v0 + (uint32_t)st * kT5TileBytes, pb = tmem + (uint32_t)(st * 128);
 #pragma unroll
-            for (int pg = 0; pg < 8; ++pg) {
+            for (int pg = 0; pg < 8; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
               const uint64_t db = smem_desc_mn_sw128(vb + (uint32_t)(pg * 2048), 16384u);
-              tc_mma_bf16_ta(tmem + 384, tmem + 256 + (uint32_t)(8 * pg), db, id_o, (i > 1 || pg > 0) ? 1u : 0u);
-              tc_mma_bf16_ta(tmem + 384, tmem + 320 + (uint32_t)(8 * pg), db, id_o, 1u);
+              const uint32_t pa = pb + (uint32_t)(32 * (pg >> 1) + 8 * (pg & 1));
+              tc_mma_bf16_ta(tmem + 256, pa, db, id_o, (i > 1 || pg > 0) ? 1u : 0u);
+              tc_mma_bf16_ta(tmem + 256, pa + 16, db, id_o, 1u);
             }
             tc_commit(att_smem_u32(&ctl->vempty[st]));
-            tc_commit(att_smem_u32(&ctl->o_done));
+            tc_commit(att_smem_u32(&ctl->o_done[st]));
+#ifdef SJ_T5_PROF
+            pc_iss += clock64() - pc_x;
+#endif
           }
         }
         it += n;
         t += n;
         ++seg;
       }
+#ifdef SJ_T5_PROF
+      if (c == 0 && a.layer == 1) printf("t5 mma thread: tiles %d total %lld clk: wait q %lld, k %lld, p %lld, v %lld, issue %lld\n", it, clock64() - pc_t0, pc_q, pc_k, pc_p, pc_v, pc_iss);
+#endif
+#undef T5P
     }
-  } else if (warp < 6) {
-    // ------------------------------ softmax: one thread per query-row slot ------------------------------
-    const int sl = 32 * (warp & 3) + lane;                  // TMEM lane == query-row slot
+  } else if (warp < 10) {
+    // ------------------------------ softmax: two threads per query-row slot, 64 keys each ------------------------------
+    // warps 2..5 take keys [0, 64) of every tile, warps 6..9 keys [64, 128); warp w reads TMEM lane quarter w % 4, so
+    // warps w and w + 4 share a quarter: they exchange their row maxima through shared memory (named barrier of
+    // their 64 threads) and keep separate sums, which are added when the segment's partial is written.
+    const int half = (warp - 2) >> 2, quarter = warp & 3;
+    const int sl = 32 * quarter + lane;                     // TMEM lane == query-row slot
     const int q = 4 * (sl & 31) + (sl >> 5);                // the query row of this slot (inverse of t5_lane_of_row)
     const bool active = q < nq;
-    const uint32_t lane_addr = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)(32 * quarter) << 16);
+    const int pair_bar = 1 + quarter;
     int it = 0, seg = 0;
     long long t = t_lo;
     bool alive = true;
     while (t < t_hi && alive) {
       const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
       const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-      // queries of this (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16 terms
+      // queries of this (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16
+      // terms; this thread converts its half of the head dimension
       if (active) {
         const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD;
         const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD : nullptr;
-        for (int d = 0; d < HD; d += 8) {
+        for (int d = 64 * half; d < 64 * half + 64; d += 8) {
           const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(qh + d));
           uint4 rawl = make_uint4(0, 0, 0, 0);
           if (ql) rawl = __ldcg(reinterpret_cast<const uint4*>(ql + d));
@@ -274,63 +327,68 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         if (!ok) { alive = false; break; }
         att_mbar_try(att_smem_u32(&ctl->s_full[sb]), (uint32_t)(g >> 1) & 1u);   // every lane observes the completed phase
         tc_fence_after();
-        const uint32_t s_addr = lane_addr + (uint32_t)(sb * 128);
-        const int key0 = (x.ti + i) * kT5Keys, n_valid = min(kT5Keys, x.L - key0);   // keys >= L are masked
-        // pass 1: the row maximum
+        const uint32_t s_addr = lane_addr + (uint32_t)(sb * 128 + 64 * half);
+        const int n_valid = min(kT5Keys, x.L - (x.ti + i) * kT5Keys) - 64 * half;   // this thread's keys >= n_valid are masked
+        float sc[64];
+        tc_ld32_nowait(s_addr, sc);
+        tc_ld32_nowait(s_addr + 32, sc + 32);
+        tc_wait_ld();
         float mx = -INFINITY;
-#pragma unroll 1
-        for (int c0 = 0; c0 < kT5Keys; c0 += 32) {
-          float s[32];
-          tc_ld32(s_addr + c0, s);
+        if (n_valid >= 64) {   // warp-uniform; every tile but a sequence's last
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, (c0 + j < n_valid) ? s[j] : -INFINITY);
+          for (int j = 0; j < 64; ++j) mx = fmaxf(mx, sc[j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 64; ++j) {
+            sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
+            mx = fmaxf(mx, sc[j]);
+          }
         }
+        ctl->mx[g & 1][half][sl] = mx;
+        bar_sync_n(pair_bar, 64);
+        mx = fmaxf(mx, ctl->mx[g & 1][half ^ 1][sl]);
         // the stabiliser only moves when the maximum outgrows it by more than 8 (p stays below 256)
         float m_new = m_used, f = 1.f;
         if (m_used == -INFINITY) m_new = mx;
-        else if (mx > m_used + 8.f) { m_new = mx; f = exp2f(m_used - m_new); }
-        if (i > 0) {   // P and O may be touched once the previous tile's P V has completed
-          if (lane == 0) ok = t5_wait(&ctl->o_done, (uint32_t)(g - 1) & 1u, ctl, w.status, 8) ? 1 : 0;
+        else if (mx > m_used + 8.f) { m_new = mx; f = ex2_approx(m_used - m_new); }
+        if (i > 0 && __any_sync(0xffffffffu, f != 1.f)) {
+          // rescale this thread's half of its row of O: only once the previous tile's P V has completed (this
+          // tile's cannot start before every thread has delivered its P)
+          if (lane == 0) ok = t5_wait(&ctl->o_done[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, ctl, w.status, 8) ? 1 : 0;
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) { alive = false; break; }
-          att_mbar_try(att_smem_u32(&ctl->o_done), (uint32_t)(g - 1) & 1u);
+          att_mbar_try(att_smem_u32(&ctl->o_done[(g - 1) & 1]), (uint32_t)((g - 1) >> 1) & 1u);
           tc_fence_after();
-          if (__any_sync(0xffffffffu, f != 1.f)) {
 #pragma unroll 1
-            for (int c0 = 0; c0 < HD; c0 += 32) {
-              float o[32];
-              tc_ld32(lane_addr + 384 + c0, o);
+          for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+            float o[32];
+            tc_ld32(lane_addr + 256 + c0, o);
 #pragma unroll
-              for (int j = 0; j < 32; ++j) o[j] *= f;
-              tc_st32f(lane_addr + 384 + c0, o);
-            }
-            l_sum *= f;
+            for (int j = 0; j < 32; ++j) o[j] *= f;
+            tc_st32f(lane_addr + 256 + c0, o);
           }
+          l_sum *= f;
         }
-        // pass 2: probabilities as two bf16 terms
-#pragma unroll 1
-        for (int c0 = 0; c0 < kT5Keys; c0 += 32) {
-          float s[32];
-          tc_ld32(s_addr + c0, s);
+        // probabilities as two bf16 terms, written over the scores: chunk of 32 keys -> [hi 16 columns | lo 16 columns];
+        // hi = p truncated to bf16, lo = the rest rounded to bf16 (16 significant bits in all)
+#pragma unroll
+        for (int c0 = 0; c0 < 64; c0 += 32) {
           uint32_t hi[16], lo[16];
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
-            const float p0 = (c0 + j < n_valid) ? exp2f(s[j] - m_new) : 0.f;
-            const float p1 = (c0 + j + 1 < n_valid) ? exp2f(s[j + 1] - m_new) : 0.f;
+            const float p0 = ex2_approx(sc[c0 + j] - m_new), p1 = ex2_approx(sc[c0 + j + 1] - m_new);   // 0 for masked keys
             l_sum += p0 + p1;
-            const __nv_bfloat162 bh = __floats2bfloat162_rn(p0, p1);
-            const float2 back = __bfloat1622float2(bh);
-            const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - back.x, p1 - back.y);
-            hi[j >> 1] = *reinterpret_cast<const uint32_t*>(&bh);
+            const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+            hi[j >> 1] = __byte_perm(b0, b1, 0x7632);
+            const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - __uint_as_float(b0 & 0xffff0000u), p1 - __uint_as_float(b1 & 0xffff0000u));
             lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&bl);
           }
-          tc_st16(lane_addr + 256 + (uint32_t)(c0 >> 1), hi);
-          tc_st16(lane_addr + 320 + (uint32_t)(c0 >> 1), lo);
+          tc_st16(s_addr + (uint32_t)c0, hi);
+          tc_st16(s_addr + (uint32_t)c0 + 16, lo);
         }
         tc_wait_st();
         tc_fence_before();
-        att_mbar_arrive(att_smem_u32(&ctl->p_full));
-        att_mbar_arrive(att_smem_u32(&ctl->s_free[sb]));
+        att_mbar_arrive(att_smem_u32(&ctl->p_full[sb]));
         m_used = m_new;
       }
       if (!alive) break;
@@ -338,17 +396,20 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       {
         const int g = it + n - 1;
         int ok = 1;
-        if (lane == 0) ok = t5_wait(&ctl->o_done, (uint32_t)g & 1u, ctl, w.status, 9) ? 1 : 0;
+        if (lane == 0) ok = t5_wait(&ctl->o_done[g & 1], (uint32_t)(g >> 1) & 1u, ctl, w.status, 9) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        att_mbar_try(att_smem_u32(&ctl->o_done), (uint32_t)g & 1u);
+        att_mbar_try(att_smem_u32(&ctl->o_done[g & 1]), (uint32_t)(g >> 1) & 1u);
         tc_fence_after();
+        ctl->mx[(g + 1) & 1][half][sl] = l_sum;           // the buffer the last tile did not use
+        bar_sync_n(pair_bar, 64);
+        const float l_tot = l_sum + ctl->mx[(g + 1) & 1][half ^ 1][sl];
         const size_t base = (((size_t)c + (size_t)x.b * Hkv + x.h) * kAttMaxSub + 0) * (size_t)nq;
-        if (active) { a.P.m[base + q] = m_used; a.P.l[base + q] = l_sum; }
+        if (active && half == 0) { a.P.m[base + q] = m_used; a.P.l[base + q] = l_tot; }
 #pragma unroll 1
-        for (int c0 = 0; c0 < HD; c0 += 32) {
+        for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
           float o[32];
-          tc_ld32(lane_addr + 384 + c0, o);
+          tc_ld32(lane_addr + 256 + c0, o);
           if (active) {
             float4* dst = reinterpret_cast<float4*>(a.P.o + (base + q) * HD + c0);
 #pragma unroll
@@ -356,16 +417,17 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
           }
         }
         tc_fence_before();
+        bar_sync_n(pair_bar, 64);   // the sums have been read before the next segment's first tile reuses the buffer
       }
       it += n;
       t += n;
       ++seg;
     }
-  } else {
+  } else if (warp < 11) {
     // ------------------------------ tails: the block's own rows, one m-tile of one (sequence, KV head) per task ------------------------------
     const AttGeom g = att_geom(HD, group, rows);
     AttWarp<HD, 2> st;
-    for (int task = (G - 1 - c) * 2 + (warp - 6); task < B * Hkv * g.MT; task += G * 2)
+    for (int task = G - 1 - c; task < B * Hkv * g.MT; task += G)
       att_tail_task<HD, 2>(st, g, a, task / g.MT, (task % g.MT) * 16, lane);
   }
   tc_fence_before();
