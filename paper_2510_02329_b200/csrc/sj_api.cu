@@ -210,7 +210,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_att_precise = 1;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_att_precise = 1, opt_a5_min_tiles = 8;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -300,13 +300,17 @@ static bool tc_shapes_ok(const sj_model_config& c) {
 
 typedef void (*MegaKernel)(const MegaMaps, const MegaParams, const StepArgs*, const KvView, const Work, const Dims);
 // The persistent kernel for a head dimension (64 or 128), a number of row slots (4, 6 or 8), with or without
-// the timeline code.
-template <bool TR>
+// the timeline code, with the mma.sync or (head dimension 128 only) the tcgen05 attention phase.
+template <bool TR, bool A5>
 static MegaKernel mega_kernel_t(int hd, int ns) {
-  if (hd == 128) return ns == 4 ? k_verify_mega<128, 4, TR> : (ns == 6 ? k_verify_mega<128, 6, TR> : k_verify_mega<128, 8, TR>);
-  return ns == 4 ? k_verify_mega<64, 4, TR> : (ns == 6 ? k_verify_mega<64, 6, TR> : k_verify_mega<64, 8, TR>);
+  if (hd == 128)
+    return ns == 4 ? k_verify_mega<128, 4, TR, A5> : (ns == 6 ? k_verify_mega<128, 6, TR, A5> : k_verify_mega<128, 8, TR, A5>);
+  return ns == 4 ? k_verify_mega<64, 4, TR, false> : (ns == 6 ? k_verify_mega<64, 6, TR, false> : k_verify_mega<64, 8, TR, false>);
 }
-static MegaKernel mega_kernel(int hd, int ns, bool trace) { return trace ? mega_kernel_t<true>(hd, ns) : mega_kernel_t<false>(hd, ns); }
+static MegaKernel mega_kernel(int hd, int ns, bool trace, bool a5) {
+  if (a5) return trace ? mega_kernel_t<true, true>(hd, ns) : mega_kernel_t<false, true>(hd, ns);
+  return trace ? mega_kernel_t<true, false>(hd, ns) : mega_kernel_t<false, false>(hd, ns);
+}
 
 extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weights* w, void* cuda_stream,
                                       sj_target** out) {
@@ -361,7 +365,7 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
   }
   const bool tc = tc_shapes_ok(c);
   t->opt_gemm = tc ? 1 : 0;
-  t->opt_attn = t->bf ? 1 : 0;
+  t->opt_attn = t->bf ? (c.head_dim == 128 ? 2 : 1) : 0;
   t->opt_graph = t->stream ? 1 : 0;  // the legacy default stream cannot be captured
 
   sj_status st = SJ_OK;
@@ -464,8 +468,9 @@ extern "C" sj_status sj_create_target(const sj_model_config* cfg, const sj_weigh
     if (e == cudaSuccess) e = cudaMemset(t->d_sumsq, 0, sizeof(float) * 2 * (c.d_model / kTileN) * kMegaMaxRows);
     if (e == cudaSuccess) e = cudaMemset(t->d_sync, 0, sizeof(unsigned) * (64 + (size_t)4 * t->sm_count * pad16(Rm) * kTileN));
     for (int ns = 4; ns <= 8 && e == cudaSuccess; ns += 2)
-      for (int tr = 0; tr < 2 && e == cudaSuccess; ++tr)
-        e = cudaFuncSetAttribute(mega_kernel(c.head_dim, ns, tr != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+      for (int v = 0; v < 4 && e == cudaSuccess; ++v)
+        e = cudaFuncSetAttribute(mega_kernel(c.head_dim, ns, (v & 1) != 0, (v & 2) != 0 && c.head_dim == 128),
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) { fail(SJ_ERR_CUDA, "whole-step kernel set-up: %s", cudaGetErrorString(e)); return bail(SJ_ERR_CUDA); }
     for (int l0 = 0; l0 < c.n_layers; l0 += kMegaMaxLayers) {
       t->mega_maps.emplace_back();
@@ -548,6 +553,9 @@ extern "C" sj_status sj_set_option(sj_target* t, const char* name, int value) {
   } else if (n == "ring_stages") {
     if (value != 0 && (value < 3 || value > kMegaMaxStages)) return fail(SJ_ERR_INVALID_ARG, "ring_stages must be 0 (auto) or 3..%d", kMegaMaxStages);
     t->opt_ring = value;
+  } else if (n == "attn_tcgen05_min_tiles") {
+    if (value < 0) return fail(SJ_ERR_INVALID_ARG, "attn_tcgen05_min_tiles must be >= 0");
+    t->opt_a5_min_tiles = value;
   } else if (n == "attn_two_term_layers") {
     if (value < 0) return fail(SJ_ERR_INVALID_ARG, "attn_two_term_layers must be >= 0");
     cudaStreamSynchronize(t->stream);
@@ -973,8 +981,9 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
       AttArgs aa{W.Qb, l < t->opt_att_precise ? W.Qlo : nullptr, W.KVn, AttPartials{W.tc_m, W.tc_l, W.tc_o}, t->sm_count + B * dm.Hkv, l};
       const size_t tc_smem = kAttStages * kAttStageBytes + sizeof(AttSmemCtl) + 1024;
       const AttPartials parts{W.tc_m, W.tc_l, W.tc_o};
-      const int items = B * dm.Hkv * nq, cgrid = std::max(1, std::min(4 * t->sm_count, (items + 7) / 8));
-      if (dm.hd == 128 && t->opt_attn == 2) {
+      // one warp per (sequence, KV head, query row, half of the head dimension): every task's loads are in flight at once
+      const int items = B * dm.Hkv * nq, cgrid = std::max(1, std::min(32 * t->sm_count, (items * (dm.hd >= 128 ? 2 : 1) + 7) / 8));
+      if (dm.hd == 128 && t->opt_attn == 2 && nq <= 128) {   // one 128-lane accumulator holds a KV head's query rows
         const size_t t5_smem = kT5SmemBytes + sizeof(T5Ctl) + 1024;
         TIMED("attn", launch(k_attn_t5, dim3(t->sm_count), dim3(kT5Threads), t5_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
         TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, kT5Keys));
@@ -1050,7 +1059,7 @@ static bool mega_usable(const sj_target* t, const sj_kv* kv, int B, int gamma) {
          group * rows <= 16 * 6 && t->stream != nullptr;
 }
 
-static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode, bool use_scratch) {
+static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode, bool use_scratch, long total_keys) {
   const Dims& dm = t->dm;
   const int rows = gamma + 1, R = B * rows, Rp = pad16(R), qd = dm.Hq * dm.hd;
   cudaStream_t s = t->stream;
@@ -1065,14 +1074,22 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   memset(&p, 0, sizeof(p));
   p.B = B; p.rows = rows; p.R = R; p.Rp = Rp;
   p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
+  // tcgen05 attention phase: head dimension 128, a KV head's query rows within two TMEM lane quarters, and caches long
+  // enough that the phase is bound by throughput (at a few tiles per block it is a chain of latencies, and the
+  // mma.sync phase, which needs no hand-over between warps, is as fast)
+  const int nq = (dm.Hq / dm.Hkv) * rows;
+  const long tiles_per_block = total_keys * dm.Hkv / kA5Keys / t->sm_count;
+  const bool a5 = dm.hd == 128 && nq <= kA5MaxRows && t->opt_attn == 2 && tiles_per_block >= t->opt_a5_min_tiles;
+  p.q_area_bytes = a5 ? a5_q_area_bytes(nq) : 0;
+  p.att_spe = p.stage_bytes >= 2 * (int)kA5Part ? 1 : 2;
   const int ctl_bytes = ((int)sizeof(MegaCtl) + 127) & ~127;
-  const int budget = 227 * 1024 - 1024 - ctl_bytes;
+  const int budget = 227 * 1024 - 1024 - ctl_bytes - p.q_area_bytes;
   p.stages = std::min(8, std::min(kMegaMaxStages, budget / p.stage_bytes));   // deeper rings did not measure faster; the rest stays L1
   if (p.stages < 3) return fail(SJ_ERR_SHAPE, "too many rows for the whole-step kernel");
   if (t->opt_ring) p.stages = std::min(p.stages, t->opt_ring);
   uint32_t tc = 32;
   while (tc < (uint32_t)(4 * Rp)) tc <<= 1;
-  p.tmem_cols = tc;
+  p.tmem_cols = a5 ? std::max(tc, (uint32_t)kA5TmemCols) : tc;
   p.lp = t->d_layer_ptrs;
   p.embed = (const bf16*)t->embed;
   p.lm_head = (const bf16*)t->lm_head;
@@ -1086,7 +1103,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   p.trace = t->opt_trace ? t->d_trace : nullptr;
   p.trace_block = t->opt_trace ? (unsigned)std::min(t->opt_trace - 1, t->sm_count - 1) : 0u;
   const int grid = t->sm_count;
-  const size_t smem = (size_t)p.stages * p.stage_bytes + ctl_bytes + 1024;
+  const size_t smem = (size_t)p.stages * p.stage_bytes + p.q_area_bytes + ctl_bytes + 1024;
   const bool timing = t->opt_timing != 0;
   const int NL = dm.n_layers;
   for (size_t ci = 0; ci < t->mega_maps.size(); ++ci) {
@@ -1118,7 +1135,7 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
     const StepArgs* args = t->d_args;
     // row slots per epilogue thread: a group gets at most (min(R, 16) + 1) / 2 rows of a 16-row chunk
     const int ns = R <= 8 ? 4 : (R <= 12 ? 6 : 8);
-    CU_TRY(cudaLaunchKernelEx(&cfg, mega_kernel(dm.hd, ns, t->opt_trace != 0), mm, p, args, kv->view, W, dm));
+    CU_TRY(cudaLaunchKernelEx(&cfg, mega_kernel(dm.hd, ns, t->opt_trace != 0, a5), mm, p, args, kv->view, W, dm));
     if (timing) {
       CU_TRY(cudaEventRecord(eb, s));
       t->timed.push_back({"verify_step", ea, eb});
@@ -1298,7 +1315,7 @@ extern "C" sj_status sj_verify(sj_target* t, sj_kv* kv, const sj_verify_args* a,
 
   StepKey key{B, gamma, a->mode, chunk_len, t->opt_gemm, t->opt_attn, t->opt_pdl, use_scratch ? 1 : 0};
   if (use_mega) {
-    if ((st = launch_mega(t, kv, B, gamma, a->mode, use_scratch)) != SJ_OK) return st;
+    if ((st = launch_mega(t, kv, B, gamma, a->mode, use_scratch, total_keys)) != SJ_OK) return st;
   } else if (t->opt_graph) {
     auto it = t->graphs.find(key);
     if (it == t->graphs.end()) {

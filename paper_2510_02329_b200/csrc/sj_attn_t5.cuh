@@ -38,6 +38,7 @@ constexpr int kT5SmemBytes = 2 * kT5TileBytes /* Q hi, lo */ + 4 * kT5TileBytes 
 
 struct T5Ctl {
   uint64_t kfull[2], kempty[2], vfull[2], vempty[2], s_full[2], p_full[2], o_done[2], q_ready;
+  uint64_t pair[4];      // the two softmax warps of a lane quarter (64 arrivals)
   uint32_t tmem_base;
   int abort_flag;
   float mx[2][2][128];   // [tile parity][key half][query-row slot]: row maxima (and, at a segment's end, sums) of the two threads of a row
@@ -114,7 +115,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void bar_sync_n(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ bool t5_wait(uint64_t* bar, uint32_t parity, T5Ctl* ctl, int* status, int where) {
   return att_mbar_wait(att_smem_u32(bar), parity, &ctl->abort_flag, status, nullptr, where, 0);
 }
@@ -142,10 +142,11 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       att_mbar_init(att_smem_u32(&ctl->o_done[i]), 1);
     }
     att_mbar_init(att_smem_u32(&ctl->q_ready), 256);
+    for (int i = 0; i < 4; ++i) att_mbar_init(att_smem_u32(&ctl->pair[i]), 64);
     ctl->abort_flag = 0;
-    att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, kT5Keys);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 2) att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, kT5Keys, lane);
   // unused query-row slots stay zero for the whole kernel
   for (int i = threadIdx.x; i < 2 * kT5TileBytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 1) {
@@ -199,17 +200,10 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       int it = 0, seg = 0;
       long long t = t_lo;
       bool alive = true;
-#ifdef SJ_T5_PROF
-      long long pc_k = 0, pc_p = 0, pc_v = 0, pc_iss = 0, pc_q = 0, pc_t0 = clock64(), pc_x;
-#define T5P(acc, stmt) pc_x = clock64(); stmt; acc += clock64() - pc_x;
-#else
-#define T5P(acc, stmt) stmt;
-#endif
       while (t < t_hi && alive) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
         const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-        bool okq;
-        T5P(pc_q, okq = t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2))
+        const bool okq = t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2);
         if (!okq) break;
         tc_fence_after();
         for (int i = 0; i <= n && alive; ++i) {
@@ -217,13 +211,9 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
             const int g = it + i, st = g & 1;
             // S buffer `st` still holds P of tile g - 2 for that tile's P V, which this thread issued earlier: the
             // tensor pipe executes one thread's MMAs in issue order, so these may overwrite it
-            bool okk;
-            T5P(pc_k, okk = t5_wait(&ctl->kfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 3))
+            const bool okk = t5_wait(&ctl->kfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 3);
             if (!okk) { alive = false; break; }
             tc_fence_after();
-#ifdef SJ_T5_PROF
-            pc_x = clock64();
-#endif
             const uint32_t kb = k0 + (uint32_t)st * kT5TileBytes, d_s = tmem + (uint32_t)(st * 128);
 #pragma unroll
             for (int k = 0; k < HD / 16; ++k) {
@@ -234,20 +224,13 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
             }
             tc_commit(att_smem_u32(&ctl->kempty[st]));
             tc_commit(att_smem_u32(&ctl->s_full[st]));
-#ifdef SJ_T5_PROF
-            pc_iss += clock64() - pc_x;
-#endif
           }
           if (i >= 1) {  // output of tile i - 1
             const int g = it + i - 1, st = g & 1;
-            bool okp, okv;
-            T5P(pc_p, okp = t5_wait(&ctl->p_full[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 5))
-            T5P(pc_v, okv = okp && t5_wait(&ctl->vfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 6))
+            const bool okp = t5_wait(&ctl->p_full[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 5);
+            const bool okv = okp && t5_wait(&ctl->vfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 6);
             if (!okv) { alive = false; break; }
             tc_fence_after();
-#ifdef SJ_T5_PROF
-            pc_x = clock64();
-#endif
             const uint32_t vb = v0 + (uint32_t)st * kT5TileBytes, pb = tmem + (uint32_t)(st * 128);
 #pragma unroll
             for (int pg = 0; pg < 8; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
@@ -258,32 +241,32 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
             }
             tc_commit(att_smem_u32(&ctl->vempty[st]));
             tc_commit(att_smem_u32(&ctl->o_done[st]));
-#ifdef SJ_T5_PROF
-            pc_iss += clock64() - pc_x;
-#endif
           }
         }
         it += n;
         t += n;
         ++seg;
       }
-#ifdef SJ_T5_PROF
-      if (c == 0 && a.layer == 1) printf("t5 mma thread: tiles %d total %lld clk: wait q %lld, k %lld, p %lld, v %lld, issue %lld\n", it, clock64() - pc_t0, pc_q, pc_k, pc_p, pc_v, pc_iss);
-#endif
-#undef T5P
     }
   } else if (warp < 10) {
     // ------------------------------ softmax: two threads per query-row slot, 64 keys each ------------------------------
     // warps 2..5 take keys [0, 64) of every tile, warps 6..9 keys [64, 128); warp w reads TMEM lane quarter w % 4, so
-    // warps w and w + 4 share a quarter: they exchange their row maxima through shared memory (named barrier of
+    // warps w and w + 4 share a quarter: they exchange their row maxima through shared memory (a barrier of
     // their 64 threads) and keep separate sums, which are added when the segment's partial is written.
     const int half = (warp - 2) >> 2, quarter = warp & 3;
     const int sl = 32 * quarter + lane;                     // TMEM lane == query-row slot
     const int q = 4 * (sl & 31) + (sl >> 5);                // the query row of this slot (inverse of t5_lane_of_row)
     const bool active = q < nq;
     const uint32_t lane_addr = tmem + ((uint32_t)(32 * quarter) << 16);
-    const int pair_bar = 1 + quarter;
-    int it = 0, seg = 0;
+    int it = 0, seg = 0, pair_n = 0;
+    // hand-over between the quarter's two warps: a shared-memory barrier with a bounded wait, so that a warp that
+    // gives up cannot strand its partner
+    auto pair_sync = [&]() -> bool {
+      att_mbar_arrive(att_smem_u32(&ctl->pair[quarter]));
+      const bool ok = t5_wait(&ctl->pair[quarter], (uint32_t)pair_n & 1u, ctl, w.status, 10);
+      ++pair_n;
+      return __all_sync(0xffffffffu, ok);
+    };
     long long t = t_lo;
     bool alive = true;
     while (t < t_hi && alive) {
@@ -333,6 +316,10 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         tc_ld32_nowait(s_addr, sc);
         tc_ld32_nowait(s_addr + 32, sc + 32);
         tc_wait_ld();
+        if (!active) {   // a row slot without a query holds whatever its lane computed: keep it from moving the stabiliser
+#pragma unroll
+          for (int j = 0; j < 64; ++j) sc[j] = 0.f;
+        }
         float mx = -INFINITY;
         if (n_valid >= 64) {   // warp-uniform; every tile but a sequence's last
 #pragma unroll
@@ -345,7 +332,7 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
           }
         }
         ctl->mx[g & 1][half][sl] = mx;
-        bar_sync_n(pair_bar, 64);
+        if (!pair_sync()) { alive = false; break; }
         mx = fmaxf(mx, ctl->mx[g & 1][half ^ 1][sl]);
         // the stabiliser only moves when the maximum outgrows it by more than 8 (p stays below 256)
         float m_new = m_used, f = 1.f;
@@ -402,7 +389,7 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         att_mbar_try(att_smem_u32(&ctl->o_done[g & 1]), (uint32_t)(g >> 1) & 1u);
         tc_fence_after();
         ctl->mx[(g + 1) & 1][half][sl] = l_sum;           // the buffer the last tile did not use
-        bar_sync_n(pair_bar, 64);
+        if (!pair_sync()) break;
         const float l_tot = l_sum + ctl->mx[(g + 1) & 1][half ^ 1][sl];
         const size_t base = (((size_t)c + (size_t)x.b * Hkv + x.h) * kAttMaxSub + 0) * (size_t)nq;
         if (active && half == 0) { a.P.m[base + q] = m_used; a.P.l[base + q] = l_tot; }
@@ -417,7 +404,7 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
           }
         }
         tc_fence_before();
-        bar_sync_n(pair_bar, 64);   // the sums have been read before the next segment's first tile reuses the buffer
+        if (!pair_sync()) break;   // the sums have been read before the next segment's first tile reuses the buffer
       }
       it += n;
       t += n;
@@ -437,6 +424,382 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
+}
+
+
+// =============================================================================================
+// The same attention as phase routines of a kernel whose shared-memory ring also carries other traffic (the
+// persistent step kernel): 64-key tiles, the queries in an area of their own, at most 64 query rows per
+// (sequence, KV head).
+//
+// A tile is one ring entry, key part then value part of 16 KiB each ([half][page][16 keys x 128 B], as above with
+// four pages): in ONE stage when a stage holds 32 KiB, else in two consecutive stages (key stage, value stage; each
+// has its own full / empty barrier).  Query row q sits in TMEM lane q and in row q of the query area, which holds
+// pad8(nq) rows per 64-dim half: the MMAs run at M = 128 all the same, their rows beyond the area read whatever
+// shared memory follows it (the caller guarantees 16 KiB of its own allocation after the last half's base) and
+// produce accumulator lanes nobody reads.
+//
+// Three issuing threads.  One thread gets a tcgen05.mma out every 110 clocks or so whatever its shape (measured: M 64 or
+// 128, N 32..128, operand A in shared or tensor memory; two threads issue twice as many), and a tile needs 8 k-steps x 2
+// query planes for the scores and 4 pages x 2 probability planes for the output.  So the scores are two accumulators,
+// S_hi = Q_hi K^T and S_lo = Q_lo K^T, each with a thread of its own (the softmax adds them), and a third thread issues
+// the output MMAs: 8 MMAs per tile and thread.  Tensor memory: S_hi twice at columns [0, 128) (the probabilities are
+// written over it), S_lo twice at [128, 256), the output at [256, 384), aliasing whatever the kernel keeps there outside
+// the attention phase.
+// =============================================================================================
+constexpr int kA5Keys = 64;
+constexpr int kA5MaxRows = 64;
+constexpr uint32_t kA5Part = 16384;
+constexpr int kA5TmemCols = 512;
+
+struct A5Bars {
+  uint64_t s_full[2];   // two arrivals: the commits of both score issuers
+  uint64_t p_full[2];   // 128 arrivals: the softmax threads
+  uint64_t o_done[2];   // one arrival: the output issuer's commit
+  uint64_t q_ready;     // 128 arrivals
+};
+struct A5Ring {
+  uint64_t* full;    // [stages], each completes on two arrivals (the expecting one and a second)
+  uint64_t* empty;   // [stages], one arrival
+  uint8_t* base;
+  int stage_stride, stages, spe;   // spe: stages per entry (1 or 2)
+  volatile int* abort_flag;
+  volatile int* abort_g;
+  int* status;
+};
+struct A5Pos {
+  int s, r;
+  __device__ __forceinline__ void next(int NS) {
+    if (++s == NS) { s = 0; ++r; }
+  }
+};
+struct A5Entry {
+  int s0, s1;
+  uint32_t par0, par1, a0, a1;   // stage, parity of this use and address of the key part (0) and the value part (1)
+};
+__host__ __device__ __forceinline__ int a5_q_half_bytes(int nq) { return ((nq + 7) & ~7) * 128; }
+__host__ __device__ __forceinline__ int a5_q_area_bytes(int nq) { return 4 * a5_q_half_bytes(nq); }   // two planes x two halves
+
+__device__ __forceinline__ A5Entry a5_entry(const A5Ring& rg, A5Pos& pos) {   // the entry at pos; pos moves past it
+  A5Entry e;
+  e.s0 = pos.s;
+  e.par0 = (uint32_t)pos.r & 1u;
+  e.a0 = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
+  if (rg.spe == 2) {
+    pos.next(rg.stages);
+    e.s1 = pos.s;
+    e.par1 = (uint32_t)pos.r & 1u;
+    e.a1 = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
+  } else {
+    e.s1 = e.s0;
+    e.par1 = e.par0;
+    e.a1 = e.a0 + kA5Part;
+  }
+  pos.next(rg.stages);
+  return e;
+}
+__device__ __forceinline__ bool a5_wait(const A5Ring& rg, uint64_t* bar, uint32_t parity, int where, int extra) {
+  return att_mbar_wait(att_smem_u32(bar), parity, rg.abort_flag, rg.status, rg.abort_g, where, extra);
+}
+
+// Sixteen lanes of one warp (pl_lane 0..15, all in the same control flow): the TMA loads of the block's tiles
+// [t_lo, t_hi) of one layer.  A tile is sixteen boxes of 2 KiB (16 keys x 64 dims: a page's slots, one swizzle span wide),
+// and one thread gets a copy out only every 200 clocks or so, far below what the tile's 32 KiB need; so every lane
+// issues ONE box of each tile (part = lane / 8, half = lane / 4 % 2, page = lane % 4) and a tile costs one instruction.
+// Lane 0 announces the bytes.  pages: the block's page ids, four per tile (clamped to the sequence's last page), for
+// its first kAttPageCache / 4 tiles.
+__device__ __forceinline__ bool a5_produce(const A5Ring& rg, A5Pos& pos, const CUtensorMap* tmKV, const KvView& kv,
+                                           const StepArgs* __restrict__ args, const AttPlan& pl, int B, int layer,
+                                           long long t_lo, long long t_hi, const int* pages, int pl_lane) {
+  const int which = pl_lane >> 3, half = (pl_lane >> 2) & 1, p = pl_lane & 3;
+  int tb = 0;
+  for (long long t = t_lo; t < t_hi; ++t, ++tb) {
+    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
+    const int seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
+    int pi = x.ti * 4 + p;
+    if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
+    const int page = (tb + 1) * 4 <= kAttPageCache ? pages[tb * 4 + p]
+                                                   : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+    const long long row = ((((long long)layer * kv.n_pages + page) * 2 + which) * kv.n_kv_heads + x.h) * 16;
+    // claim the entry's stage(s): every lane waits (same flow), lane 0 announces
+    uint32_t dst = 0, bar = 0;
+    for (int st = 0; st < rg.spe; ++st) {
+      if (pos.r > 0 && !a5_wait(rg, &rg.empty[pos.s], (uint32_t)(pos.r - 1) & 1u, 1, pos.r)) return false;
+      const uint32_t b_st = att_smem_u32(&rg.full[pos.s]);
+      const uint32_t d_st = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
+      if (pl_lane == 0) {
+        att_mbar_expect_tx(b_st, rg.spe == 2 ? kA5Part : 2 * kA5Part);
+        att_mbar_arrive(b_st);   // the stage's second arrival
+      }
+      if (rg.spe == 1) { bar = b_st; dst = d_st + (uint32_t)which * kA5Part; }
+      else if (st == which) { bar = b_st; dst = d_st; }
+      pos.next(rg.stages);
+    }
+    att_tma_2d(dst + (uint32_t)(half * 8192 + p * 2048), tmKV, bar, half * 64, (int)row);
+  }
+  return true;
+}
+
+// One thread per query plane (0: hi, 1: lo): S_plane = Q_plane K^T of the block's tiles.  gt: tiles of earlier layers
+// (the barriers' phases run on across layers), segs: segments of earlier layers; both advanced.
+__device__ __forceinline__ bool a5_issue_qk(const A5Ring& rg, A5Pos& pos, A5Bars* ab, uint32_t tmem, uint32_t q_area, int nq,
+                                            int plane, const AttPlan& pl, int B, long long t_lo, long long t_hi, int& gt,
+                                            int& segs) {
+  const uint32_t id_s = instr_desc_bf16_mn(kA5Keys, 0);
+  const uint32_t hs = (uint32_t)a5_q_half_bytes(nq);
+  long long t = t_lo;
+  while (t < t_hi) {
+    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
+    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    if (!a5_wait(rg, &ab->q_ready, (uint32_t)segs & 1u, 2, segs)) return false;
+    tc_fence_after();
+    for (int i = 0; i < n; ++i) {
+      const int g = gt + i, sb = g & 1;
+      const A5Entry e = a5_entry(rg, pos);
+      // score buffer sb held the probabilities of tile g - 2: its P V (the other issuer's) must have completed
+      if (!a5_wait(rg, &rg.full[e.s0], e.par0, 3, g) ||
+          (g >= 2 && !a5_wait(rg, &ab->o_done[sb], (uint32_t)((g >> 1) - 1) & 1u, 4, g)))
+        return false;
+      tc_fence_after();
+      const uint32_t d_s = tmem + (uint32_t)(128 * plane + sb * kA5Keys);
+      const uint64_t dq = smem_desc_sw128(q_area + (uint32_t)plane * 2 * hs), dk = smem_desc_sw128(e.a0);
+      const uint64_t dq_half = (uint64_t)(hs >> 4), dk_half = (uint64_t)(8192 >> 4);   // start-address field, 16-byte units
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        tc_mma_bf16(d_s, dq + (k >> 2) * dq_half + 2 * (k & 3), dk + (k >> 2) * dk_half + 2 * (k & 3), id_s, k > 0 ? 1u : 0u);
+      tc_commit(att_smem_u32(&ab->s_full[sb]));   // the output issuer frees the stage
+    }
+    gt += n;
+    t += n;
+    ++segs;
+  }
+  return true;
+}
+
+// One thread: O += P V of the block's tiles.
+__device__ __forceinline__ bool a5_issue_pv(const A5Ring& rg, A5Pos& pos, A5Bars* ab, uint32_t tmem, const AttPlan& pl, int B,
+                                            long long t_lo, long long t_hi, int& gt) {
+  const uint32_t id_o = instr_desc_bf16_mn(128, 1);
+  long long t = t_lo;
+  while (t < t_hi) {
+    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
+    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    for (int i = 0; i < n; ++i) {
+      const int g = gt + i, sb = g & 1;
+      const A5Entry e = a5_entry(rg, pos);
+      if (!a5_wait(rg, &ab->p_full[sb], (uint32_t)(g >> 1) & 1u, 5, g) || !a5_wait(rg, &rg.full[e.s1], e.par1, 6, g)) return false;
+      tc_fence_after();
+      const uint32_t pb = tmem + (uint32_t)(sb * kA5Keys);
+      const uint64_t dv = smem_desc_mn_sw128(e.a1, 8192u);
+#pragma unroll
+      for (int pg = 0; pg < 4; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
+        const uint64_t db = dv + (uint64_t)(pg * (2048 >> 4));
+        const uint32_t pa = pb + (uint32_t)(32 * (pg >> 1) + 8 * (pg & 1));
+        tc_mma_bf16_ta(tmem + 256, pa, db, id_o, (i > 0 || pg > 0) ? 1u : 0u);
+        tc_mma_bf16_ta(tmem + 256, pa + 16, db, id_o, 1u);
+      }
+      // both score chains of this tile completed before its probabilities were written: the key part is free too
+      if (rg.spe == 2) tc_commit(att_smem_u32(&rg.empty[e.s0]));
+      tc_commit(att_smem_u32(&rg.empty[e.s1]));
+      tc_commit(att_smem_u32(&ab->o_done[sb]));
+    }
+    gt += n;
+    t += n;
+  }
+  return true;
+}
+
+// byte offset of (row, dim) in one plane of the query area (two K-major halves `hs` bytes apart, 128-byte swizzle)
+__device__ __forceinline__ uint32_t a5_q_off(int row, int dim, uint32_t hs) {
+  return (uint32_t)(dim >> 6) * hs + (uint32_t)(row * 128 + ((((dim & 63) >> 3) ^ (row & 7)) << 4) + (dim & 7) * 2);
+}
+
+// The softmax side: four warps, two threads per query row.  quarter (0, 1): the TMEM lane quarter == rows
+// [32 * quarter, +32); half (0, 1): keys [32 * half, +32) of every tile and dims [64 * half, +64) of the row's queries
+// and output.  mx: [2][2][64] floats of shared memory; pair_bar: a shared-memory barrier of the quarter's 64 threads (count 64;
+// every wait is bounded, so a warp that gives up cannot strand its partner), pair_n: its phases so far.
+// slot0: the partial slot of the block's segment is slot0 + b * Hkv + h (sub-partial 0).
+// ev: optional timeline of the block's last segment (global-timer ns), stamped by the first softmax warp:
+// [0] queries delivered, [1] last tile's probabilities delivered, [2] partial stored, [3] first scores seen.
+__device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_t tmem, uint8_t* q_area, float* mx, uint64_t* pair_bar, int& pair_n,
+                                           const AttArgs& a, const AttPlan& pl, int B, int Hkv, int nq, long long t_lo,
+                                           long long t_hi, int& gt, int slot0, int quarter, int half, int lane,
+                                           unsigned long long* ev = nullptr) {
+  constexpr int HD = 128;
+  const bool stamp = ev && quarter == 0 && half == 0 && lane == 0;
+  const int q = 32 * quarter + lane;   // query row == TMEM lane == row of the query area
+  const bool active = q < nq;
+  const uint32_t hs = (uint32_t)a5_q_half_bytes(nq);
+  const uint32_t lane_addr = tmem + ((uint32_t)(32 * quarter) << 16);
+  float* mx_own = mx + half * 64 + q;
+  float* mx_other = mx + (half ^ 1) * 64 + q;   // + 128 * (tile parity)
+  auto pair_sync = [&]() -> bool {
+    att_mbar_arrive(att_smem_u32(pair_bar));
+    const bool ok = a5_wait(rg, pair_bar, (uint32_t)pair_n & 1u, 10, pair_n);
+    ++pair_n;
+    return __all_sync(0xffffffffu, ok);
+  };
+  long long t = t_lo;
+  while (t < t_hi) {
+    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
+    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    // queries of this (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16
+    // terms.  The previous segment's score MMAs have completed: this thread saw the s_full of its last tile.
+    if (active) {
+      const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD;
+      const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD : nullptr;
+      uint4 raw[8], rawl[8];
+#pragma unroll
+      for (int d8 = 0; d8 < 8; ++d8) {   // all loads first
+        raw[d8] = __ldcg(reinterpret_cast<const uint4*>(qh + 64 * half + 8 * d8));
+        rawl[d8] = ql ? __ldcg(reinterpret_cast<const uint4*>(ql + 64 * half + 8 * d8)) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int d8 = 0; d8 < 8; ++d8) {
+        const __half2* h2 = reinterpret_cast<const __half2*>(&raw[d8]);
+        const __half2* l2 = reinterpret_cast<const __half2*>(&rawl[d8]);
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 v = __half22float2(h2[e]);
+          const float2 vl = __half22float2(l2[e]);
+          v.x += vl.x;
+          v.y += vl.y;
+          const __nv_bfloat162 bh = __floats2bfloat162_rn(v.x, v.y);
+          const float2 back = __bfloat1622float2(bh);
+          const __nv_bfloat162 bl = __floats2bfloat162_rn(v.x - back.x, v.y - back.y);
+          hi[e] = *reinterpret_cast<const uint32_t*>(&bh);
+          lo[e] = *reinterpret_cast<const uint32_t*>(&bl);
+        }
+        const uint32_t off = a5_q_off(q, 64 * half + 8 * d8, hs);
+        *reinterpret_cast<uint4*>(q_area + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(q_area + 2 * hs + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read these generic-proxy stores
+    att_mbar_arrive(att_smem_u32(&ab->q_ready));
+    if (stamp) ev[0] = att_timer_ns();
+    float m_used = -INFINITY, l_sum = 0.f;
+    for (int i = 0; i < n; ++i) {
+      const int g = gt + i, sb = g & 1;
+      const uint32_t par = (uint32_t)(g >> 1) & 1u;
+      int ok = 1;
+      if (lane == 0) ok = a5_wait(rg, &ab->s_full[sb], par, 7, g) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) return false;
+      if (stamp && i == 0) ev[3] = att_timer_ns();
+      att_mbar_try(att_smem_u32(&ab->s_full[sb]), par);   // every lane observes the completed phase
+      tc_fence_after();
+      const uint32_t s_addr = lane_addr + (uint32_t)(sb * kA5Keys + 32 * half);
+      const int n_valid = min(kA5Keys, x.L - (x.ti + i) * kA5Keys) - 32 * half;   // this thread's keys >= n_valid are masked
+      float sc[32];
+      {
+        float lo[32];
+        tc_ld32_nowait(s_addr, sc);
+        tc_ld32_nowait(s_addr + 128, lo);
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[j] += lo[j];
+      }
+      if (!active) {   // a row slot without a query holds whatever its lane computed: keep it from moving the stabiliser
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sc[j] = 0.f;
+      }
+      float m_tile = -INFINITY;
+      if (n_valid >= 32) {   // warp-uniform; every tile but a sequence's last
+#pragma unroll
+        for (int j = 0; j < 32; ++j) m_tile = fmaxf(m_tile, sc[j]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
+          m_tile = fmaxf(m_tile, sc[j]);
+        }
+      }
+      mx_own[128 * sb] = m_tile;
+      if (!pair_sync()) return false;
+      m_tile = fmaxf(m_tile, mx_other[128 * sb]);
+      // the stabiliser only moves when the maximum outgrows it by more than 8 (p stays below 256)
+      float m_new = m_used, f = 1.f;
+      if (m_used == -INFINITY) m_new = m_tile;
+      else if (m_tile > m_used + 8.f) { m_new = m_tile; f = ex2_approx(m_used - m_new); }
+      if (i > 0 && __any_sync(0xffffffffu, f != 1.f)) {
+        // rescale this thread's half of its row of O: only once the previous tile's P V has completed (this
+        // tile's cannot start before every thread has delivered its P)
+        const uint32_t po = (uint32_t)((g - 1) >> 1) & 1u;
+        if (lane == 0) ok = a5_wait(rg, &ab->o_done[(g - 1) & 1], po, 8, g) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) return false;
+        att_mbar_try(att_smem_u32(&ab->o_done[(g - 1) & 1]), po);
+        tc_fence_after();
+#pragma unroll 1
+        for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+          float o[32];
+          tc_ld32(lane_addr + 256 + c0, o);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] *= f;
+          tc_st32f(lane_addr + 256 + c0, o);
+        }
+        l_sum *= f;
+      }
+      // probabilities as two bf16 terms over the scores: [hi 16 columns | lo 16 columns]; hi = p truncated to bf16,
+      // lo = the rest rounded to bf16 (16 significant bits in all)
+      {
+        uint32_t hi[16], lo[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = ex2_approx(sc[j] - m_new), p1 = ex2_approx(sc[j + 1] - m_new);   // 0 for masked keys
+          l_sum += p0 + p1;
+          const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
+          hi[j >> 1] = __byte_perm(b0, b1, 0x7632);
+          const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - __uint_as_float(b0 & 0xffff0000u), p1 - __uint_as_float(b1 & 0xffff0000u));
+          lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&bl);
+        }
+        tc_st16(s_addr, hi);
+        tc_st16(s_addr + 16, lo);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      att_mbar_arrive(att_smem_u32(&ab->p_full[sb]));
+      m_used = m_new;
+    }
+    if (stamp) ev[1] = att_timer_ns();
+    // the segment's partial: wait for the last P V, then (m, l, o) of every real query row
+    {
+      const int g = gt + n - 1;
+      const uint32_t po = (uint32_t)(g >> 1) & 1u;
+      int ok = 1;
+      if (lane == 0) ok = a5_wait(rg, &ab->o_done[g & 1], po, 9, g) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) return false;
+      att_mbar_try(att_smem_u32(&ab->o_done[g & 1]), po);
+      tc_fence_after();
+      mx_own[128 * ((g + 1) & 1)] = l_sum;   // the buffer the last tile did not use
+      if (!pair_sync()) return false;
+      const float l_tot = l_sum + mx_other[128 * ((g + 1) & 1)];
+      const size_t base = (((size_t)slot0 + (size_t)x.b * Hkv + x.h) * kAttMaxSub + 0) * (size_t)nq;
+      if (active && half == 0) {
+        a.P.m[base + q] = m_used;
+        a.P.l[base + q] = l_tot;
+      }
+#pragma unroll 1
+      for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+        float o[32];
+        tc_ld32(lane_addr + 256 + c0, o);
+        if (active) {
+          float4* dst = reinterpret_cast<float4*>(a.P.o + (base + q) * HD + c0);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) dst[j] = make_float4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        }
+      }
+      tc_fence_before();
+      if (!pair_sync()) return false;   // the sums have been read before the next segment's first tile reuses the buffer
+      if (stamp) ev[2] = att_timer_ns();
+    }
+    gt += n;
+    t += n;
+  }
+  return true;
 }
 
 }  // namespace sj

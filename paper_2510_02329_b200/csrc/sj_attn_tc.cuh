@@ -379,18 +379,32 @@ struct AttPlan {
   long long T;               // total ring tiles
 };
 
-// Filled by one thread; callers synchronise afterwards.
+// Filled by one full warp (every lane calls it); callers synchronise afterwards.  Lane i takes sequences i, i + 32, ...:
+// the cache lengths are loaded side by side (one thread alone would wait for each load in turn, half a microsecond
+// apiece at a batch of 32) and the tile counts summed by a warp prefix sum.
 __device__ __forceinline__ void att_plan_fill(AttPlan* pl, const int* __restrict__ row_pos, int B, int rows, int Hkv,
-                                              int KPS) {
-  int acc = 0;
-  for (int b = 0; b < B; ++b) {
-    const int L = row_pos[b * rows];
-    pl->L[b] = L;
-    pl->pre[b] = acc;
-    acc += Hkv * ((L + KPS - 1) / KPS);
+                                              int KPS, int lane) {
+  int carry = 0;
+  for (int b0 = 0; b0 < B; b0 += 32) {
+    const int b = b0 + lane;
+    const int L = b < B ? row_pos[b * rows] : 0;
+    const int n = b < B ? Hkv * ((L + KPS - 1) / KPS) : 0;
+    int incl = n;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += up;
+    }
+    if (b < B) {
+      pl->L[b] = L;
+      pl->pre[b] = carry + incl - n;
+    }
+    carry += __shfl_sync(0xffffffffu, incl, 31);
   }
-  pl->pre[B] = acc;
-  pl->T = acc;
+  if (lane == 0) {
+    pl->pre[B] = carry;
+    pl->T = carry;
+  }
 }
 
 __device__ __forceinline__ int att_find_seq(const int* pre, int B, int t) {
@@ -665,9 +679,9 @@ k_attn_tc(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       ctl->cons_cnt[i] = 0;
     }
     ctl->abort_flag = 0;
-    att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, g.KPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 1) att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, g.KPS, lane);
   __syncthreads();
   const AttPlan& pl = ctl->plan;
   const int G = gridDim.x, c = blockIdx.x;
@@ -829,7 +843,7 @@ __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dim
   const int B = args->B, rows = args->gamma + 1;
   AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
   if (keys_per_tile > 0) { g.KPS = keys_per_tile; g.KS = 1; g.KW = keys_per_tile; }
-  if (threadIdx.x == 0) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS);
+  if (threadIdx.x < 32) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS, threadIdx.x);
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
   const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;

@@ -26,7 +26,11 @@
 //   gate/up (tiles interleave 64 gate and 64 up features) -> silu(g) * u -> down-projection input planes
 //   down  -> as O
 //   LM head -> softmax statistics per (vocabulary tile, row), logit of the drafted token
-// Attention: see sj_attn_tc.cuh; its cache tiles travel through the same ring.
+// Attention: its cache tiles travel through the same ring.  Two implementations, chosen per launch: fp16 mma.sync in
+// the worker warps (sj_attn_tc.cuh), or -- head dimension 128, at most 64 query rows per KV head and sequence --
+// tcgen05 (the routines at the end of sj_attn_t5.cuh): warps 1 and 2 issue the score MMAs, warp 3 the output MMAs, four
+// worker warps run the softmax on tensor memory, the other four the causal tails; the queries sit in an area of their own
+// after the ring, the accumulators alias the GEMM phases' tensor-memory columns.
 //
 // Every wait is bounded; the first one to run out raises a device-wide abort word that all other waits
 // poll, so that a logic error ends the kernel with SJ_ERR_TIMEOUT instead of hanging the GPU.
@@ -34,6 +38,7 @@
 
 #include "sj_attn_tc.cuh"
 #include "sj_gemm_tc.cuh"
+#include "sj_attn_t5.cuh"
 
 namespace sj {
 
@@ -89,6 +94,8 @@ struct MegaParams {
   int* abort_g;               // device-wide abort word        }
   int n_tail_base;
   int att_precise_layers;     // layers [0, n) run the attention with two-term (hi + lo fp16) queries and probabilities
+  int att_spe;                // tcgen05 attention: ring stages per 64-key tile (1: keys and values share a stage, 2: one each)
+  int q_area_bytes;           // tcgen05 attention: bytes of the query area between the ring and the control block
   // optional timeline (global-timer nanoseconds), block `trace_block`:
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
   //   [2*kMegaTraceBarriers + 8*s + e]  event e of GEMM phase s: 0 activation producer released, 1 its last
@@ -128,6 +135,8 @@ struct MegaCtl {
   uint32_t tmem_base;
   int abort_flag;
   int bars_passed;
+  A5Bars a5;                   // tcgen05 attention: score / probability / output hand-offs
+  uint64_t a5_pair[2];         // ... and the barrier of each lane quarter's two softmax warps
   int bcast[6];   // [2 * group + accumulator]: the group's wait on that accumulator succeeded; [4], [5] spare
   float inv[kMegaMaxRows];
   float zd[kMegaMaxRows];      // top-k test: raw logit of each row's drafted token, computed before the LM head
@@ -143,9 +152,14 @@ struct MegaCtl {
   int att_pages[kAttPageCache];   // page ids of this block's first ring tiles (the same in every layer)
   union {
     float exch[2][128][9];      // [group][feature][row of the chunk]
+    float a5_mx[2][2][64];      // tcgen05 attention: [tile parity][key half][query row] maxima / sums of a row's two threads
     RowStat sred[kMegaWorkers];
   } u;
 };
+
+// The tcgen05 attention's M = 128 descriptors read up to 16 KiB past the last half of the query area, which this
+// block follows: those bytes must be the kernel's own.
+static_assert(sizeof(MegaCtl) >= 16384, "the control block no longer covers the query area's over-read");
 
 struct SiteInfo {
   int n_tiles, KB;
@@ -943,16 +957,18 @@ __device__ __forceinline__ void mega_finalize(MegaCtl* ctl, const MegaParams& p,
 // ---------------------------------------------------------------------------------------------
 // the kernel
 // ---------------------------------------------------------------------------------------------
-template <int HD, int SLOTS, bool kTr>
+template <int HD, int SLOTS, bool kTr, bool A5>
 __global__ void __launch_bounds__(kMegaThreads, 1)
 k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const StepArgs* __restrict__ args, const KvView kv,
               const Work w, const Dims dm) {
   extern __shared__ uint8_t mega_smem_raw[];
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(mega_smem_raw) + 1023) & ~(uintptr_t)1023);
-  MegaCtl* ctl = reinterpret_cast<MegaCtl*>(ring + (size_t)p.stages * p.stage_bytes);
+  uint8_t* q_area = ring + (size_t)p.stages * p.stage_bytes;
+  MegaCtl* ctl = reinterpret_cast<MegaCtl*>(q_area + p.q_area_bytes);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int c = blockIdx.x, G = gridDim.x, NS = p.stages, B = p.B, R = p.R, Rp = p.Rp, rows = p.rows;
-  const AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+  AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
+  if constexpr (A5) { g.KPS = kA5Keys; g.KS = 1; g.KW = kA5Keys; }   // one sub-partial per block segment
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -963,7 +979,12 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[i]), kMegaWorkers);
+      mbar_init(smem_u32(&ctl->a5.s_full[i]), 2);
+      mbar_init(smem_u32(&ctl->a5.p_full[i]), 128);
+      mbar_init(smem_u32(&ctl->a5.o_done[i]), 1);
+      mbar_init(smem_u32(&ctl->a5_pair[i]), 64);
     }
+    mbar_init(smem_u32(&ctl->a5.q_ready), 128);
     ctl->abort_flag = 0;
     ctl->bars_passed = 0;
     int acc = 0;
@@ -1002,7 +1023,8 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
 
   const AttPlan& pl = ctl->plan;
   const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
-  const int n_att = (int)(t_hi - t_lo);
+  const int n_att = (int)(t_hi - t_lo) * (A5 ? p.att_spe : 1);   // ring stages of one attention phase
+  const A5Ring a5r{ctl->full, ctl->empty, ring, p.stage_bytes, NS, p.att_spe, &ctl->abort_flag, p.abort_g, w.status};
   att_fill_pages(ctl->att_pages, pl, kv, args, B, g.KPS, t_lo, t_hi, threadIdx.x, blockDim.x);
   __syncthreads();
   auto stage_addr = [&](int s) -> uint32_t { return smem_u32(ring + (size_t)s * p.stage_bytes); };
@@ -1015,7 +1037,10 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kMegaRegsLight));
   if (warp == 0) {
     // ------------------------------ weight / cache-tile producer ------------------------------
-    if (lane == 0) {
+    // One lane; sixteen with the tcgen05 attention, whose cache tiles are sixteen small copies each (one per lane, one
+    // instruction per tile).  All lanes run the same control flow and wait on the same barriers; lane 0 alone announces
+    // bytes and issues the weight copies.
+    if (lane < (A5 ? 16 : 1)) {
       const uint64_t pol_w = l2_policy_evict_first();
       RingPos rp{0, 0, NS};
       int sidx = 0;
@@ -1045,18 +1070,27 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
           else tm0 = &mp.lm;
           for (int kb = sg.a; kb < sg.b; ++kb) {
             if (!wait_slot()) { alive = false; return; }
-            const uint32_t bar = smem_u32(&ctl->full[rp.s]), dst = stage_addr(rp.s);
-            mbar_expect_tx(bar, kWTileBytes);
-            tma_load_2d(dst, tm0, bar, kb * kBK, row, pol_w);
-            if (site == SITE_GU) tma_load_2d(dst + 8192u, tm1, bar, kb * kBK, row, pol_w);
+            if (lane == 0) {
+              const uint32_t bar = smem_u32(&ctl->full[rp.s]), dst = stage_addr(rp.s);
+              mbar_expect_tx(bar, kWTileBytes);
+              tma_load_2d(dst, tm0, bar, kb * kBK, row, pol_w);
+              if (site == SITE_GU) tma_load_2d(dst + 8192u, tm1, bar, kb * kBK, row, pol_w);
+            }
             rp.next();
           }
         }
-        MEGA_EV(sidx, 7);
+        if (lane == 0) MEGA_EV(sidx, 7);
         ++sidx;
       };
       auto fatt = [&](int l) {
         if (!alive) return;
+        if constexpr (A5) {
+          A5Pos ap{rp.s, rp.r};
+          alive = a5_produce(a5r, ap, &mp.pool, kv, args, pl, B, l, t_lo, t_hi, ctl->att_pages, lane);
+          rp.s = ap.s;
+          rp.r = ap.r;
+          return;
+        }
         for (long long t = t_lo; t < t_hi; ++t) {
           if (!wait_slot()) { alive = false; return; }
           const uint32_t bar = smem_u32(&ctl->full[rp.s]);
@@ -1117,7 +1151,18 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         MEGA_EV(sidx, 3);
         ++sidx;
       };
-      auto fatt = [&](int l) { rp.advance(n_att); };
+      int a5_tiles = 0, a5_segs = 0;
+      auto fatt = [&](int l) {
+        if constexpr (A5) {
+          if (!alive) return;
+          A5Pos ap{rp.s, rp.r};
+          alive = a5_issue_qk(a5r, ap, &ctl->a5, tmem_base, smem_u32(q_area), g.nq, 0, pl, B, t_lo, t_hi, a5_tiles, a5_segs);
+          rp.s = ap.s;
+          rp.r = ap.r;
+        } else {
+          rp.advance(n_att);
+        }
+      };
       mega_walk(p, fsite, fatt);
     }
   } else {
@@ -1164,7 +1209,22 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         ++sidx;
         nb += (site == SITE_QKV) ? 3 : 1;
       };
-      auto fatt = [&](int l) { rp.advance(n_att); };
+      int a5_tiles = 0, a5_segs = 0;
+      auto fatt = [&](int l) {
+        if constexpr (A5) {
+          // the attention's other two issuers: warp 2 the scores of the lo query plane, warp 3 the output MMAs
+          if (!alive) return;
+          A5Pos ap{rp.s, rp.r};
+          if (mine == 0)
+            alive = a5_issue_qk(a5r, ap, &ctl->a5, ctl->tmem_base, smem_u32(q_area), g.nq, 1, pl, B, t_lo, t_hi, a5_tiles, a5_segs);
+          else
+            alive = a5_issue_pv(a5r, ap, &ctl->a5, ctl->tmem_base, pl, B, t_lo, t_hi, a5_tiles);
+          rp.s = ap.s;
+          rp.r = ap.r;
+        } else {
+          rp.advance(n_att);
+        }
+      };
       mega_walk(p, fsite, fatt);
     }
   }
@@ -1173,6 +1233,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     // ------------------------------ workers ------------------------------
     const int wt = threadIdx.x - 128, ww = wt >> 5;
     int nbar = 0, gseq = 0, seg = 0, it = 0;
+    int a5_tiles = 0, a5_pairs = 0;
     bool alive = true;
     if (p.do_embed) {
       mega_embed(ctl, p, args, kv, w, dm, wt);
@@ -1195,14 +1256,29 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       }
       // attention over the cache tiles of the ring, then the combine
       if (alive) {
-        // attention events of block 0 go to the second event set of the layer's QKV phase
-        unsigned long long* ev = (kTr && p.trace && c == 0 && (l - p.l0) * 4 < kMegaTraceSites)
+        // attention events of the traced block go to the second event set of the layer's QKV phase
+        unsigned long long* ev = (kTr && p.trace && c == (int)p.trace_block && (l - p.l0) * 4 < kMegaTraceSites)
                                      ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8
                                      : nullptr;
         AttRing rg{ctl->full, ctl->empty, ctl->cons_cnt, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status, ev};
         AttArgs aa{w.Qb, l < p.att_precise_layers ? w.Qlo : nullptr, w.KVn, AttPartials{w.tc_m, w.tc_l, w.tc_o}, p.n_tail_base, l};
-        int it2 = it;
-        att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
+        if constexpr (A5) {
+          if ((ww & 3) < 2) {
+            // softmax warps: lane quarter ww & 3, key / dim half ww >> 2
+            alive = a5_softmax(a5r, &ctl->a5, ctl->tmem_base, q_area, &ctl->u.a5_mx[0][0][0], &ctl->a5_pair[ww & 3], a5_pairs, aa, pl, B,
+                               dm.Hkv, g.nq, t_lo, t_hi, a5_tiles, c, ww & 3, ww >> 2, lane, ev);
+          } else {
+            // the other four warps: the causal tails (one m-tile of one (sequence, KV head) per task), dealt over
+            // all blocks from the last block down
+            AttWarp<HD, 2> st;
+            const int k = (ww & 1) + 2 * (ww >> 2);
+            for (int q = (G - 1 - c) * 4 + k; q < B * dm.Hkv * g.MT; q += G * 4)
+              att_tail_task<HD, 2>(st, g, aa, q / g.MT, (q % g.MT) * 16, lane);
+          }
+        } else {
+          int it2 = it;
+          att_consume_dispatch<HD>(rg, it2, pl, g, args, kv, aa, dm.Hkv, c, G, ww, lane);
+        }
       }
       it += n_att;
       alive = mega_grid_sync<kTr>(ctl, p, w.status, nbar, wt);

@@ -379,6 +379,32 @@ def test_tcgen05_attention(name, shape, kv_lens, gamma):
         case.close()
 
 
+A5_CASES = [
+    ("llama-8b-cut2", synth.LLAMA_8B.cut(2), [210, 4096], 8),                  # config 3 widths, two sequences: 18 rows
+    ("llama-8b-cut1-edges", synth.LLAMA_8B.cut(1), [1, 63, 64, 65, 0, 129], 4),  # 64-key tile edges; an empty cache
+    ("llama-8b-cut1-g10", synth.LLAMA_8B.cut(1), [3000], 10),                  # 44 query rows
+    ("qwen-32b-cut1", synth.QWEN_32B.cut(1), [40, 1300, 515], 8),              # group 5 (45 query rows), qkv bias, 36 KiB ring stages
+]
+
+
+@pytest.mark.parametrize("name,shape,kv_lens,gamma", A5_CASES, ids=[c[0] for c in A5_CASES])
+def test_tcgen05_attention_in_persistent_kernel(name, shape, kv_lens, gamma):
+    """The persistent kernel's tcgen05 attention phase (64-key tiles through the shared ring, three issuing threads),
+    forced on whatever the cache lengths, against the oracle and against the mma.sync phase on the same inputs."""
+    case = harness.Case(shape, torch.bfloat16, kv_lens, gamma, seed=8, cache="fill",
+                        gen_device="cuda").gpu_setup(max_rows=len(kv_lens) * (gamma + 1))
+    try:
+        for mode, T in [(orc.GREEDY, 1.0), (orc.SAMPLING, 1.0)]:
+            rep, g = _run(case, mode, T, options={"gemm_impl": 1, "step_impl": 1, "attn_impl": 2, "attn_tcgen05_min_tiles": 0})
+            assert rep.exact + rep.margin == len(kv_lens)
+            rep1, g1 = _run(case, mode, T, options={"gemm_impl": 1, "step_impl": 1, "attn_impl": 1})
+            d = np.abs(g["hidden"] - g1["hidden"]).max()
+            assert 0 < d < 5e-3 or max(kv_lens) == 0   # close, and not the same code path
+            print(name, "mode", mode, rep, "vs mma.sync", d)
+    finally:
+        case.close()
+
+
 def test_more_than_256_rows_keep_both_activation_planes():
     """29 sequences x 9 rows = 261 rows: the two bf16 activation planes no longer fit side by side in tensor
     memory and the lo plane is accumulated into the hi plane's columns."""
