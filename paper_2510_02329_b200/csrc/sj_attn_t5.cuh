@@ -14,16 +14,18 @@
 //               log2 domain: then the thread rescales its row of O), and writes P = exp2(S - m) over the scores it
 //               has just read, as two bf16 terms per 32-key chunk ([hi 16 columns | lo 16 columns]).  S is double-
 //               buffered, so the next tile's scores are computed while this tile's P V runs.
-//   O += P V    A = P from tensor memory (M = 128 slots, K = 16 keys per step = one page), B = the page's V rows
+//   O += P V    (two accumulators, one for the even and one for the odd tiles: each has its own issuing thread; they are
+//               added when the segment ends)  A = P from tensor memory (M = 128 slots, K = 16 keys per step = one page), B = the page's V rows
 //               as an MN-major operand (the head dim is the contiguous one: leading byte offset = the 16 KiB
 //               between the two halves, stride byte offset = the 1 KiB between 8-key groups), N = head dim.
 // A segment (the block's run of tiles of one (sequence, KV head)) ends with the unnormalised partial (m, l, o)
 // per query row, in the format of sj_attn_tc.cuh, whose combine pass merges them; the block's own gamma+1 rows
-// (the causal tail) are handled by two extra warps with that file's mma.sync routine.
+// (the causal tail) are handled with that file's mma.sync routine.
 //
-// Roles (384 threads): warps 0 and 11 TMA producers (keys, values), warp 1 MMA issuer (owns tensor memory: S twice,
-// O = 384 of the 512 columns it allocates), warps 2..9 softmax (two threads per query row, TMEM lane quarter =
-// warp % 4), warp 10 tails.  Every wait is bounded.
+// Roles (384 threads): warp 0 TMA producer of the key tiles, warp 11 of the value tiles (sixteen lanes each), warps 1
+// and 10 issue the MMAs of the even and the odd tiles (warp 1 owns tensor memory: S twice, O twice = all 512 columns),
+// warps 2..9 softmax (two threads per query row, TMEM lane quarter = warp % 4) and, after their tiles, the causal tails.
+// Every wait is bounded.
 #pragma once
 
 #include "sj_attn_tc.cuh"
@@ -161,15 +163,17 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
   const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
   att_fill_pages(ctl->pages, pl, kv, args, B, kT5Keys, t_lo, t_hi, threadIdx.x, blockDim.x);
   __syncthreads();
-  const uint32_t tmem = ctl->tmem_base;   // columns: [0,256) S twice (P overwrites S in place), [256,384) O
+  const uint32_t tmem = ctl->tmem_base;   // columns: [0,256) S twice (P overwrites S in place), [256,512) O twice (one per issuer)
   volatile int* abort_flag = &ctl->abort_flag;
 
   if (warp == 0 || warp == 11) {
     // ------------------------------ TMA producers: warp 0 the key tiles, warp 11 the value tiles ------------------------------
-    // (two threads, so that the key tiles, which the scores need first, never queue behind a value stage that is
-    // still waiting for its P V)
-    if (lane == 0) {
-      const int which = warp == 0 ? 0 : 1;
+    // Two warps, so that the key tiles, which the scores need first, never queue behind a value stage that is still
+    // waiting for its P V.  A tile is sixteen boxes of 2 KiB (16 keys x 64 dims: a page's slots, one swizzle span
+    // wide) and one thread gets a copy out only every 200 clocks or so: sixteen lanes issue one box each (half =
+    // lane / 8, page = lane % 8), all in the same flow; lane 0 announces the bytes.
+    if (lane < 16) {
+      const int which = warp == 0 ? 0 : 1, half = lane >> 3, p = lane & 7;
       uint64_t* full = which ? ctl->vfull : ctl->kfull;
       uint64_t* empty = which ? ctl->vempty : ctl->kempty;
       uint8_t* base = which ? sV : sK;
@@ -177,71 +181,68 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       for (long long t = t_lo; t < t_hi; ++t, ++g) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
         const int st = g & 1, seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
+        int pi = x.ti * 8 + p;
+        if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
+        const int page = (g + 1) * 8 <= kAttPageCache ? ctl->pages[g * 8 + p]
+                                                      : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+        const long long row = ((((long long)a.layer * kv.n_pages + page) * 2 + which) * kv.n_kv_heads + x.h) * 16;
         if (g >= 2 && !t5_wait(&empty[st], (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 1)) break;
         const uint32_t bar = att_smem_u32(&full[st]);
         const uint32_t dst = att_smem_u32(base + (size_t)st * kT5TileBytes);
-        att_mbar_expect_tx(bar, kT5TileBytes);
-        for (int p = 0; p < 8; ++p) {
-          int pi = x.ti * 8 + p;
-          if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
-          const int page = (g + 1) * 8 <= kAttPageCache ? ctl->pages[g * 8 + p]
-                                                        : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
-          const long long row = ((((long long)a.layer * kv.n_pages + page) * 2 + which) * kv.n_kv_heads + x.h) * 16;
-          att_tma_2d(dst + (uint32_t)(p * 2048), &tmKV, bar, 0, (int)row);
-          att_tma_2d(dst + 16384u + (uint32_t)(p * 2048), &tmKV, bar, 64, (int)row);
-        }
+        if (lane == 0) att_mbar_expect_tx(bar, kT5TileBytes);
+        att_tma_2d(dst + (uint32_t)(half * 16384 + p * 2048), &tmKV, bar, half * 64, (int)row);
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+  } else if (warp == 1 || warp == 10) {
+    // ------------------------------ MMA issuers: warp 1 the even tiles, warp 10 the odd ones ------------------------------
+    // One thread gets a tcgen05.mma out every 110 clocks or so whatever its shape, and a tile needs 16 for the scores
+    // and 16 for the output; a second issuing thread doubles the rate.  The split is by tile parity: thread X owns
+    // stage X of the key and value tiles, score buffer X and an output accumulator of its own (O_X; the two share the
+    // rows' stabiliser and are added when the segment ends).  Within a thread the order is scores(g), output(g),
+    // scores(g + 2): the tensor pipe executes one thread's MMAs in issue order, which is all the ordering the reuse of
+    // score buffer X needs, and while the thread waits for the probabilities of its tile the other one issues.
     if (lane == 0) {
+      const int X = warp == 1 ? 0 : 1;
       const uint32_t id_s = instr_desc_bf16_mn(kT5Keys, 0), id_o = instr_desc_bf16_mn(HD, 1);
-      const uint32_t q0 = att_smem_u32(sQ), k0 = att_smem_u32(sK), v0 = att_smem_u32(sV);
+      const uint64_t dq = smem_desc_sw128(att_smem_u32(sQ)), dql = smem_desc_sw128(att_smem_u32(sQ) + kT5TileBytes);
+      const uint64_t dk = smem_desc_sw128(att_smem_u32(sK) + (uint32_t)X * kT5TileBytes);
+      const uint64_t dv = smem_desc_mn_sw128(att_smem_u32(sV) + (uint32_t)X * kT5TileBytes, 16384u);
+      const uint32_t d_s = tmem + (uint32_t)(X * 128), d_o = tmem + (uint32_t)(256 + X * 128);
       int it = 0, seg = 0;
       long long t = t_lo;
       bool alive = true;
       while (t < t_hi && alive) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
         const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-        const bool okq = t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2);
-        if (!okq) break;
-        tc_fence_after();
-        for (int i = 0; i <= n && alive; ++i) {
-          if (i < n) {   // scores of tile i
-            const int g = it + i, st = g & 1;
-            // S buffer `st` still holds P of tile g - 2 for that tile's P V, which this thread issued earlier: the
-            // tensor pipe executes one thread's MMAs in issue order, so these may overwrite it
-            const bool okk = t5_wait(&ctl->kfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 3);
-            if (!okk) { alive = false; break; }
-            tc_fence_after();
-            const uint32_t kb = k0 + (uint32_t)st * kT5TileBytes, d_s = tmem + (uint32_t)(st * 128);
+        bool first = true;
+        // every segment's queries are waited for, also where this thread owns none of its tiles: a parity wait that
+        // skipped a phase would be satisfied one phase early
+        if (!t5_wait(&ctl->q_ready, (uint32_t)seg & 1u, ctl, w.status, 2)) break;
+        for (int i = ((it & 1) == X) ? 0 : 1; i < n; i += 2) {
+          const int g = it + i;
+          const uint32_t par = (uint32_t)(g >> 1) & 1u;
+          if (!t5_wait(&ctl->kfull[X], par, ctl, w.status, 3)) { alive = false; break; }
+          tc_fence_after();
 #pragma unroll
-            for (int k = 0; k < HD / 16; ++k) {
-              const uint32_t off = (uint32_t)((k >> 2) * 16384 + (k & 3) * 32);
-              const uint64_t db = smem_desc_sw128(kb + off);
-              tc_mma_bf16(d_s, smem_desc_sw128(q0 + off), db, id_s, k > 0 ? 1u : 0u);
-              tc_mma_bf16(d_s, smem_desc_sw128(q0 + kT5TileBytes + off), db, id_s, 1u);
-            }
-            tc_commit(att_smem_u32(&ctl->kempty[st]));
-            tc_commit(att_smem_u32(&ctl->s_full[st]));
+          for (int k = 0; k < HD / 16; ++k) {
+            const uint64_t off = (uint64_t)((k >> 2) * (16384 >> 4) + (k & 3) * 2);   // start-address field, 16-byte units
+            tc_mma_bf16(d_s, dq + off, dk + off, id_s, k > 0 ? 1u : 0u);
+            tc_mma_bf16(d_s, dql + off, dk + off, id_s, 1u);
           }
-          if (i >= 1) {  // output of tile i - 1
-            const int g = it + i - 1, st = g & 1;
-            const bool okp = t5_wait(&ctl->p_full[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 5);
-            const bool okv = okp && t5_wait(&ctl->vfull[st], (uint32_t)(g >> 1) & 1u, ctl, w.status, 6);
-            if (!okv) { alive = false; break; }
-            tc_fence_after();
-            const uint32_t vb = v0 + (uint32_t)st * kT5TileBytes, pb = tmem + (uint32_t)(st * 128);
+          tc_commit(att_smem_u32(&ctl->kempty[X]));
+          tc_commit(att_smem_u32(&ctl->s_full[X]));
+          if (!t5_wait(&ctl->p_full[X], par, ctl, w.status, 5) || !t5_wait(&ctl->vfull[X], par, ctl, w.status, 6)) { alive = false; break; }
+          tc_fence_after();
 #pragma unroll
-            for (int pg = 0; pg < 8; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
-              const uint64_t db = smem_desc_mn_sw128(vb + (uint32_t)(pg * 2048), 16384u);
-              const uint32_t pa = pb + (uint32_t)(32 * (pg >> 1) + 8 * (pg & 1));
-              tc_mma_bf16_ta(tmem + 256, pa, db, id_o, (i > 1 || pg > 0) ? 1u : 0u);
-              tc_mma_bf16_ta(tmem + 256, pa + 16, db, id_o, 1u);
-            }
-            tc_commit(att_smem_u32(&ctl->vempty[st]));
-            tc_commit(att_smem_u32(&ctl->o_done[st]));
+          for (int pg = 0; pg < 8; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
+            const uint64_t db = dv + (uint64_t)(pg * (2048 >> 4));
+            const uint32_t pa = d_s + (uint32_t)(32 * (pg >> 1) + 8 * (pg & 1));
+            tc_mma_bf16_ta(d_o, pa, db, id_o, (!first || pg > 0) ? 1u : 0u);
+            tc_mma_bf16_ta(d_o, pa + 16, db, id_o, 1u);
           }
+          tc_commit(att_smem_u32(&ctl->vempty[X]));
+          tc_commit(att_smem_u32(&ctl->o_done[X]));
+          first = false;
         }
         it += n;
         t += n;
@@ -267,40 +268,49 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       ++pair_n;
       return __all_sync(0xffffffffu, ok);
     };
-    long long t = t_lo;
-    bool alive = true;
-    while (t < t_hi && alive) {
-      const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
-      const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-      // queries of this (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16
-      // terms; this thread converts its half of the head dimension
+    // queries of a (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16 terms;
+    // this thread converts its half of the head dimension (all loads first: one at a time they cost 0.4 us each)
+    auto deliver_q = [&](const AttTile& x) {
       if (active) {
-        const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD;
-        const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD : nullptr;
-        for (int d = 64 * half; d < 64 * half + 64; d += 8) {
-          const uint4 raw = __ldcg(reinterpret_cast<const uint4*>(qh + d));
-          uint4 rawl = make_uint4(0, 0, 0, 0);
-          if (ql) rawl = __ldcg(reinterpret_cast<const uint4*>(ql + d));
-          const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-          const __half2* l2 = reinterpret_cast<const __half2*>(&rawl);
+        const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD + 64 * half;
+        const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD + 64 * half : nullptr;
+        uint4 raw[8], rawl[8];
+#pragma unroll
+        for (int d8 = 0; d8 < 8; ++d8) {
+          raw[d8] = __ldcg(reinterpret_cast<const uint4*>(qh + 8 * d8));
+          rawl[d8] = ql ? __ldcg(reinterpret_cast<const uint4*>(ql + 8 * d8)) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int d8 = 0; d8 < 8; ++d8) {
+          const __half2* h2 = reinterpret_cast<const __half2*>(&raw[d8]);
+          const __half2* l2 = reinterpret_cast<const __half2*>(&rawl[d8]);
           uint32_t hi[4], lo[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             float2 v = __half22float2(h2[e]);
             const float2 vl = __half22float2(l2[e]);
-            v.x += vl.x; v.y += vl.y;
+            v.x += vl.x;
+            v.y += vl.y;
             const __nv_bfloat162 bh = __floats2bfloat162_rn(v.x, v.y);
             const float2 back = __bfloat1622float2(bh);
             const __nv_bfloat162 bl = __floats2bfloat162_rn(v.x - back.x, v.y - back.y);
             hi[e] = *reinterpret_cast<const uint32_t*>(&bh);
             lo[e] = *reinterpret_cast<const uint32_t*>(&bl);
           }
-          *reinterpret_cast<uint4*>(sQ + t5_q_off(sl, d)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(sQ + kT5TileBytes + t5_q_off(sl, d)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          const uint32_t off = t5_q_off(sl, 64 * half + 8 * d8);
+          *reinterpret_cast<uint4*>(sQ + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(sQ + kT5TileBytes + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read these generic-proxy stores
       att_mbar_arrive(att_smem_u32(&ctl->q_ready));
+    };
+    long long t = t_lo;
+    bool alive = true;
+    while (t < t_hi && alive) {
+      const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
+      const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+      if (seg == 0) deliver_q(x);   // later segments' queries were delivered while the segment before them ended
       float m_used = -INFINITY, l_sum = 0.f;
       for (int i = 0; i < n && alive; ++i) {
         const int g = it + i, sb = g & 1;
@@ -339,21 +349,27 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         if (m_used == -INFINITY) m_new = mx;
         else if (mx > m_used + 8.f) { m_new = mx; f = ex2_approx(m_used - m_new); }
         if (i > 0 && __any_sync(0xffffffffu, f != 1.f)) {
-          // rescale this thread's half of its row of O: only once the previous tile's P V has completed (this
-          // tile's cannot start before every thread has delivered its P)
+          // rescale this thread's half of its row of both output accumulators: the previous tile's, once its P V has
+          // completed (this tile's cannot start before every thread has delivered its P), and, from the segment's third
+          // tile on, this tile's own (its last P V completed before the scores just read were computed: same issuer)
           if (lane == 0) ok = t5_wait(&ctl->o_done[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, ctl, w.status, 8) ? 1 : 0;
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) { alive = false; break; }
           att_mbar_try(att_smem_u32(&ctl->o_done[(g - 1) & 1]), (uint32_t)((g - 1) >> 1) & 1u);
           tc_fence_after();
 #pragma unroll 1
-          for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
-            float o[32];
-            tc_ld32(lane_addr + 256 + c0, o);
+          for (int k = 0; k < (i >= 2 ? 2 : 1); ++k) {
+            const uint32_t o_addr = lane_addr + (uint32_t)(256 + 128 * ((g - 1 + k) & 1));
+#pragma unroll 1
+            for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+              float o[32];
+              tc_ld32(o_addr + c0, o);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] *= f;
-            tc_st32f(lane_addr + 256 + c0, o);
+              for (int j = 0; j < 32; ++j) o[j] *= f;
+              tc_st32f(o_addr + c0, o);
+            }
           }
+          tc_wait_st();
           l_sum *= f;
         }
         // probabilities as two bf16 terms, written over the scores: chunk of 32 keys -> [hi 16 columns | lo 16 columns];
@@ -379,14 +395,22 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         m_used = m_new;
       }
       if (!alive) break;
-      // the segment's partial: wait for the last P V, then (m, l, o) of every real query row
+      // The next segment's queries, before this one is wound up: every score MMA of this segment has completed (this
+      // thread saw the scores of its last tile), so the query tiles are free, and the issuers start on the next
+      // segment's scores while the partial below is read out (its first P V waits for probabilities that this thread
+      // delivers only afterwards, so the output accumulators are not touched early).
+      if (t + n < t_hi) deliver_q(att_locate(pl, B, kT5Keys, (int)(t + n)));
+      // the segment's partial: wait for the last P V of either issuer, then (m, l, o) of every real query row
       {
         const int g = it + n - 1;
         int ok = 1;
-        if (lane == 0) ok = t5_wait(&ctl->o_done[g & 1], (uint32_t)(g >> 1) & 1u, ctl, w.status, 9) ? 1 : 0;
+        if (lane == 0)
+          ok = (t5_wait(&ctl->o_done[g & 1], (uint32_t)(g >> 1) & 1u, ctl, w.status, 9) &&
+                (n < 2 || t5_wait(&ctl->o_done[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, ctl, w.status, 9))) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         att_mbar_try(att_smem_u32(&ctl->o_done[g & 1]), (uint32_t)(g >> 1) & 1u);
+        if (n >= 2) att_mbar_try(att_smem_u32(&ctl->o_done[(g - 1) & 1]), (uint32_t)((g - 1) >> 1) & 1u);
         tc_fence_after();
         ctl->mx[(g + 1) & 1][half][sl] = l_sum;           // the buffer the last tile did not use
         if (!pair_sync()) break;
@@ -396,7 +420,13 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
 #pragma unroll 1
         for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
           float o[32];
-          tc_ld32(lane_addr + 256 + c0, o);
+          tc_ld32(lane_addr + (uint32_t)(256 + 128 * (g & 1)) + c0, o);
+          if (n >= 2) {   // the other issuer's accumulator holds the other half of the segment's tiles
+            float o2[32];
+            tc_ld32(lane_addr + (uint32_t)(256 + 128 * ((g - 1) & 1)) + c0, o2);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] += o2[j];
+          }
           if (active) {
             float4* dst = reinterpret_cast<float4*>(a.P.o + (base + q) * HD + c0);
 #pragma unroll
@@ -410,12 +440,14 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       t += n;
       ++seg;
     }
-  } else if (warp < 11) {
-    // ------------------------------ tails: the block's own rows, one m-tile of one (sequence, KV head) per task ------------------------------
-    const AttGeom g = att_geom(HD, group, rows);
-    AttWarp<HD, 2> st;
-    for (int task = G - 1 - c; task < B * Hkv * g.MT; task += G)
-      att_tail_task<HD, 2>(st, g, a, task / g.MT, (task % g.MT) * 16, lane);
+    // the causal tails (the step's own rows as keys; mma.sync): one m-tile of one (sequence, KV head) per task, dealt
+    // over all blocks' softmax warps from the last block down
+    if (alive) {
+      const AttGeom g = att_geom(HD, group, rows);
+      AttWarp<HD, 2> st;
+      for (int task = (G - 1 - c) * 8 + (warp - 2); task < B * Hkv * g.MT; task += G * 8)
+        att_tail_task<HD, 2>(st, g, a, task / g.MT, (task % g.MT) * 16, lane);
+    }
   }
   tc_fence_before();
   __syncthreads();
