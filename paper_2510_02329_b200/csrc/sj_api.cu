@@ -986,13 +986,13 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
       if (dm.hd == 128 && t->opt_attn == 2 && nq <= 128) {   // one 128-lane accumulator holds a KV head's query rows
         const size_t t5_smem = kT5SmemBytes + sizeof(T5Ctl) + 1024;
         TIMED("attn", launch(k_attn_t5, dim3(t->sm_count), dim3(kT5Threads), t5_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, kT5Keys));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, kT5Keys, kT5Pad));
       } else if (dm.hd == 128) {
         TIMED("attn", launch(k_attn_tc<128>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0, 0));
       } else {
         TIMED("attn", launch(k_attn_tc<64>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<64>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0));
+        TIMED("attn_combine", launch(k_attn_combine_tc<64>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0, 0));
       }
     } else {
       TIMED("attn", launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));

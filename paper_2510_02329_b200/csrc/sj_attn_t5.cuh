@@ -34,6 +34,7 @@
 namespace sj {
 
 constexpr int kT5Keys = 128;               // keys per tile
+constexpr int kT5Pad = 5;                  // empty tiles the plan counts per (sequence, KV head): what a segment costs a block beyond its tiles
 constexpr int kT5Threads = 384;
 constexpr int kT5TileBytes = 32768;        // one K or V tile: 2 halves x 8 pages x 2 KiB
 constexpr int kT5SmemBytes = 2 * kT5TileBytes /* Q hi, lo */ + 4 * kT5TileBytes /* K, V double-buffered */;
@@ -148,7 +149,7 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
     ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 2) att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, kT5Keys, lane);
+  if (warp == 2) att_plan_fill(&ctl->plan, w.row_pos, B, rows, Hkv, kT5Keys, lane, kT5Pad);
   // unused query-row slots stay zero for the whole kernel
   for (int i = threadIdx.x; i < 2 * kT5TileBytes / 16; i += blockDim.x) reinterpret_cast<uint4*>(sQ)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 1) {
@@ -177,20 +178,22 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       uint64_t* full = which ? ctl->vfull : ctl->kfull;
       uint64_t* empty = which ? ctl->vempty : ctl->kempty;
       uint8_t* base = which ? sV : sK;
-      int g = 0;
-      for (long long t = t_lo; t < t_hi; ++t, ++g) {
+      int g = 0;   // real tiles so far
+      for (long long t = t_lo; t < t_hi; ++t) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
-        const int st = g & 1, seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
+        if (x.ti >= x.nt_real) continue;   // one of the plan's empty tiles
+        const int st = g & 1, seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16, tb = (int)(t - t_lo);
         int pi = x.ti * 8 + p;
         if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
-        const int page = (g + 1) * 8 <= kAttPageCache ? ctl->pages[g * 8 + p]
-                                                      : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
+        const int page = (tb + 1) * 8 <= kAttPageCache ? ctl->pages[tb * 8 + p]
+                                                       : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
         const long long row = ((((long long)a.layer * kv.n_pages + page) * 2 + which) * kv.n_kv_heads + x.h) * 16;
         if (g >= 2 && !t5_wait(&empty[st], (uint32_t)((g >> 1) - 1) & 1u, ctl, w.status, 1)) break;
         const uint32_t bar = att_smem_u32(&full[st]);
         const uint32_t dst = att_smem_u32(base + (size_t)st * kT5TileBytes);
         if (lane == 0) att_mbar_expect_tx(bar, kT5TileBytes);
         att_tma_2d(dst + (uint32_t)(half * 16384 + p * 2048), &tmKV, bar, half * 64, (int)row);
+        ++g;
       }
     }
   } else if (warp == 1 || warp == 10) {
@@ -213,7 +216,10 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       bool alive = true;
       while (t < t_hi && alive) {
         const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
-        const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+        const int nv = (int)min((long long)(x.nt_b - x.ti), t_hi - t);   // with the plan's empty tiles
+        const int n = max(0, min(nv, x.nt_real - x.ti));
+        t += nv;
+        if (n == 0) continue;   // only empty tiles of this (sequence, KV head): no segment
         bool first = true;
         // every segment's queries are waited for, also where this thread owns none of its tiles: a parity wait that
         // skipped a phase would be satisfied one phase early
@@ -245,7 +251,6 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
           first = false;
         }
         it += n;
-        t += n;
         ++seg;
       }
     }
@@ -307,9 +312,25 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
     };
     long long t = t_lo;
     bool alive = true;
+    // the block's next run of real tiles at or after tile t: (sequence, KV head, first tile), its length n, and nv,
+    // the same with the plan's empty tiles; n == 0 when only empty tiles are left of that (sequence, KV head)
+    auto run_at = [&](long long t, AttTile& x, int& n, int& nv) {
+      x = att_locate(pl, B, kT5Keys, (int)t);
+      nv = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+      n = max(0, min(nv, x.nt_real - x.ti));
+    };
     while (t < t_hi && alive) {
-      const AttTile x = att_locate(pl, B, kT5Keys, (int)t);
-      const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+      AttTile x;
+      int n, nv;
+      run_at(t, x, n, nv);
+      if (n == 0) {
+        // only empty tiles of this (sequence, KV head) fell to this block: the combine pass still reads the block's
+        // slot for it, so it gets a partial of weight zero (the stored outputs are finite: old values or zeros)
+        const size_t base = (((size_t)c + (size_t)x.b * Hkv + x.h) * kAttMaxSub + 0) * (size_t)nq;
+        if (active && half == 0) { a.P.m[base + q] = -INFINITY; a.P.l[base + q] = 0.f; }
+        t += nv;
+        continue;
+      }
       if (seg == 0) deliver_q(x);   // later segments' queries were delivered while the segment before them ended
       float m_used = -INFINITY, l_sum = 0.f;
       for (int i = 0; i < n && alive; ++i) {
@@ -330,17 +351,14 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
 #pragma unroll
           for (int j = 0; j < 64; ++j) sc[j] = 0.f;
         }
-        float mx = -INFINITY;
-        if (n_valid >= 64) {   // warp-uniform; every tile but a sequence's last
+        if (n_valid < 64) {   // warp-uniform; only a sequence's last tile
 #pragma unroll
-          for (int j = 0; j < 64; ++j) mx = fmaxf(mx, sc[j]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 64; ++j) {
-            sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
-            mx = fmaxf(mx, sc[j]);
-          }
+          for (int j = 0; j < 64; ++j) sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
         }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains: a single one is 64 dependent steps
+#pragma unroll
+        for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         ctl->mx[g & 1][half][sl] = mx;
         if (!pair_sync()) { alive = false; break; }
         mx = fmaxf(mx, ctl->mx[g & 1][half ^ 1][sl]);
@@ -374,13 +392,14 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         }
         // probabilities as two bf16 terms, written over the scores: chunk of 32 keys -> [hi 16 columns | lo 16 columns];
         // hi = p truncated to bf16, lo = the rest rounded to bf16 (16 significant bits in all)
+        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 32) {
           uint32_t hi[16], lo[16];
 #pragma unroll
           for (int j = 0; j < 32; j += 2) {
             const float p0 = ex2_approx(sc[c0 + j] - m_new), p1 = ex2_approx(sc[c0 + j + 1] - m_new);   // 0 for masked keys
-            l_sum += p0 + p1;
+            ls4[(j >> 1) & 3] += p0 + p1;
             const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
             hi[j >> 1] = __byte_perm(b0, b1, 0x7632);
             const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - __uint_as_float(b0 & 0xffff0000u), p1 - __uint_as_float(b1 & 0xffff0000u));
@@ -389,6 +408,7 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
           tc_st16(s_addr + (uint32_t)c0, hi);
           tc_st16(s_addr + (uint32_t)c0 + 16, lo);
         }
+        l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
         tc_wait_st();
         tc_fence_before();
         att_mbar_arrive(att_smem_u32(&ctl->p_full[sb]));
@@ -399,7 +419,13 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
       // thread saw the scores of its last tile), so the query tiles are free, and the issuers start on the next
       // segment's scores while the partial below is read out (its first P V waits for probabilities that this thread
       // delivers only afterwards, so the output accumulators are not touched early).
-      if (t + n < t_hi) deliver_q(att_locate(pl, B, kT5Keys, (int)(t + n)));
+      for (long long t2 = t + nv; t2 < t_hi;) {
+        AttTile x2;
+        int n2, nv2;
+        run_at(t2, x2, n2, nv2);
+        if (n2 > 0) { deliver_q(x2); break; }
+        t2 += nv2;
+      }
       // the segment's partial: wait for the last P V of either issuer, then (m, l, o) of every real query row
       {
         const int g = it + n - 1;
@@ -437,7 +463,7 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
         if (!pair_sync()) break;   // the sums have been read before the next segment's first tile reuses the buffer
       }
       it += n;
-      t += n;
+      t += nv;
       ++seg;
     }
     // the causal tails (the step's own rows as keys; mma.sync): one m-tile of one (sequence, KV head) per task, dealt
@@ -737,17 +763,14 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
 #pragma unroll
         for (int j = 0; j < 32; ++j) sc[j] = 0.f;
       }
-      float m_tile = -INFINITY;
-      if (n_valid >= 32) {   // warp-uniform; every tile but a sequence's last
+      if (n_valid < 32) {   // warp-uniform; only a sequence's last tile
 #pragma unroll
-        for (int j = 0; j < 32; ++j) m_tile = fmaxf(m_tile, sc[j]);
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
-          m_tile = fmaxf(m_tile, sc[j]);
-        }
+        for (int j = 0; j < 32; ++j) sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
       }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains: a single one is 32 dependent steps
+#pragma unroll
+      for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+      float m_tile = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       mx_own[128 * sb] = m_tile;
       if (!pair_sync()) return false;
       m_tile = fmaxf(m_tile, mx_other[128 * sb]);
@@ -778,15 +801,17 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
       // lo = the rest rounded to bf16 (16 significant bits in all)
       {
         uint32_t hi[16], lo[16];
+        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
           const float p0 = ex2_approx(sc[j] - m_new), p1 = ex2_approx(sc[j + 1] - m_new);   // 0 for masked keys
-          l_sum += p0 + p1;
+          ls4[(j >> 1) & 3] += p0 + p1;
           const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
           hi[j >> 1] = __byte_perm(b0, b1, 0x7632);
           const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - __uint_as_float(b0 & 0xffff0000u), p1 - __uint_as_float(b1 & 0xffff0000u));
           lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&bl);
         }
+        l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
         tc_st16(s_addr, hi);
         tc_st16(s_addr + 16, lo);
       }

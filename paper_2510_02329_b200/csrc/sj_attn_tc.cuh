@@ -377,18 +377,23 @@ struct AttPlan {
   int L[kMaxBatch];          // cached keys per sequence
   int pre[kMaxBatch + 1];    // ring tiles before sequence b (all KV heads)
   long long T;               // total ring tiles
+  // Empty tiles counted after the real ones of every (sequence, KV head) with a non-empty cache.  Tiles are dealt to
+  // blocks in equal numbers, and a block pays a fixed price for every (sequence, KV head) it touches (queries, the
+  // pipeline's start and drain, the partial): counting that price in tiles keeps ragged batches balanced.  Nobody
+  // loads or computes an empty tile.
+  int pad;
 };
 
 // Filled by one full warp (every lane calls it); callers synchronise afterwards.  Lane i takes sequences i, i + 32, ...:
 // the cache lengths are loaded side by side (one thread alone would wait for each load in turn, half a microsecond
 // apiece at a batch of 32) and the tile counts summed by a warp prefix sum.
 __device__ __forceinline__ void att_plan_fill(AttPlan* pl, const int* __restrict__ row_pos, int B, int rows, int Hkv,
-                                              int KPS, int lane) {
+                                              int KPS, int lane, int pad = 0) {
   int carry = 0;
   for (int b0 = 0; b0 < B; b0 += 32) {
     const int b = b0 + lane;
     const int L = b < B ? row_pos[b * rows] : 0;
-    const int n = b < B ? Hkv * ((L + KPS - 1) / KPS) : 0;
+    const int n = (b < B && L > 0) ? Hkv * ((L + KPS - 1) / KPS + pad) : 0;
     int incl = n;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
@@ -404,6 +409,7 @@ __device__ __forceinline__ void att_plan_fill(AttPlan* pl, const int* __restrict
   if (lane == 0) {
     pl->pre[B] = carry;
     pl->T = carry;
+    pl->pad = pad;
   }
 }
 
@@ -512,12 +518,13 @@ __device__ __forceinline__ void att_issue_tile(const CUtensorMap* tmKV, const Kv
 }
 
 // Map ring tile t to (sequence, KV head, tile index, tiles of that (sequence, head)).
-struct AttTile { int b, h, ti, nt_b, L; };
+struct AttTile { int b, h, ti, nt_b, L, nt_real; };   // nt_b counts the plan's empty tiles, nt_real does not
 __device__ __forceinline__ AttTile att_locate(const AttPlan& pl, int B, int KPS, int t) {
   AttTile x;
   x.b = att_find_seq(pl.pre, B, t);
   x.L = pl.L[x.b];
-  x.nt_b = (x.L + KPS - 1) / KPS;
+  x.nt_real = (x.L + KPS - 1) / KPS;
+  x.nt_b = x.nt_real + pl.pad;
   const int rem = t - pl.pre[x.b];
   x.h = rem / x.nt_b;
   x.ti = rem % x.nt_b;
@@ -745,7 +752,7 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
   const int item = item_part / SPLIT, part = item_part % SPLIT;
   const int q = item % g.nq, bh = item / g.nq, b = bh / Hkv, h = bh % Hkv;
   const int L = pl.L[b];
-  const int nt_b = (L + g.KPS - 1) / g.KPS;
+  const int nt_b = L > 0 ? (L + g.KPS - 1) / g.KPS + pl.pad : 0;
   int c_first = 0, n_cta = 0;
   if (nt_b > 0) {
     const long long t0 = (long long)pl.pre[b] + (long long)h * nt_b;
@@ -832,18 +839,19 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
   for (int i = 0; i < DPL; ++i) store_act<T>(ATT, R, Hq * HD, r, head * HD + (part * 32 + lane) * DPL + i, acc[i] * inv);
 }
 
-// keys_per_tile > 0: the partials come from a pass that cut the cache into tiles of that many keys with one
-// sub-partial per block segment (the tcgen05 attention); 0: this file's own geometry.
+// keys_per_tile > 0: the partials come from a pass that cut the cache into tiles of that many keys (plus tile_pad empty
+// ones per (sequence, KV head)) with one sub-partial per block segment (the tcgen05 attention); 0: this file's own
+// geometry.
 template <int HD>
 __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dims dm, AttPartials P, int G_att,
-                                  int n_tail_base, int keys_per_tile) {
+                                  int n_tail_base, int keys_per_tile, int tile_pad) {
   __shared__ AttPlan pl;
   pdl_wait();
   pdl_launch();
   const int B = args->B, rows = args->gamma + 1;
   AttGeom g = att_geom(HD, dm.Hq / dm.Hkv, rows);
   if (keys_per_tile > 0) { g.KPS = keys_per_tile; g.KS = 1; g.KW = keys_per_tile; }
-  if (threadIdx.x < 32) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS, threadIdx.x);
+  if (threadIdx.x < 32) att_plan_fill(&pl, w.row_pos, B, rows, dm.Hkv, g.KPS, threadIdx.x, keys_per_tile > 0 ? tile_pad : 0);
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
   const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;

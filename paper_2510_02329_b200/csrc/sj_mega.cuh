@@ -996,6 +996,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     }
     ctl->plan.pre[B] = acc;
     ctl->plan.T = acc;
+    ctl->plan.pad = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
