@@ -41,7 +41,7 @@ UNIT = "tokens/s"
 # workload's shape (summaries under profiles/); traffic grows in proportion to the streamed bytes (nothing is
 # re-read), so a full step's traffic is this ratio times its algorithmic bytes.  A workload without a capture
 # of the kernel as it stands has no entry and reports null.
-MEGA_DRAM_TRAFFIC_RATIO = {"cfg3": 1.0091}   # profiles/k_verify_mega_cfg3_4layers_full.md
+MEGA_DRAM_TRAFFIC_RATIO = {"cfg3": 1.0088}   # profiles/k_verify_mega_cfg3_4layers_full.md
 
 
 def measured_peaks():
