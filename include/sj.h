@@ -103,9 +103,10 @@ sj_status sj_load_judge_head(sj_target *t, const float *w_host, float bias, floa
  *                2 = tcgen05 kernel (bf16 models, head_dim 128, at most 128 query rows per KV head and sequence, else
  *                it runs as 1); default: 2 at head_dim 128, else 1, for bf16 models; 0 for fp32 models.  The
  *                persistent kernel's attention phase is the tcgen05 one when this is 2, head_dim is 128, a KV
- *                head has at most 64 query rows per sequence and the step's caches hold at least
- *                "attn_tcgen05_min_tiles" 64-key tiles per thread block; else the mma.sync one.
- *   "attn_tcgen05_min_tiles"  n >= 0 (default 8; 0 = always): see "attn_impl"
+ *                head has at most 64 query rows per sequence, the block has at least 49 rows (its ring stages then
+ *                hold a 32 KiB key tile) and the step's caches hold at least "attn_tcgen05_min_tiles" 128-key
+ *                tiles per thread block; else the mma.sync one.
+ *   "attn_tcgen05_min_tiles"  n >= 0 (default 4; 0 = always): see "attn_impl"
  *   "step_impl"  1 = the whole step as one persistent cooperative kernel (bf16, tcgen05 GEMMs, at most 80
  *                block rows; default when the shape allows), 0 = one kernel per stage
  *   "attn_two_term_layers"  n >= 0 (default 1): in layers [0, n) the tensor-core attention carries queries and

@@ -210,7 +210,7 @@ struct sj_target {
   double* d_inv_freq = nullptr;
   float theta = 0.5f, judge_bias = 0.f;
   bool has_judge = false;
-  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_att_precise = 1, opt_a5_min_tiles = 8;
+  int opt_gemm = 0, opt_attn = 0, opt_graph = 1, opt_pdl = 1, opt_timing = 0, opt_step = 0, opt_trace = 0, opt_ring = 0, opt_att_precise = 1, opt_a5_min_tiles = 4;
   bool mega_shapes = false, coop = false;
   MegaLayerPtrs* d_layer_ptrs = nullptr;
   float* d_sumsq = nullptr;
@@ -986,13 +986,13 @@ static sj_status enqueue_step(sj_target* t, sj_kv* kv, int B, int gamma, int mod
       if (dm.hd == 128 && t->opt_attn == 2 && nq <= 128) {   // one 128-lane accumulator holds a KV head's query rows
         const size_t t5_smem = kT5SmemBytes + sizeof(T5Ctl) + 1024;
         TIMED("attn", launch(k_attn_t5, dim3(t->sm_count), dim3(kT5Threads), t5_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, kT5Keys, kT5Pad));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128, 8>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, kT5Keys, kT5Pad));
       } else if (dm.hd == 128) {
         TIMED("attn", launch(k_attn_tc<128>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<128>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0, 0));
+        TIMED("attn_combine", launch(k_attn_combine_tc<128, 0>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0, 0));
       } else {
         TIMED("attn", launch(k_attn_tc<64>, dim3(t->sm_count), dim3(kAttTcThreads), tc_smem, s, pdl, kv->tm_pool, args, kv->view, W, dm, aa));
-        TIMED("attn_combine", launch(k_attn_combine_tc<64>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0, 0));
+        TIMED("attn_combine", launch(k_attn_combine_tc<64, 0>, dim3(cgrid), dim3(256), 0, s, pdl, args, W, dm, parts, t->sm_count, aa.n_tail_base, 0, 0));
       }
     } else {
       TIMED("attn", launch(k_attn_simt<T>, dim3(att_grid), dim3(kAttThreads), att_smem, s, pdl, args, kv->view, W, dm, l, chunk_len));
@@ -1074,14 +1074,15 @@ static sj_status launch_mega(sj_target* t, sj_kv* kv, int B, int gamma, int mode
   memset(&p, 0, sizeof(p));
   p.B = B; p.rows = rows; p.R = R; p.Rp = Rp;
   p.stage_bytes = kWTileBytes + round_up(2 * Rp * 128, 1024);
-  // tcgen05 attention phase: head dimension 128, a KV head's query rows within two TMEM lane quarters, and caches long
-  // enough that the phase is bound by throughput (at a few tiles per block it is a chain of latencies, and the
-  // mma.sync phase, which needs no hand-over between warps, is as fast)
+  // tcgen05 attention phase: head dimension 128, a KV head's query rows within two TMEM lane quarters, ring stages
+  // that hold a 32 KiB key or value tile (49 block rows or more), and caches long enough that the phase is bound by
+  // throughput (at a few tiles per block it is a chain of latencies, and the mma.sync phase, which needs no hand-over
+  // between warps, is as fast)
   const int nq = (dm.Hq / dm.Hkv) * rows;
   const long tiles_per_block = total_keys * dm.Hkv / kA5Keys / t->sm_count;
-  const bool a5 = dm.hd == 128 && nq <= kA5MaxRows && t->opt_attn == 2 && tiles_per_block >= t->opt_a5_min_tiles;
+  const bool a5 = dm.hd == 128 && nq <= kA5MaxRows && t->opt_attn == 2 && p.stage_bytes >= (int)kA5Part &&
+                  tiles_per_block >= t->opt_a5_min_tiles;
   p.q_area_bytes = a5 ? a5_q_area_bytes(nq) : 0;
-  p.att_spe = p.stage_bytes >= 2 * (int)kA5Part ? 1 : 2;
   const int ctl_bytes = ((int)sizeof(MegaCtl) + 127) & ~127;
   const int budget = 227 * 1024 - 1024 - ctl_bytes - p.q_area_bytes;
   p.stages = std::min(8, std::min(kMegaMaxStages, budget / p.stage_bytes));   // deeper rings did not measure faster; the rest stays L1

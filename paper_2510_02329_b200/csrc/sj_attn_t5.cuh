@@ -487,40 +487,36 @@ k_attn_t5(const __grid_constant__ CUtensorMap tmKV, const StepArgs* __restrict__
 
 // =============================================================================================
 // The same attention as phase routines of a kernel whose shared-memory ring also carries other traffic (the
-// persistent step kernel): 64-key tiles, the queries in an area of their own, at most 64 query rows per
-// (sequence, KV head).
+// persistent step kernel), for at most 64 query rows per (sequence, KV head) and ring stages of at least 32 KiB.
 //
-// A tile is one ring entry, key part then value part of 16 KiB each ([half][page][16 keys x 128 B], as above with
-// four pages): in ONE stage when a stage holds 32 KiB, else in two consecutive stages (key stage, value stage; each
-// has its own full / empty barrier).  Query row q sits in TMEM lane q and in row q of the query area, which holds
-// pad8(nq) rows per 64-dim half: the MMAs run at M = 128 all the same, their rows beyond the area read whatever
-// shared memory follows it (the caller guarantees 16 KiB of its own allocation after the last half's base) and
-// produce accumulator lanes nobody reads.
+// A 128-key tile is two ring entries, the key tile and then the value tile, one stage each ([half][page][16 keys x
+// 128 B] as above; each stage has its own full / empty barrier).  Query row q sits in TMEM lane q and in row q of a
+// query area of its own, which holds pad8(nq) rows per 64-dim half: the MMAs run at M = 128 all the same, their rows
+// beyond the area read whatever shared memory follows it (the caller guarantees 16 KiB of its own allocation after the
+// last half's base) and produce accumulator lanes nobody reads; so only the lane quarters 0 and 1 carry rows, and four
+// warps run the softmax (two threads per row, 64 keys each).
 //
-// Three issuing threads.  One thread gets a tcgen05.mma out every 110 clocks or so whatever its shape (measured: M 64 or
-// 128, N 32..128, operand A in shared or tensor memory; two threads issue twice as many), and a tile needs 8 k-steps x 2
-// query planes for the scores and 4 pages x 2 probability planes for the output.  So the scores are two accumulators,
-// S_hi = Q_hi K^T and S_lo = Q_lo K^T, each with a thread of its own (the softmax adds them), and a third thread issues
-// the output MMAs: 8 MMAs per tile and thread.  Tensor memory: S_hi twice at columns [0, 128) (the probabilities are
-// written over it), S_lo twice at [128, 256), the output at [256, 384), aliasing whatever the kernel keeps there outside
-// the attention phase.
+// Two issuing threads, split by tile parity as in the kernel above: thread X owns score buffer X (columns
+// [128 X, +128); the probabilities are written over it) and output accumulator X (columns [256 + 128 X, +128)), issues
+// scores(g), output(g), scores(g + 2) in that order, and the softmax adds the two accumulators when the segment ends.
+// All 512 columns alias whatever the kernel keeps there outside the attention phase.
 // =============================================================================================
-constexpr int kA5Keys = 64;
+constexpr int kA5Keys = 128;
 constexpr int kA5MaxRows = 64;
-constexpr uint32_t kA5Part = 16384;
+constexpr uint32_t kA5Part = 32768;   // bytes of a key tile or a value tile: the least a ring stage must hold
 constexpr int kA5TmemCols = 512;
 
 struct A5Bars {
-  uint64_t s_full[2];   // two arrivals: the commits of both score issuers
+  uint64_t s_full[2];   // one arrival: issuer X's commit after the score MMAs
   uint64_t p_full[2];   // 128 arrivals: the softmax threads
-  uint64_t o_done[2];   // one arrival: the output issuer's commit
+  uint64_t o_done[2];   // one arrival: issuer X's commit after the output MMAs
   uint64_t q_ready;     // 128 arrivals
 };
 struct A5Ring {
   uint64_t* full;    // [stages], each completes on two arrivals (the expecting one and a second)
   uint64_t* empty;   // [stages], one arrival
   uint8_t* base;
-  int stage_stride, stages, spe;   // spe: stages per entry (1 or 2)
+  int stage_stride, stages;
   volatile int* abort_flag;
   volatile int* abort_g;
   int* status;
@@ -533,26 +529,20 @@ struct A5Pos {
 };
 struct A5Entry {
   int s0, s1;
-  uint32_t par0, par1, a0, a1;   // stage, parity of this use and address of the key part (0) and the value part (1)
+  uint32_t par0, par1, a0, a1;   // stage, parity of this use and address of the key tile (0) and the value tile (1)
 };
 __host__ __device__ __forceinline__ int a5_q_half_bytes(int nq) { return ((nq + 7) & ~7) * 128; }
 __host__ __device__ __forceinline__ int a5_q_area_bytes(int nq) { return 4 * a5_q_half_bytes(nq); }   // two planes x two halves
 
-__device__ __forceinline__ A5Entry a5_entry(const A5Ring& rg, A5Pos& pos) {   // the entry at pos; pos moves past it
+__device__ __forceinline__ A5Entry a5_entry(const A5Ring& rg, A5Pos& pos) {   // the tile at pos; pos moves past it
   A5Entry e;
   e.s0 = pos.s;
   e.par0 = (uint32_t)pos.r & 1u;
   e.a0 = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
-  if (rg.spe == 2) {
-    pos.next(rg.stages);
-    e.s1 = pos.s;
-    e.par1 = (uint32_t)pos.r & 1u;
-    e.a1 = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
-  } else {
-    e.s1 = e.s0;
-    e.par1 = e.par0;
-    e.a1 = e.a0 + kA5Part;
-  }
+  pos.next(rg.stages);
+  e.s1 = pos.s;
+  e.par1 = (uint32_t)pos.r & 1u;
+  e.a1 = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
   pos.next(rg.stages);
   return e;
 }
@@ -560,109 +550,96 @@ __device__ __forceinline__ bool a5_wait(const A5Ring& rg, uint64_t* bar, uint32_
   return att_mbar_wait(att_smem_u32(bar), parity, rg.abort_flag, rg.status, rg.abort_g, where, extra);
 }
 
-// Sixteen lanes of one warp (pl_lane 0..15, all in the same control flow): the TMA loads of the block's tiles
-// [t_lo, t_hi) of one layer.  A tile is sixteen boxes of 2 KiB (16 keys x 64 dims: a page's slots, one swizzle span wide),
-// and one thread gets a copy out only every 200 clocks or so, far below what the tile's 32 KiB need; so every lane
-// issues ONE box of each tile (part = lane / 8, half = lane / 4 % 2, page = lane % 4) and a tile costs one instruction.
-// Lane 0 announces the bytes.  pages: the block's page ids, four per tile (clamped to the sequence's last page), for
-// its first kAttPageCache / 4 tiles.
+// All 32 lanes of one warp (same control flow): the TMA loads of the block's tiles [t_lo, t_hi) of one layer.  A tile
+// is sixteen boxes of 2 KiB for the keys and sixteen for the values (16 keys x 64 dims: a page's slots, one swizzle
+// span wide), and one thread gets a copy out only every 200 clocks or so: every lane issues ONE box of each tile (lanes
+// 0..15 keys, 16..31 values; half = lane / 8 % 2, page = lane % 8), so a tile costs one instruction.  Lane 0 announces
+// the bytes.  pages: the block's page ids, eight per tile (clamped to the sequence's last page), for its first
+// kAttPageCache / 8 tiles.
 __device__ __forceinline__ bool a5_produce(const A5Ring& rg, A5Pos& pos, const CUtensorMap* tmKV, const KvView& kv,
                                            const StepArgs* __restrict__ args, const AttPlan& pl, int B, int layer,
-                                           long long t_lo, long long t_hi, const int* pages, int pl_lane) {
-  const int which = pl_lane >> 3, half = (pl_lane >> 2) & 1, p = pl_lane & 3;
+                                           long long t_lo, long long t_hi, const int* pages, int lane) {
+  const int which = lane >> 4, half = (lane >> 3) & 1, p = lane & 7;
   int tb = 0;
   for (long long t = t_lo; t < t_hi; ++t, ++tb) {
     const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
     const int seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
-    int pi = x.ti * 4 + p;
+    int pi = x.ti * 8 + p;
     if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
-    const int page = (tb + 1) * 4 <= kAttPageCache ? pages[tb * 4 + p]
+    const int page = (tb + 1) * 8 <= kAttPageCache ? pages[tb * 8 + p]
                                                    : __ldg(kv.block_table + (size_t)seq * kv.max_pages_per_seq + pi);
     const long long row = ((((long long)layer * kv.n_pages + page) * 2 + which) * kv.n_kv_heads + x.h) * 16;
-    // claim the entry's stage(s): every lane waits (same flow), lane 0 announces
+    // claim the key stage and the value stage: every lane waits (same flow), lane 0 announces
     uint32_t dst = 0, bar = 0;
-    for (int st = 0; st < rg.spe; ++st) {
+    for (int st = 0; st < 2; ++st) {
       if (pos.r > 0 && !a5_wait(rg, &rg.empty[pos.s], (uint32_t)(pos.r - 1) & 1u, 1, pos.r)) return false;
       const uint32_t b_st = att_smem_u32(&rg.full[pos.s]);
-      const uint32_t d_st = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
-      if (pl_lane == 0) {
-        att_mbar_expect_tx(b_st, rg.spe == 2 ? kA5Part : 2 * kA5Part);
+      if (lane == 0) {
+        att_mbar_expect_tx(b_st, kA5Part);
         att_mbar_arrive(b_st);   // the stage's second arrival
       }
-      if (rg.spe == 1) { bar = b_st; dst = d_st + (uint32_t)which * kA5Part; }
-      else if (st == which) { bar = b_st; dst = d_st; }
+      if (st == which) {
+        bar = b_st;
+        dst = att_smem_u32(rg.base + (size_t)pos.s * rg.stage_stride);
+      }
       pos.next(rg.stages);
     }
-    att_tma_2d(dst + (uint32_t)(half * 8192 + p * 2048), tmKV, bar, half * 64, (int)row);
+    att_tma_2d(dst + (uint32_t)(half * 16384 + p * 2048), tmKV, bar, half * 64, (int)row);
   }
   return true;
 }
 
-// One thread per query plane (0: hi, 1: lo): S_plane = Q_plane K^T of the block's tiles.  gt: tiles of earlier layers
-// (the barriers' phases run on across layers), segs: segments of earlier layers; both advanced.
-__device__ __forceinline__ bool a5_issue_qk(const A5Ring& rg, A5Pos& pos, A5Bars* ab, uint32_t tmem, uint32_t q_area, int nq,
-                                            int plane, const AttPlan& pl, int B, long long t_lo, long long t_hi, int& gt,
-                                            int& segs) {
-  const uint32_t id_s = instr_desc_bf16_mn(kA5Keys, 0);
+// One thread per tile parity X: the score MMAs and the output MMAs of the block's tiles g with g % 2 == X.  gt: tiles of
+// earlier layers (the barriers' phases run on across layers), segs: segments of earlier layers; both advanced.
+__device__ __forceinline__ bool a5_issue(const A5Ring& rg, A5Pos& pos, A5Bars* ab, uint32_t tmem, uint32_t q_area, int nq, int X,
+                                         const AttPlan& pl, int B, long long t_lo, long long t_hi, int& gt, int& segs) {
+  const uint32_t id_s = instr_desc_bf16_mn(kA5Keys, 0), id_o = instr_desc_bf16_mn(128, 1);
   const uint32_t hs = (uint32_t)a5_q_half_bytes(nq);
+  const uint64_t dq = smem_desc_sw128(q_area), dql = smem_desc_sw128(q_area + 2 * hs);
+  const uint64_t q_half = (uint64_t)(hs >> 4), k_half = (uint64_t)(16384 >> 4);   // start-address field, 16-byte units
+  const uint32_t d_s = tmem + (uint32_t)(128 * X), d_o = tmem + (uint32_t)(256 + 128 * X);
   long long t = t_lo;
   while (t < t_hi) {
     const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
     const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    // every segment's queries are waited for, also where this thread owns none of its tiles: a parity wait that
+    // skipped a phase would be satisfied one phase early
     if (!a5_wait(rg, &ab->q_ready, (uint32_t)segs & 1u, 2, segs)) return false;
     tc_fence_after();
+    bool first = true;
     for (int i = 0; i < n; ++i) {
-      const int g = gt + i, sb = g & 1;
+      const int g = gt + i;
       const A5Entry e = a5_entry(rg, pos);
-      // score buffer sb held the probabilities of tile g - 2: its P V (the other issuer's) must have completed
-      if (!a5_wait(rg, &rg.full[e.s0], e.par0, 3, g) ||
-          (g >= 2 && !a5_wait(rg, &ab->o_done[sb], (uint32_t)((g >> 1) - 1) & 1u, 4, g)))
-        return false;
+      if ((g & 1) != X) continue;
+      const uint32_t par = (uint32_t)(g >> 1) & 1u;
+      if (!a5_wait(rg, &rg.full[e.s0], e.par0, 3, g)) return false;
       tc_fence_after();
-      const uint32_t d_s = tmem + (uint32_t)(128 * plane + sb * kA5Keys);
-      const uint64_t dq = smem_desc_sw128(q_area + (uint32_t)plane * 2 * hs), dk = smem_desc_sw128(e.a0);
-      const uint64_t dq_half = (uint64_t)(hs >> 4), dk_half = (uint64_t)(8192 >> 4);   // start-address field, 16-byte units
+      const uint64_t dk = smem_desc_sw128(e.a0);
 #pragma unroll
-      for (int k = 0; k < 8; ++k)
-        tc_mma_bf16(d_s, dq + (k >> 2) * dq_half + 2 * (k & 3), dk + (k >> 2) * dk_half + 2 * (k & 3), id_s, k > 0 ? 1u : 0u);
-      tc_commit(att_smem_u32(&ab->s_full[sb]));   // the output issuer frees the stage
+      for (int k = 0; k < 8; ++k) {
+        const uint64_t ko = (uint64_t)(k >> 2) * k_half + (uint64_t)(2 * (k & 3)), qo = (uint64_t)(k >> 2) * q_half + (uint64_t)(2 * (k & 3));
+        tc_mma_bf16(d_s, dq + qo, dk + ko, id_s, k > 0 ? 1u : 0u);
+        tc_mma_bf16(d_s, dql + qo, dk + ko, id_s, 1u);
+      }
+      tc_commit(att_smem_u32(&rg.empty[e.s0]));
+      tc_commit(att_smem_u32(&ab->s_full[X]));
+      if (!a5_wait(rg, &ab->p_full[X], par, 5, g) || !a5_wait(rg, &rg.full[e.s1], e.par1, 6, g)) return false;
+      tc_fence_after();
+      const uint64_t dv = smem_desc_mn_sw128(e.a1, 16384u);
+#pragma unroll
+      for (int pg = 0; pg < 8; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
+        const uint64_t db = dv + (uint64_t)(pg * (2048 >> 4));
+        const uint32_t pa = d_s + (uint32_t)(32 * (pg >> 1) + 8 * (pg & 1));
+        tc_mma_bf16_ta(d_o, pa, db, id_o, (!first || pg > 0) ? 1u : 0u);
+        tc_mma_bf16_ta(d_o, pa + 16, db, id_o, 1u);
+      }
+      tc_commit(att_smem_u32(&rg.empty[e.s1]));
+      tc_commit(att_smem_u32(&ab->o_done[X]));
+      first = false;
     }
     gt += n;
     t += n;
     ++segs;
-  }
-  return true;
-}
-
-// One thread: O += P V of the block's tiles.
-__device__ __forceinline__ bool a5_issue_pv(const A5Ring& rg, A5Pos& pos, A5Bars* ab, uint32_t tmem, const AttPlan& pl, int B,
-                                            long long t_lo, long long t_hi, int& gt) {
-  const uint32_t id_o = instr_desc_bf16_mn(128, 1);
-  long long t = t_lo;
-  while (t < t_hi) {
-    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
-    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-    for (int i = 0; i < n; ++i) {
-      const int g = gt + i, sb = g & 1;
-      const A5Entry e = a5_entry(rg, pos);
-      if (!a5_wait(rg, &ab->p_full[sb], (uint32_t)(g >> 1) & 1u, 5, g) || !a5_wait(rg, &rg.full[e.s1], e.par1, 6, g)) return false;
-      tc_fence_after();
-      const uint32_t pb = tmem + (uint32_t)(sb * kA5Keys);
-      const uint64_t dv = smem_desc_mn_sw128(e.a1, 8192u);
-#pragma unroll
-      for (int pg = 0; pg < 4; ++pg) {   // the 16 keys of page pg: P's 32-column chunk pg / 2 holds [hi 16 | lo 16]
-        const uint64_t db = dv + (uint64_t)(pg * (2048 >> 4));
-        const uint32_t pa = pb + (uint32_t)(32 * (pg >> 1) + 8 * (pg & 1));
-        tc_mma_bf16_ta(tmem + 256, pa, db, id_o, (i > 0 || pg > 0) ? 1u : 0u);
-        tc_mma_bf16_ta(tmem + 256, pa + 16, db, id_o, 1u);
-      }
-      // both score chains of this tile completed before its probabilities were written: the key part is free too
-      if (rg.spe == 2) tc_commit(att_smem_u32(&rg.empty[e.s0]));
-      tc_commit(att_smem_u32(&rg.empty[e.s1]));
-      tc_commit(att_smem_u32(&ab->o_done[sb]));
-    }
-    gt += n;
-    t += n;
   }
   return true;
 }
@@ -673,14 +650,14 @@ __device__ __forceinline__ uint32_t a5_q_off(int row, int dim, uint32_t hs) {
 }
 
 // The softmax side: four warps, two threads per query row.  quarter (0, 1): the TMEM lane quarter == rows
-// [32 * quarter, +32); half (0, 1): keys [32 * half, +32) of every tile and dims [64 * half, +64) of the row's queries
-// and output.  mx: [2][2][64] floats of shared memory; pair_bar: a shared-memory barrier of the quarter's 64 threads (count 64;
-// every wait is bounded, so a warp that gives up cannot strand its partner), pair_n: its phases so far.
+// [32 * quarter, +32); half (0, 1): keys [64 * half, +64) of every tile and dims [64 * half, +64) of the row's queries
+// and output.  mx: [2][2][64] floats of shared memory; pair_bar: a shared-memory barrier of the quarter's 64 threads
+// (count 64; every wait is bounded, so a warp that gives up cannot strand its partner), pair_n: its phases so far.
 // slot0: the partial slot of the block's segment is slot0 + b * Hkv + h (sub-partial 0).
 // ev: optional timeline of the block's last segment (global-timer ns), stamped by the first softmax warp:
 // [0] queries delivered, [1] last tile's probabilities delivered, [2] partial stored, [3] first scores seen.
-__device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_t tmem, uint8_t* q_area, float* mx, uint64_t* pair_bar, int& pair_n,
-                                           const AttArgs& a, const AttPlan& pl, int B, int Hkv, int nq, long long t_lo,
+__device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_t tmem, uint8_t* q_area, float* mx, uint64_t* pair_bar,
+                                           int& pair_n, const AttArgs& a, const AttPlan& pl, int B, int Hkv, int nq, long long t_lo,
                                            long long t_hi, int& gt, int slot0, int quarter, int half, int lane,
                                            unsigned long long* ev = nullptr) {
   constexpr int HD = 128;
@@ -697,20 +674,17 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
     ++pair_n;
     return __all_sync(0xffffffffu, ok);
   };
-  long long t = t_lo;
-  while (t < t_hi) {
-    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
-    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
-    // queries of this (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16
-    // terms.  The previous segment's score MMAs have completed: this thread saw the s_full of its last tile.
+  // queries of a (sequence, KV head): fp16 (plus what its rounding dropped, in the two-term layers) -> two bf16 terms;
+  // this thread converts its half of the head dimension (all loads first)
+  auto deliver_q = [&](const AttTile& x) {
     if (active) {
-      const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD;
-      const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD : nullptr;
+      const __half* qh = a.Qb + (((size_t)x.b * Hkv + x.h) * nq + q) * HD + 64 * half;
+      const __half* ql = a.Qlo ? a.Qlo + (((size_t)x.b * Hkv + x.h) * nq + q) * HD + 64 * half : nullptr;
       uint4 raw[8], rawl[8];
 #pragma unroll
-      for (int d8 = 0; d8 < 8; ++d8) {   // all loads first
-        raw[d8] = __ldcg(reinterpret_cast<const uint4*>(qh + 64 * half + 8 * d8));
-        rawl[d8] = ql ? __ldcg(reinterpret_cast<const uint4*>(ql + 64 * half + 8 * d8)) : make_uint4(0, 0, 0, 0);
+      for (int d8 = 0; d8 < 8; ++d8) {
+        raw[d8] = __ldcg(reinterpret_cast<const uint4*>(qh + 8 * d8));
+        rawl[d8] = ql ? __ldcg(reinterpret_cast<const uint4*>(ql + 8 * d8)) : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
       for (int d8 = 0; d8 < 8; ++d8) {
@@ -736,6 +710,14 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read these generic-proxy stores
     att_mbar_arrive(att_smem_u32(&ab->q_ready));
+  };
+  long long t = t_lo;
+  bool first_seg = true;
+  while (t < t_hi) {
+    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
+    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    if (first_seg) deliver_q(x);   // later segments' queries were delivered while the segment before them ended
+    first_seg = false;
     if (stamp) ev[0] = att_timer_ns();
     float m_used = -INFINITY, l_sum = 0.f;
     for (int i = 0; i < n; ++i) {
@@ -748,28 +730,23 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
       if (stamp && i == 0) ev[3] = att_timer_ns();
       att_mbar_try(att_smem_u32(&ab->s_full[sb]), par);   // every lane observes the completed phase
       tc_fence_after();
-      const uint32_t s_addr = lane_addr + (uint32_t)(sb * kA5Keys + 32 * half);
-      const int n_valid = min(kA5Keys, x.L - (x.ti + i) * kA5Keys) - 32 * half;   // this thread's keys >= n_valid are masked
-      float sc[32];
-      {
-        float lo[32];
-        tc_ld32_nowait(s_addr, sc);
-        tc_ld32_nowait(s_addr + 128, lo);
-        tc_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) sc[j] += lo[j];
-      }
+      const uint32_t s_addr = lane_addr + (uint32_t)(sb * 128 + 64 * half);
+      const int n_valid = min(kA5Keys, x.L - (x.ti + i) * kA5Keys) - 64 * half;   // this thread's keys >= n_valid are masked
+      float sc[64];
+      tc_ld32_nowait(s_addr, sc);
+      tc_ld32_nowait(s_addr + 32, sc + 32);
+      tc_wait_ld();
       if (!active) {   // a row slot without a query holds whatever its lane computed: keep it from moving the stabiliser
 #pragma unroll
-        for (int j = 0; j < 32; ++j) sc[j] = 0.f;
+        for (int j = 0; j < 64; ++j) sc[j] = 0.f;
       }
-      if (n_valid < 32) {   // warp-uniform; only a sequence's last tile
+      if (n_valid < 64) {   // warp-uniform; only a sequence's last tile
 #pragma unroll
-        for (int j = 0; j < 32; ++j) sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
+        for (int j = 0; j < 64; ++j) sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
       }
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains: a single one is 32 dependent steps
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+      for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
       float m_tile = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       mx_own[128 * sb] = m_tile;
       if (!pair_sync()) return false;
@@ -779,8 +756,9 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
       if (m_used == -INFINITY) m_new = m_tile;
       else if (m_tile > m_used + 8.f) { m_new = m_tile; f = ex2_approx(m_used - m_new); }
       if (i > 0 && __any_sync(0xffffffffu, f != 1.f)) {
-        // rescale this thread's half of its row of O: only once the previous tile's P V has completed (this
-        // tile's cannot start before every thread has delivered its P)
+        // rescale this thread's half of its row of both output accumulators: the previous tile's, once its P V has
+        // completed (this tile's cannot start before every thread has delivered its P), and, from the segment's third
+        // tile on, this tile's own (its last P V completed before the scores just read were computed: same issuer)
         const uint32_t po = (uint32_t)((g - 1) >> 1) & 1u;
         if (lane == 0) ok = a5_wait(rg, &ab->o_done[(g - 1) & 1], po, 8, g) ? 1 : 0;
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -788,48 +766,61 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
         att_mbar_try(att_smem_u32(&ab->o_done[(g - 1) & 1]), po);
         tc_fence_after();
 #pragma unroll 1
-        for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
-          float o[32];
-          tc_ld32(lane_addr + 256 + c0, o);
+        for (int k = 0; k < (i >= 2 ? 2 : 1); ++k) {
+          const uint32_t o_addr = lane_addr + (uint32_t)(256 + 128 * ((g - 1 + k) & 1));
+#pragma unroll 1
+          for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
+            float o[32];
+            tc_ld32(o_addr + c0, o);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] *= f;
-          tc_st32f(lane_addr + 256 + c0, o);
+            for (int j = 0; j < 32; ++j) o[j] *= f;
+            tc_st32f(o_addr + c0, o);
+          }
         }
+        tc_wait_st();
         l_sum *= f;
       }
-      // probabilities as two bf16 terms over the scores: [hi 16 columns | lo 16 columns]; hi = p truncated to bf16,
-      // lo = the rest rounded to bf16 (16 significant bits in all)
-      {
+      // probabilities as two bf16 terms over the scores: chunk of 32 keys -> [hi 16 columns | lo 16 columns]; hi = p
+      // truncated to bf16, lo = the rest rounded to bf16 (16 significant bits in all)
+      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 32) {
         uint32_t hi[16], lo[16];
-        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
-          const float p0 = ex2_approx(sc[j] - m_new), p1 = ex2_approx(sc[j + 1] - m_new);   // 0 for masked keys
+          const float p0 = ex2_approx(sc[c0 + j] - m_new), p1 = ex2_approx(sc[c0 + j + 1] - m_new);   // 0 for masked keys
           ls4[(j >> 1) & 3] += p0 + p1;
           const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
           hi[j >> 1] = __byte_perm(b0, b1, 0x7632);
           const __nv_bfloat162 bl = __floats2bfloat162_rn(p0 - __uint_as_float(b0 & 0xffff0000u), p1 - __uint_as_float(b1 & 0xffff0000u));
           lo[j >> 1] = *reinterpret_cast<const uint32_t*>(&bl);
         }
-        l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-        tc_st16(s_addr, hi);
-        tc_st16(s_addr + 16, lo);
+        tc_st16(s_addr + (uint32_t)c0, hi);
+        tc_st16(s_addr + (uint32_t)c0 + 16, lo);
       }
+      l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       tc_wait_st();
       tc_fence_before();
       att_mbar_arrive(att_smem_u32(&ab->p_full[sb]));
       m_used = m_new;
     }
     if (stamp) ev[1] = att_timer_ns();
-    // the segment's partial: wait for the last P V, then (m, l, o) of every real query row
+    // The next segment's queries, before this one is wound up: every score MMA of this segment has completed (this
+    // thread saw the scores of its last tile), so the query area is free, and the issuers start on the next segment's
+    // scores while the partial below is read out (its first P V waits for probabilities that this thread delivers only
+    // afterwards, so the output accumulators are not touched early).
+    if (t + n < t_hi) deliver_q(att_locate(pl, B, kA5Keys, (int)(t + n)));
+    // the segment's partial: wait for the last P V of either issuer, then (m, l, o) of every real query row
     {
       const int g = gt + n - 1;
-      const uint32_t po = (uint32_t)(g >> 1) & 1u;
       int ok = 1;
-      if (lane == 0) ok = a5_wait(rg, &ab->o_done[g & 1], po, 9, g) ? 1 : 0;
+      if (lane == 0)
+        ok = (a5_wait(rg, &ab->o_done[g & 1], (uint32_t)(g >> 1) & 1u, 9, g) &&
+              (n < 2 || a5_wait(rg, &ab->o_done[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, 9, g))) ? 1 : 0;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) return false;
-      att_mbar_try(att_smem_u32(&ab->o_done[g & 1]), po);
+      att_mbar_try(att_smem_u32(&ab->o_done[g & 1]), (uint32_t)(g >> 1) & 1u);
+      if (n >= 2) att_mbar_try(att_smem_u32(&ab->o_done[(g - 1) & 1]), (uint32_t)((g - 1) >> 1) & 1u);
       tc_fence_after();
       mx_own[128 * ((g + 1) & 1)] = l_sum;   // the buffer the last tile did not use
       if (!pair_sync()) return false;
@@ -842,7 +833,13 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
 #pragma unroll 1
       for (int c0 = 64 * half; c0 < 64 * half + 64; c0 += 32) {
         float o[32];
-        tc_ld32(lane_addr + 256 + c0, o);
+        tc_ld32(lane_addr + (uint32_t)(256 + 128 * (g & 1)) + c0, o);
+        if (n >= 2) {   // the other issuer's accumulator holds the other half of the segment's tiles
+          float o2[32];
+          tc_ld32(lane_addr + (uint32_t)(256 + 128 * ((g - 1) & 1)) + c0, o2);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] += o2[j];
+        }
         if (active) {
           float4* dst = reinterpret_cast<float4*>(a.P.o + (base + q) * HD + c0);
 #pragma unroll

@@ -744,7 +744,10 @@ template <> struct AttVec<2> {
 // dims a lane holds per sub-partial are one 8-byte load and all sub-partials of a config-3 item (39) are in
 // flight at once; with one warp per item they need two dependent batches.
 template <int HD> struct AttCombineSplit { static constexpr int value = HD >= 128 ? 2 : 1; };
-template <typename T, int HD>
+// OBN: output rows one lane keeps in flight (0: 40 or 24, sized for the 30..40 sub-partials of short tiles; 8 where long
+// tiles leave an item a handful of sub-partials: the clamped repeats of the last row would be most of the pass's L2
+// traffic)
+template <typename T, int HD, int OBN = 0>
 __device__ __forceinline__ void att_combine_item(const AttPartials& P, const AttPlan& pl, const AttGeom& g, int G_att,
                                                  int n_tail_base, int Hkv, int item_part, void* ATT, int R, int Hq, int lane,
                                                  unsigned long long* ev = nullptr) {
@@ -775,7 +778,7 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
     return (long long)(cc + 1) * pl.T / G_att > (long long)cc * pl.T / G_att;
   };
   constexpr int DPL = HD / 32 / SPLIT;   // dims per lane
-  constexpr int OB = DPL <= 2 ? 40 : 24;   // output rows whose loads one lane keeps in flight
+  constexpr int OB = OBN > 0 ? OBN : (DPL <= 2 ? 40 : 24);   // output rows whose loads one lane keeps in flight
   constexpr int RS = HD / DPL;             // row stride of the outputs in units of V
   typedef typename AttVec<DPL>::type V;
   const V* Po = reinterpret_cast<const V*>(P.o) + part * 32 + lane;   // row r of the outputs starts at Po + r * RS
@@ -842,7 +845,7 @@ __device__ __forceinline__ void att_combine_item(const AttPartials& P, const Att
 // keys_per_tile > 0: the partials come from a pass that cut the cache into tiles of that many keys (plus tile_pad empty
 // ones per (sequence, KV head)) with one sub-partial per block segment (the tcgen05 attention); 0: this file's own
 // geometry.
-template <int HD>
+template <int HD, int OBN>
 __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dims dm, AttPartials P, int G_att,
                                   int n_tail_base, int keys_per_tile, int tile_pad) {
   __shared__ AttPlan pl;
@@ -856,7 +859,7 @@ __global__ void k_attn_combine_tc(const StepArgs* __restrict__ args, Work w, Dim
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, wpb = blockDim.x >> 5;
   const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;
   for (int item = warp * gridDim.x + blockIdx.x; item < items; item += gridDim.x * wpb)   // spread over blocks first
-    att_combine_item<bf16, HD>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, w.ATT, B * rows, dm.Hq, lane);
+    att_combine_item<bf16, HD, OBN>(P, pl, g, G_att, n_tail_base, dm.Hkv, item, w.ATT, B * rows, dm.Hq, lane);
 }
 
 }  // namespace sj

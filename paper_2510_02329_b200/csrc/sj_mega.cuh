@@ -28,8 +28,8 @@
 //   LM head -> softmax statistics per (vocabulary tile, row), logit of the drafted token
 // Attention: its cache tiles travel through the same ring.  Two implementations, chosen per launch: fp16 mma.sync in
 // the worker warps (sj_attn_tc.cuh), or -- head dimension 128, at most 64 query rows per KV head and sequence --
-// tcgen05 (the routines at the end of sj_attn_t5.cuh): warps 1 and 2 issue the score MMAs, warp 3 the output MMAs, four
-// worker warps run the softmax on tensor memory, the other four the causal tails; the queries sit in an area of their own
+// tcgen05 (the routines at the end of sj_attn_t5.cuh; ring stages of at least 32 KiB): warps 1 and 2 issue the MMAs of
+// the even and the odd 128-key tiles, four worker warps run the softmax on tensor memory, the other four the causal tails; the queries sit in an area of their own
 // after the ring, the accumulators alias the GEMM phases' tensor-memory columns.
 //
 // Every wait is bounded; the first one to run out raises a device-wide abort word that all other waits
@@ -94,7 +94,6 @@ struct MegaParams {
   int* abort_g;               // device-wide abort word        }
   int n_tail_base;
   int att_precise_layers;     // layers [0, n) run the attention with two-term (hi + lo fp16) queries and probabilities
-  int att_spe;                // tcgen05 attention: ring stages per 64-key tile (1: keys and values share a stage, 2: one each)
   int q_area_bytes;           // tcgen05 attention: bytes of the query area between the ring and the control block
   // optional timeline (global-timer nanoseconds), block `trace_block`:
   //   [2k], [2k+1]                      arrival at / release from device-wide barrier k (k >= 1)
@@ -979,7 +978,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctl->tmem_full[i]), 1);
       mbar_init(smem_u32(&ctl->tmem_empty[i]), kMegaWorkers);
-      mbar_init(smem_u32(&ctl->a5.s_full[i]), 2);
+      mbar_init(smem_u32(&ctl->a5.s_full[i]), 1);
       mbar_init(smem_u32(&ctl->a5.p_full[i]), 128);
       mbar_init(smem_u32(&ctl->a5.o_done[i]), 1);
       mbar_init(smem_u32(&ctl->a5_pair[i]), 64);
@@ -1024,8 +1023,8 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
 
   const AttPlan& pl = ctl->plan;
   const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
-  const int n_att = (int)(t_hi - t_lo) * (A5 ? p.att_spe : 1);   // ring stages of one attention phase
-  const A5Ring a5r{ctl->full, ctl->empty, ring, p.stage_bytes, NS, p.att_spe, &ctl->abort_flag, p.abort_g, w.status};
+  const int n_att = (int)(t_hi - t_lo) * (A5 ? 2 : 1);   // ring stages of one attention phase (tcgen05: key stage, value stage)
+  const A5Ring a5r{ctl->full, ctl->empty, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status};
   att_fill_pages(ctl->att_pages, pl, kv, args, B, g.KPS, t_lo, t_hi, threadIdx.x, blockDim.x);
   __syncthreads();
   auto stage_addr = [&](int s) -> uint32_t { return smem_u32(ring + (size_t)s * p.stage_bytes); };
@@ -1038,10 +1037,10 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kMegaRegsLight));
   if (warp == 0) {
     // ------------------------------ weight / cache-tile producer ------------------------------
-    // One lane; sixteen with the tcgen05 attention, whose cache tiles are sixteen small copies each (one per lane, one
+    // One lane; all 32 with the tcgen05 attention, whose cache tiles are 32 small copies each (one per lane, one
     // instruction per tile).  All lanes run the same control flow and wait on the same barriers; lane 0 alone announces
     // bytes and issues the weight copies.
-    if (lane < (A5 ? 16 : 1)) {
+    if (lane < (A5 ? 32 : 1)) {
       const uint64_t pol_w = l2_policy_evict_first();
       RingPos rp{0, 0, NS};
       int sidx = 0;
@@ -1157,7 +1156,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         if constexpr (A5) {
           if (!alive) return;
           A5Pos ap{rp.s, rp.r};
-          alive = a5_issue_qk(a5r, ap, &ctl->a5, tmem_base, smem_u32(q_area), g.nq, 0, pl, B, t_lo, t_hi, a5_tiles, a5_segs);
+          alive = a5_issue(a5r, ap, &ctl->a5, tmem_base, smem_u32(q_area), g.nq, 0, pl, B, t_lo, t_hi, a5_tiles, a5_segs);
           rp.s = ap.s;
           rp.r = ap.r;
         } else {
@@ -1213,18 +1212,17 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       int a5_tiles = 0, a5_segs = 0;
       auto fatt = [&](int l) {
         if constexpr (A5) {
-          // the attention's other two issuers: warp 2 the scores of the lo query plane, warp 3 the output MMAs
-          if (!alive) return;
-          A5Pos ap{rp.s, rp.r};
-          if (mine == 0)
-            alive = a5_issue_qk(a5r, ap, &ctl->a5, ctl->tmem_base, smem_u32(q_area), g.nq, 1, pl, B, t_lo, t_hi, a5_tiles, a5_segs);
-          else
-            alive = a5_issue_pv(a5r, ap, &ctl->a5, ctl->tmem_base, pl, B, t_lo, t_hi, a5_tiles);
-          rp.s = ap.s;
-          rp.r = ap.r;
-        } else {
-          rp.advance(n_att);
+          // warp 2 issues the attention MMAs of the odd tiles (warp 1 those of the even ones)
+          if (mine == 0) {
+            if (!alive) return;
+            A5Pos ap{rp.s, rp.r};
+            alive = a5_issue(a5r, ap, &ctl->a5, ctl->tmem_base, smem_u32(q_area), g.nq, 1, pl, B, t_lo, t_hi, a5_tiles, a5_segs);
+            rp.s = ap.s;
+            rp.r = ap.r;
+            return;
+          }
         }
+        rp.advance(n_att);
       };
       mega_walk(p, fsite, fatt);
     }
@@ -1287,7 +1285,7 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
         const AttPartials P{w.tc_m, w.tc_l, w.tc_o};
         const int items = B * dm.Hkv * g.nq * AttCombineSplit<HD>::value;
         for (int item = ww * G + c; item < items; item += G * 8)   // spread over blocks first
-          att_combine_item<bf16, HD>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane,
+          att_combine_item<bf16, HD, A5 ? 8 : 0>(P, pl, g, G, p.n_tail_base, dm.Hkv, item, w.ATT, R, dm.Hq, lane,
                                      (kTr && p.trace && c == 0 && ww == 0 && (l - p.l0) * 4 < kMegaTraceSites)
                                          ? p.trace + 2 * kMegaTraceBarriers + 8 * kMegaTraceSites + (size_t)(l - p.l0) * 4 * 8 + 4
                                          : nullptr);

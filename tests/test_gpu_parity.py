@@ -379,17 +379,18 @@ def test_tcgen05_attention(name, shape, kv_lens, gamma):
         case.close()
 
 
+# at least 49 block rows each: the persistent kernel's ring stages then hold a 32 KiB key or value tile
 A5_CASES = [
-    ("llama-8b-cut2", synth.LLAMA_8B.cut(2), [210, 4096], 8),                  # config 3 widths, two sequences: 18 rows
-    ("llama-8b-cut1-edges", synth.LLAMA_8B.cut(1), [1, 63, 64, 65, 0, 129], 4),  # 64-key tile edges; an empty cache
-    ("llama-8b-cut1-g10", synth.LLAMA_8B.cut(1), [3000], 10),                  # 44 query rows
-    ("qwen-32b-cut1", synth.QWEN_32B.cut(1), [40, 1300, 515], 8),              # group 5 (45 query rows), qkv bias, 36 KiB ring stages
+    ("llama-8b-cut2-b6", synth.LLAMA_8B.cut(2), [4096, 210, 1, 129, 128, 777], 8),       # config 3 widths; 36 query rows
+    ("llama-8b-cut1-edges", synth.LLAMA_8B.cut(1), [1, 63, 64, 65, 0, 127, 128, 129, 255, 256, 257, 300], 4),  # tile edges; an empty cache
+    ("llama-8b-cut2-g10", synth.LLAMA_8B.cut(2), [3000, 500, 40, 1000, 2000], 10),      # 44 query rows
+    ("qwen-32b-cut1-b8", synth.QWEN_32B.cut(1), [40, 1300, 515, 2048, 1, 900, 128, 3000], 8),  # group 5 (45 query rows), qkv bias, 36 KiB stages
 ]
 
 
 @pytest.mark.parametrize("name,shape,kv_lens,gamma", A5_CASES, ids=[c[0] for c in A5_CASES])
 def test_tcgen05_attention_in_persistent_kernel(name, shape, kv_lens, gamma):
-    """The persistent kernel's tcgen05 attention phase (64-key tiles through the shared ring, three issuing threads),
+    """The persistent kernel's tcgen05 attention phase (128-key tiles through the shared ring, two issuing threads),
     forced on whatever the cache lengths, against the oracle and against the mma.sync phase on the same inputs."""
     case = harness.Case(shape, torch.bfloat16, kv_lens, gamma, seed=8, cache="fill",
                         gen_device="cuda").gpu_setup(max_rows=len(kv_lens) * (gamma + 1))
