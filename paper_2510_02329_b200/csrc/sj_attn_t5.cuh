@@ -732,22 +732,18 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
       tc_fence_after();
       const uint32_t s_addr = lane_addr + (uint32_t)(sb * 128 + 64 * half);
       const int n_valid = min(kA5Keys, x.L - (x.ti + i) * kA5Keys) - 64 * half;   // this thread's keys >= n_valid are masked
-      float sc[64];
-      tc_ld32_nowait(s_addr, sc);
-      tc_ld32_nowait(s_addr + 32, sc + 32);
-      tc_wait_ld();
-      if (!active) {   // a row slot without a query holds whatever its lane computed: keep it from moving the stabiliser
-#pragma unroll
-        for (int j = 0; j < 64; ++j) sc[j] = 0.f;
-      }
-      if (n_valid < 64) {   // warp-uniform; only a sequence's last tile
-#pragma unroll
-        for (int j = 0; j < 64; ++j) sc[j] = (j < n_valid) ? sc[j] : -INFINITY;
-      }
+      // Two passes over the thread's 64 scores, 32 at a time (the maximum first, then the probabilities): tensor memory
+      // is cheap to read twice, and 64 scores held in registers beside the epilogues' state made the kernel spill.
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+      for (int c0 = 0; c0 < 64; c0 += 32) {
+        float sc[32];
+        tc_ld32(s_addr + (uint32_t)c0, sc);
 #pragma unroll
-      for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+        for (int j = 0; j < 32; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], (c0 + j < n_valid) ? sc[j] : -INFINITY);
+      }
       float m_tile = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      if (!active) m_tile = 0.f;   // a row slot without a query holds whatever its lane computed: keep it from moving the stabiliser
       mx_own[128 * sb] = m_tile;
       if (!pair_sync()) return false;
       m_tile = fmaxf(m_tile, mx_other[128 * sb]);
@@ -783,12 +779,18 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
       // probabilities as two bf16 terms over the scores: chunk of 32 keys -> [hi 16 columns | lo 16 columns]; hi = p
       // truncated to bf16, lo = the rest rounded to bf16 (16 significant bits in all)
       float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
+#pragma unroll 1
       for (int c0 = 0; c0 < 64; c0 += 32) {
+        float sc[32];
+        tc_ld32(s_addr + (uint32_t)c0, sc);
+        if (c0 + 32 > n_valid) {   // warp-uniform; only in a sequence's last tile
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sc[j] = (c0 + j < n_valid) ? sc[j] : -INFINITY;
+        }
         uint32_t hi[16], lo[16];
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
-          const float p0 = ex2_approx(sc[c0 + j] - m_new), p1 = ex2_approx(sc[c0 + j + 1] - m_new);   // 0 for masked keys
+          const float p0 = ex2_approx(sc[j] - m_new), p1 = ex2_approx(sc[j + 1] - m_new);   // 0 for masked keys
           ls4[(j >> 1) & 3] += p0 + p1;
           const uint32_t b0 = __float_as_uint(p0), b1 = __float_as_uint(p1);
           hi[j >> 1] = __byte_perm(b0, b1, 0x7632);
