@@ -505,6 +505,7 @@ constexpr int kA5Keys = 128;
 constexpr int kA5MaxRows = 64;
 constexpr uint32_t kA5Part = 32768;   // bytes of a key tile or a value tile: the least a ring stage must hold
 constexpr int kA5TmemCols = 512;
+constexpr int kA5Pad = 3;   // empty tiles the plan counts per (sequence, KV head), see AttPlan::pad
 
 struct A5Bars {
   uint64_t s_full[2];   // one arrival: issuer X's commit after the score MMAs
@@ -560,10 +561,10 @@ __device__ __forceinline__ bool a5_produce(const A5Ring& rg, A5Pos& pos, const C
                                            const StepArgs* __restrict__ args, const AttPlan& pl, int B, int layer,
                                            long long t_lo, long long t_hi, const int* pages, int lane) {
   const int which = lane >> 4, half = (lane >> 3) & 1, p = lane & 7;
-  int tb = 0;
-  for (long long t = t_lo; t < t_hi; ++t, ++tb) {
+  for (long long t = t_lo; t < t_hi; ++t) {
     const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
-    const int seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16;
+    if (x.ti >= x.nt_real) continue;   // one of the plan's empty tiles: no ring entry
+    const int seq = args->seq_ids[x.b], last_page = (x.L - 1) / 16, tb = (int)(t - t_lo);
     int pi = x.ti * 8 + p;
     if (pi > last_page) pi = last_page;   // keys there are masked; reload a valid page
     const int page = (tb + 1) * 8 <= kAttPageCache ? pages[tb * 8 + p]
@@ -601,7 +602,10 @@ __device__ __forceinline__ bool a5_issue(const A5Ring& rg, A5Pos& pos, A5Bars* a
   long long t = t_lo;
   while (t < t_hi) {
     const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
-    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    const int nv = (int)min((long long)(x.nt_b - x.ti), t_hi - t);   // with the plan's empty tiles
+    const int n = max(0, min(nv, x.nt_real - x.ti));
+    t += nv;
+    if (n == 0) continue;   // only empty tiles of this (sequence, KV head): no segment
     // every segment's queries are waited for, also where this thread owns none of its tiles: a parity wait that
     // skipped a phase would be satisfied one phase early
     if (!a5_wait(rg, &ab->q_ready, (uint32_t)segs & 1u, 2, segs)) return false;
@@ -638,7 +642,6 @@ __device__ __forceinline__ bool a5_issue(const A5Ring& rg, A5Pos& pos, A5Bars* a
       first = false;
     }
     gt += n;
-    t += n;
     ++segs;
   }
   return true;
@@ -711,11 +714,30 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read these generic-proxy stores
     att_mbar_arrive(att_smem_u32(&ab->q_ready));
   };
+  // the block's run of real tiles at tile t: (sequence, KV head, first tile), its length n, and nv, the same with the
+  // plan's empty tiles; n == 0 when only empty tiles of that (sequence, KV head) fell to this block
+  auto run_at = [&](long long t, AttTile& x, int& n, int& nv) {
+    x = att_locate(pl, B, kA5Keys, (int)t);
+    nv = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    n = max(0, min(nv, x.nt_real - x.ti));
+  };
   long long t = t_lo;
   bool first_seg = true;
   while (t < t_hi) {
-    const AttTile x = att_locate(pl, B, kA5Keys, (int)t);
-    const int n = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+    AttTile x;
+    int n, nv;
+    run_at(t, x, n, nv);
+    if (n == 0) {
+      // the combine pass still reads the block's slot for this (sequence, KV head): a partial of weight zero (the
+      // stored outputs are finite: old values or zeros)
+      const size_t base = (((size_t)slot0 + (size_t)x.b * Hkv + x.h) * kAttMaxSub + 0) * (size_t)nq;
+      if (active && half == 0) {
+        a.P.m[base + q] = -INFINITY;
+        a.P.l[base + q] = 0.f;
+      }
+      t += nv;
+      continue;
+    }
     if (first_seg) deliver_q(x);   // later segments' queries were delivered while the segment before them ended
     first_seg = false;
     if (stamp) ev[0] = att_timer_ns();
@@ -811,7 +833,16 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
     // thread saw the scores of its last tile), so the query area is free, and the issuers start on the next segment's
     // scores while the partial below is read out (its first P V waits for probabilities that this thread delivers only
     // afterwards, so the output accumulators are not touched early).
-    if (t + n < t_hi) deliver_q(att_locate(pl, B, kA5Keys, (int)(t + n)));
+    for (long long t2 = t + nv; t2 < t_hi;) {
+      AttTile x2;
+      int n2, nv2;
+      run_at(t2, x2, n2, nv2);
+      if (n2 > 0) {
+        deliver_q(x2);
+        break;
+      }
+      t2 += nv2;
+    }
     // the segment's partial: wait for the last P V of either issuer, then (m, l, o) of every real query row
     {
       const int g = gt + n - 1;
@@ -853,7 +884,7 @@ __device__ __forceinline__ bool a5_softmax(const A5Ring& rg, A5Bars* ab, uint32_
       if (stamp) ev[2] = att_timer_ns();
     }
     gt += n;
-    t += n;
+    t += nv;
   }
   return true;
 }

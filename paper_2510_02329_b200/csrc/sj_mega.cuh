@@ -991,11 +991,11 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
       const int L = kv.kv_len[args->seq_ids[b]];
       ctl->plan.L[b] = L;
       ctl->plan.pre[b] = acc;
-      acc += dm.Hkv * ((L + g.KPS - 1) / g.KPS);
+      acc += L > 0 ? dm.Hkv * ((L + g.KPS - 1) / g.KPS + (A5 ? kA5Pad : 0)) : 0;
     }
     ctl->plan.pre[B] = acc;
     ctl->plan.T = acc;
-    ctl->plan.pad = 0;
+    ctl->plan.pad = A5 ? kA5Pad : 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -1023,7 +1023,18 @@ k_verify_mega(const __grid_constant__ MegaMaps mp, const MegaParams p, const Ste
 
   const AttPlan& pl = ctl->plan;
   const long long t_lo = (long long)c * pl.T / G, t_hi = (long long)(c + 1) * pl.T / G;
-  const int n_att = (int)(t_hi - t_lo) * (A5 ? 2 : 1);   // ring stages of one attention phase (tcgen05: key stage, value stage)
+  // ring stages of one attention phase: one per tile, or (tcgen05) a key stage and a value stage per real tile
+  int n_att = (int)(t_hi - t_lo);
+  if constexpr (A5) {
+    int n_real = 0;
+    for (long long t = t_lo; t < t_hi;) {
+      const AttTile x = att_locate(pl, B, g.KPS, (int)t);
+      const int nv = (int)min((long long)(x.nt_b - x.ti), t_hi - t);
+      n_real += max(0, min(nv, x.nt_real - x.ti));
+      t += nv;
+    }
+    n_att = 2 * n_real;
+  }
   const A5Ring a5r{ctl->full, ctl->empty, ring, p.stage_bytes, NS, &ctl->abort_flag, p.abort_g, w.status};
   att_fill_pages(ctl->att_pages, pl, kv, args, B, g.KPS, t_lo, t_hi, threadIdx.x, blockDim.x);
   __syncthreads();
